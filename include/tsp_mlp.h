@@ -1,0 +1,146 @@
+/*
+ * tsp_mlp.h - C ABI of the B200 (sm_100a) TSP gated ring MLP library.
+ *
+ * The library computes the per-rank work of the TSP gated ring MLP (Algorithm 2 of
+ * "Folding Tensor and Sequence Parallelism ...") for all D ranks on ONE GPU: rank r
+ * owns token rows [r*S/D, (r+1)*S/D) of X and, at ring step t, applies weight shard
+ * k = (r - t) mod D:   Y_r += (silu(X_r Wg_k) * (X_r Wu_k)) Wd_k,   t = 0..D-1.
+ * The ring transfer itself is absent (all shards are resident); the ring only fixes
+ * the order in which each rank's fp32 accumulator meets the shards.
+ *
+ * Conventions for every entry point
+ *   - All matrix arguments are DEVICE pointers unless the name ends in _host.
+ *     Row-major, bf16 (2 bytes) unless stated; 16-byte aligned.
+ *       X, Y, dY, dX : [S, H]            rank r = rows [r*S/D, (r+1)*S/D)
+ *       Wg, Wu       : [D][H][F/D]       shard k = gate/up columns k*F/D .. (k+1)*F/D
+ *       Wd           : [D][F/D][H]       shard k = down rows       k*F/D .. (k+1)*F/D
+ *       dWg, dWu, dWd: same shapes as the weights, FP32, overwritten (not accumulated)
+ *   - The caller owns every buffer, including the workspace.  The library owns only
+ *     the plan (host tables, tensor maps, a 4-byte device status word, profiling events).
+ *     tsp_mlp_forward / tsp_mlp_backward allocate nothing.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream).  Argument and launch errors are returned at once; a device
+ *     wait that ran out of time is reported by tsp_mlp_status after a synchronize.
+ *   - No exceptions, no abort, no CPU fallback.  Unsupported shapes are refused before
+ *     any launch.  Supported: H % 256 == 0, (F/D) % 128 == 0, (S/D) % 128 == 0, F % D == 0,
+ *     S % D == 0, 1 <= D <= 64.
+ *   - A plan must not be used from two host threads at once, nor on two streams at
+ *     once (the workspace and status word are shared).
+ *   - Results are deterministic: no atomics, fixed accumulation order.
+ */
+#ifndef TSP_MLP_H
+#define TSP_MLP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tsp_mlp_plan tsp_mlp_plan_t; /* opaque; created by tsp_mlp_plan, owned by the library */
+
+typedef enum {
+    TSP_OK = 0,
+    TSP_ERR_INVALID_ARG = -1,        /* null pointer, misaligned pointer, D differs from the plan, S <= 0 */
+    TSP_ERR_UNSUPPORTED_SHAPE = -2,  /* divisibility rules above not met */
+    TSP_ERR_UNSUPPORTED_DEVICE = -3, /* current device is not compute capability 10.x */
+    TSP_ERR_CUDA = -4,               /* a CUDA runtime / driver call failed (see tsp_mlp_last_cuda_error) */
+    TSP_ERR_WORKSPACE = -5,          /* workspace missing or smaller than tsp_mlp_workspace_bytes */
+    TSP_ERR_DEVICE_TIMEOUT = -6      /* a bounded device-side wait expired; outputs are invalid */
+} tsp_status_t;
+
+/* Which passes a workspace must serve. */
+#define TSP_WS_FORWARD 0
+#define TSP_WS_BACKWARD 1
+
+/*
+ * tsp_mlp_plan - validate (H, F, D) for the current device and build a plan.
+ * Follows the inputs of Algorithm 2: hidden size H, intermediate width F (the paper's
+ * F*h), world size D.  *out receives the plan; release it with tsp_mlp_plan_destroy.
+ * Allocates a 4-byte device status word.  Errors: INVALID_ARG, UNSUPPORTED_SHAPE,
+ * UNSUPPORTED_DEVICE, CUDA.
+ */
+tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out);
+tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan);
+
+/*
+ * Workspace: scratch for the bf16 intermediate A = silu(G)*U [S,F] (forward) and for
+ * A, dG, dU [S,F] each (backward).  tsp_mlp_workspace_bytes returns the size needed
+ * for S tokens (`pass` = TSP_WS_FORWARD or TSP_WS_BACKWARD; backward covers forward);
+ * 0 on bad arguments.  tsp_mlp_set_workspace hands a caller-owned device buffer
+ * (256-byte aligned) to the plan; it must stay valid while calls using it are in flight.
+ */
+size_t tsp_mlp_workspace_bytes(const tsp_mlp_plan_t* plan, int64_t S, int pass);
+tsp_status_t tsp_mlp_set_workspace(tsp_mlp_plan_t* plan, void* dev_ptr, size_t bytes);
+
+/*
+ * tsp_mlp_forward - Algorithm 2 for all D ranks: Y = (silu(X Wg) * (X Wu)) Wd with
+ * each rank's fp32 accumulator visiting the shards in ring order k = (r - t) mod D.
+ * Two kernels: gate|up GEMM with the SwiGLU epilogue (G, U live only in tensor memory,
+ * A is rounded once to bf16), then the down projection accumulated in tensor memory
+ * over all D shards with one bf16 store of Y.  `D` must equal the plan's.
+ */
+tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu,
+                             const void* Wd, void* Y, int64_t S, int D, void* cuda_stream);
+
+/*
+ * tsp_mlp_backward - gradients of the forward above for upstream dY (the backward
+ * pass mirrors the forward weight movement; the partial weight gradients every rank
+ * produces for shard k are summed to the owner, Sections 4.3.4 and 4.7).  G and U are
+ * recomputed from X; dA = dY Wd^T; dU = dA*silu(G); dG = dA*U*silu'(G); A, dG, dU are
+ * rounded once to bf16 into the workspace.  dX [S,H] bf16 accumulates over shards in
+ * ring order; dWg, dWu [D][H][F/D] and dWd [D][F/D][H] are fp32 and contract over all S
+ * tokens, rank order r = (k + t) mod D.
+ */
+tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu,
+                              const void* Wd, const void* dY, void* dX, float* dWg, float* dWu,
+                              float* dWd, int64_t S, int D, void* cuda_stream);
+
+/*
+ * tsp_mlp_forward_host - the same forward for callers whose tensors live in HOST
+ * memory (pinned memory gives asynchronous copies).  Copies X, Wg, Wu, Wd to device
+ * staging inside the workspace, runs tsp_mlp_forward, copies Y back; all on
+ * `cuda_stream`.  Needs a workspace of tsp_mlp_workspace_bytes_host(plan, S) bytes.
+ */
+size_t tsp_mlp_workspace_bytes_host(const tsp_mlp_plan_t* plan, int64_t S);
+tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, const void* Wg_host,
+                                  const void* Wu_host, const void* Wd_host, void* Y_host,
+                                  int64_t S, int D, void* cuda_stream);
+
+/*
+ * tsp_mlp_status - synchronizes nothing; reads (and clears) the plan's device status
+ * word with a blocking 4-byte copy.  Call after synchronizing the stream.  Returns
+ * TSP_OK or TSP_ERR_DEVICE_TIMEOUT (or TSP_ERR_CUDA if the copy failed).
+ */
+tsp_status_t tsp_mlp_status(tsp_mlp_plan_t* plan);
+
+/* Static, never-null description of a status code. */
+const char* tsp_mlp_error_string(tsp_status_t status);
+/* The cudaError_t / CUresult value of the last failed CUDA call on this plan (0 if none). */
+int tsp_mlp_last_cuda_error(const tsp_mlp_plan_t* plan);
+
+/*
+ * tsp_mlp_ring_order - fill table[r*D + t] with the shard rank r uses at ring step t
+ * (Algorithm 2: send to (p+1) mod D, receive from (p-1) mod D).  Host pointer, D*D ints.
+ */
+tsp_status_t tsp_mlp_ring_order(const tsp_mlp_plan_t* plan, int* table_host);
+
+/*
+ * Per-kernel timing.  tsp_mlp_profile_begin makes the plan record CUDA events on the
+ * caller's stream around each kernel of the next `max_calls` forward/backward calls
+ * (creates events; no device memory).  After synchronizing, tsp_mlp_profile_read
+ * returns for call `call_index` the number of kernels and their durations in ms
+ * (`ms_out` holds up to 8 floats; order: launch order).  tsp_mlp_profile_end frees the events.
+ */
+tsp_status_t tsp_mlp_profile_begin(tsp_mlp_plan_t* plan, int max_calls);
+tsp_status_t tsp_mlp_profile_read(tsp_mlp_plan_t* plan, int call_index, int* n_kernels_out, float* ms_out);
+tsp_status_t tsp_mlp_profile_end(tsp_mlp_plan_t* plan);
+
+/* Number of kernels one forward (pass=TSP_WS_FORWARD) or backward call launches. */
+int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSP_MLP_H */

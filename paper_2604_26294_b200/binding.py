@@ -1,0 +1,184 @@
+"""ctypes binding of libtsp_mlp.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs inside the CUDA library.  If the library is missing the
+functions raise; there is no fallback of any kind.  Tensors are torch CUDA tensors
+(torch is used for device memory and streams only) or, for ``*_host`` calls, host
+tensors / numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+TSP_OK = 0
+TSP_ERR_INVALID_ARG = -1
+TSP_ERR_UNSUPPORTED_SHAPE = -2
+TSP_ERR_UNSUPPORTED_DEVICE = -3
+TSP_ERR_CUDA = -4
+TSP_ERR_WORKSPACE = -5
+TSP_ERR_DEVICE_TIMEOUT = -6
+TSP_WS_FORWARD = 0
+TSP_WS_BACKWARD = 1
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtsp_mlp.so")
+
+# name -> (restype, argtypes); mirrors include/tsp_mlp.h
+_P = ctypes.c_void_p
+SIGNATURES = {
+    "tsp_mlp_plan": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(_P)]),
+    "tsp_mlp_plan_destroy": (ctypes.c_int, [_P]),
+    "tsp_mlp_workspace_bytes": (ctypes.c_size_t, [_P, ctypes.c_int64, ctypes.c_int]),
+    "tsp_mlp_workspace_bytes_host": (ctypes.c_size_t, [_P, ctypes.c_int64]),
+    "tsp_mlp_set_workspace": (ctypes.c_int, [_P, _P, ctypes.c_size_t]),
+    "tsp_mlp_forward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_mlp_forward_host": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_mlp_backward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_mlp_status": (ctypes.c_int, [_P]),
+    "tsp_mlp_error_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "tsp_mlp_last_cuda_error": (ctypes.c_int, [_P]),
+    "tsp_mlp_ring_order": (ctypes.c_int, [_P, ctypes.POINTER(ctypes.c_int)]),
+    "tsp_mlp_profile_begin": (ctypes.c_int, [_P, ctypes.c_int]),
+    "tsp_mlp_profile_read": (ctypes.c_int, [_P, ctypes.c_int, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]),
+    "tsp_mlp_profile_end": (ctypes.c_int, [_P]),
+    "tsp_mlp_kernels_per_call": (ctypes.c_int, [_P, ctypes.c_int]),
+}
+
+_lib = None
+
+
+class TspError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        msg = f"{where}: {error_string(code)} ({code})"
+        if detail:
+            msg += f" [{detail}]"
+        super().__init__(msg)
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libtsp_mlp.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with __graft_entry__.build() "
+                "(python -m paper_2604_26294_b200.build); there is no CPU fallback")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def tsp_mlp_error_string(code: int) -> str:
+    return load_library().tsp_mlp_error_string(code).decode()
+
+
+error_string = tsp_mlp_error_string
+
+
+def _ptr(t) -> int:
+    """Address of a torch tensor's / numpy array's first element; None -> 0."""
+    if t is None:
+        return 0
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    if hasattr(t, "ctypes"):
+        return t.ctypes.data
+    return int(t)
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream
+    if hasattr(stream, "cuda_stream"):
+        return stream.cuda_stream
+    return int(stream)
+
+
+def _check(code: int, where: str, plan=None):
+    if code != TSP_OK:
+        detail = ""
+        if plan is not None and code == TSP_ERR_CUDA:
+            detail = f"cuda error {load_library().tsp_mlp_last_cuda_error(plan)}"
+        raise TspError(code, where, detail)
+
+
+# --------------------------------------------------------------------------- C ABI, same names
+def tsp_mlp_plan(H: int, F: int, D: int):
+    """Create a plan for hidden H, intermediate width F, D shards on the current device."""
+    out = ctypes.c_void_p()
+    _check(load_library().tsp_mlp_plan(H, F, D, ctypes.byref(out)), "tsp_mlp_plan")
+    return out
+
+
+def tsp_mlp_plan_destroy(plan) -> None:
+    _check(load_library().tsp_mlp_plan_destroy(plan), "tsp_mlp_plan_destroy")
+
+
+def tsp_mlp_workspace_bytes(plan, S: int, backward: int = TSP_WS_FORWARD) -> int:
+    return int(load_library().tsp_mlp_workspace_bytes(plan, S, backward))
+
+
+def tsp_mlp_workspace_bytes_host(plan, S: int) -> int:
+    return int(load_library().tsp_mlp_workspace_bytes_host(plan, S))
+
+
+def tsp_mlp_set_workspace(plan, buf, nbytes: int | None = None) -> None:
+    if nbytes is None:
+        nbytes = buf.numel() * buf.element_size()
+    _check(load_library().tsp_mlp_set_workspace(plan, _ptr(buf), nbytes), "tsp_mlp_set_workspace")
+
+
+def tsp_mlp_forward(plan, X, Wg, Wu, Wd, Y, S: int, D: int, stream=None) -> None:
+    _check(load_library().tsp_mlp_forward(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(Y), S, D,
+                                          _stream_handle(stream)), "tsp_mlp_forward", plan)
+
+
+def tsp_mlp_forward_host(plan, X, Wg, Wu, Wd, Y, S: int, D: int, stream=None) -> None:
+    _check(load_library().tsp_mlp_forward_host(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(Y), S, D,
+                                               _stream_handle(stream)), "tsp_mlp_forward_host", plan)
+
+
+def tsp_mlp_backward(plan, X, Wg, Wu, Wd, dY, dX, dWg, dWu, dWd, S: int, D: int, stream=None) -> None:
+    _check(load_library().tsp_mlp_backward(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(dY), _ptr(dX),
+                                           _ptr(dWg), _ptr(dWu), _ptr(dWd), S, D, _stream_handle(stream)),
+           "tsp_mlp_backward", plan)
+
+
+def tsp_mlp_status(plan) -> int:
+    """Device status word as a status code (TSP_OK or TSP_ERR_DEVICE_TIMEOUT); does not raise."""
+    return int(load_library().tsp_mlp_status(plan))
+
+
+def tsp_mlp_last_cuda_error(plan) -> int:
+    return int(load_library().tsp_mlp_last_cuda_error(plan))
+
+
+def tsp_mlp_ring_order(plan, D: int):
+    table = (ctypes.c_int * (D * D))()
+    _check(load_library().tsp_mlp_ring_order(plan, table), "tsp_mlp_ring_order")
+    return [[table[r * D + t] for t in range(D)] for r in range(D)]
+
+
+def tsp_mlp_profile_begin(plan, max_calls: int) -> None:
+    _check(load_library().tsp_mlp_profile_begin(plan, max_calls), "tsp_mlp_profile_begin", plan)
+
+
+def tsp_mlp_profile_read(plan, call_index: int):
+    n = ctypes.c_int()
+    ms = (ctypes.c_float * 8)()
+    _check(load_library().tsp_mlp_profile_read(plan, call_index, ctypes.byref(n), ms), "tsp_mlp_profile_read", plan)
+    return [float(ms[i]) for i in range(n.value)]
+
+
+def tsp_mlp_profile_end(plan) -> None:
+    _check(load_library().tsp_mlp_profile_end(plan), "tsp_mlp_profile_end")
+
+
+def tsp_mlp_kernels_per_call(plan, backward: int = TSP_WS_FORWARD) -> int:
+    return int(load_library().tsp_mlp_kernels_per_call(plan, backward))

@@ -1,0 +1,413 @@
+// C-ABI of the TSP gated ring MLP library: plan, shape checks, tensor-map encoding, launches.
+// Every step of the path runs in the kernels of fwd_kernels.cuh / bwd_kernels.cuh; this file only
+// validates, encodes TMA descriptors and enqueues.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/tsp_mlp.h"
+#include "bwd_kernels.cuh"
+#include "fwd_kernels.cuh"
+
+namespace {
+
+using tsp::GateUpParams;
+using tsp::DownParams;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kMaxKernelsPerCall = 8;
+
+struct ProfileCall {
+    cudaEvent_t ev[kMaxKernelsPerCall + 1];
+    int n_kernels;
+};
+
+}  // namespace
+
+struct tsp_mlp_plan {
+    int H, F, D;
+    int device;
+    int sm_count;
+    int max_smem;
+    int* status_dev;
+    void* workspace;
+    size_t workspace_bytes;
+    int last_cuda_error;
+    unsigned long long timeout_ns;
+    EncodeTiledFn encode;
+    std::vector<ProfileCall> profile;
+    int profile_next;
+};
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+tsp_status_t cuda_fail(tsp_mlp_plan_t* plan, int err) {
+    if (plan) plan->last_cuda_error = err;
+    return TSP_ERR_CUDA;
+}
+
+// 3-D bf16 tensor map with 128-byte swizzle: dims (d0 innermost, d1, d2), byte strides of d1 and d2.
+bool encode_map(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, CUtensorMapDataType dtype, size_t elem,
+                uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1, uint64_t stride2, uint32_t box0,
+                uint32_t box1) {
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {stride1, stride2};
+    cuuint32_t box[3] = {box0, box1, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    (void)elem;
+    CUresult r = plan->encode(map, dtype, 3, const_cast<void*>(base), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        plan->last_cuda_error = static_cast<int>(r);
+        return false;
+    }
+    return true;
+}
+
+// [rows, cols] row-major bf16 matrix viewed as (cols, rows, 1).
+bool encode_matrix(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box0,
+                   uint32_t box1) {
+    return encode_map(plan, map, base, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, cols, rows, 1, cols * 2, rows * cols * 2,
+                      box0, box1);
+}
+// [D][rows][cols] row-major bf16 viewed as (cols, rows, D).
+bool encode_sharded(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, uint64_t D, uint64_t rows, uint64_t cols,
+                    uint32_t box0, uint32_t box1) {
+    return encode_map(plan, map, base, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, cols, rows, D, cols * 2, rows * cols * 2,
+                      box0, box1);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+tsp_status_t check_call(const tsp_mlp_plan_t* plan, int64_t S, int D) {
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    if (D != plan->D || S <= 0) return TSP_ERR_INVALID_ARG;
+    if (S % D != 0 || (S / D) % 128 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (S > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    return TSP_OK;
+}
+
+int pick_stages(const tsp_mlp_plan_t* plan, size_t stage_bytes, int want) {
+    const size_t fixed = sizeof(tsp::SharedCtl) + 1024;
+    int s = want;
+    while (s > 2 && s * stage_bytes + fixed > static_cast<size_t>(plan->max_smem)) --s;
+    return s;
+}
+
+struct Profiler {
+    tsp_mlp_plan_t* plan;
+    cudaStream_t stream;
+    ProfileCall* call;
+    int n;
+    Profiler(tsp_mlp_plan_t* p, cudaStream_t s) : plan(p), stream(s), call(nullptr), n(0) {
+        if (p->profile_next < static_cast<int>(p->profile.size())) {
+            call = &p->profile[p->profile_next++];
+            call->n_kernels = 0;
+            cudaEventRecord(call->ev[0], stream);
+        }
+    }
+    void mark() {
+        if (call && n < kMaxKernelsPerCall) {
+            ++n;
+            cudaEventRecord(call->ev[n], stream);
+            call->n_kernels = n;
+        }
+    }
+};
+
+// ---------------------------------------------------------------------------------------------
+// launches
+// ---------------------------------------------------------------------------------------------
+tsp_status_t launch_gate_up(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A, int64_t S,
+                            cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
+    GateUpParams p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    p.A = static_cast<__nv_bfloat16*>(A);
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.m_blocks = static_cast<int>(S / 128);
+    p.blocks_per_rank = static_cast<int>(S / D / 128);
+    p.jl_blocks = F_d / 128;
+    const int band_cap = static_cast<int>((64ull << 20) / (128ull * H * 2));
+    p.band = band_cap < 1 ? 1 : (band_cap > p.m_blocks ? p.m_blocks : band_cap);
+    p.num_tiles = p.m_blocks * D * p.jl_blocks;
+    p.stages = pick_stages(plan, 48 * 1024, 4);
+    p.status = plan->status_dev;
+    p.timeout_ns = plan->timeout_ns;
+    const size_t smem = p.stages * 48 * 1024 + sizeof(tsp::SharedCtl) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(tsp::gate_up_swiglu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
+    tsp::gate_up_swiglu_kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
+}
+
+tsp_status_t launch_down(tsp_mlp_plan_t* plan, const void* A, const void* Wd, void* Y, int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D;
+    DownParams p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_a, A, S, F, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 64)) return TSP_ERR_CUDA;
+    p.Y = static_cast<__nv_bfloat16*>(Y);
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.m_blocks = static_cast<int>(S / 128);
+    p.n_blocks = H / 256;
+    p.blocks_per_rank = static_cast<int>(S / D / 128);
+    p.group = p.m_blocks < 16 ? p.m_blocks : 16;
+    p.num_tiles = p.m_blocks * p.n_blocks;
+    p.stages = pick_stages(plan, 48 * 1024, 4);
+    p.status = plan->status_dev;
+    p.timeout_ns = plan->timeout_ns;
+    const size_t smem = p.stages * 48 * 1024 + sizeof(tsp::SharedCtl) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(tsp::down_accumulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
+    tsp::down_accumulate_kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------------------------
+extern "C" {
+
+tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
+    if (!out) return TSP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (H <= 0 || F <= 0 || D <= 0 || D > 64) return TSP_ERR_INVALID_ARG;
+    if (F % D != 0 || (F / D) % 128 != 0 || H % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (H > (1 << 20) || F > (1 << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return TSP_ERR_CUDA;
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) return TSP_ERR_CUDA;
+    if (prop.major != 10) return TSP_ERR_UNSUPPORTED_DEVICE;
+
+    tsp_mlp_plan_t* plan = new (std::nothrow) tsp_mlp_plan_t();
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    plan->H = H; plan->F = F; plan->D = D;
+    plan->device = dev;
+    plan->sm_count = prop.multiProcessorCount;
+    plan->max_smem = static_cast<int>(prop.sharedMemPerBlockOptin);
+    plan->status_dev = nullptr;
+    plan->workspace = nullptr;
+    plan->workspace_bytes = 0;
+    plan->last_cuda_error = 0;
+    plan->profile_next = 0;
+    plan->timeout_ns = 2000ull * 1000 * 1000;
+    if (const char* t = std::getenv("TSP_MLP_TIMEOUT_MS")) {
+        const long ms = std::atol(t);
+        if (ms > 0) plan->timeout_ns = static_cast<unsigned long long>(ms) * 1000 * 1000;
+    }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
+        delete plan;
+        return TSP_ERR_CUDA;
+    }
+    plan->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    e = cudaMalloc(reinterpret_cast<void**>(&plan->status_dev), sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(plan->status_dev, 0, sizeof(int));
+    if (e != cudaSuccess) {
+        if (plan->status_dev) cudaFree(plan->status_dev);
+        delete plan;
+        return TSP_ERR_CUDA;
+    }
+    *out = plan;
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan) {
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    tsp_mlp_profile_end(plan);
+    if (plan->status_dev) cudaFree(plan->status_dev);
+    delete plan;
+    return TSP_OK;
+}
+
+size_t tsp_mlp_workspace_bytes(const tsp_mlp_plan_t* plan, int64_t S, int pass) {
+    if (!plan || S <= 0 || (pass != TSP_WS_FORWARD && pass != TSP_WS_BACKWARD)) return 0;
+    const size_t one = align_up(static_cast<size_t>(S) * plan->F * 2, 256);
+    return pass == TSP_WS_BACKWARD ? 3 * one : one;
+}
+
+size_t tsp_mlp_workspace_bytes_host(const tsp_mlp_plan_t* plan, int64_t S) {
+    if (!plan || S <= 0) return 0;
+    const size_t a = align_up(static_cast<size_t>(S) * plan->F * 2, 256);
+    const size_t x = align_up(static_cast<size_t>(S) * plan->H * 2, 256);
+    const size_t w = align_up(static_cast<size_t>(plan->H) * plan->F * 2, 256);
+    return a + 2 * x + 3 * w;
+}
+
+tsp_status_t tsp_mlp_set_workspace(tsp_mlp_plan_t* plan, void* dev_ptr, size_t bytes) {
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return TSP_ERR_INVALID_ARG;
+    plan->workspace = dev_ptr;
+    plan->workspace_bytes = dev_ptr ? bytes : 0;
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
+                             void* Y, int64_t S, int D, void* cuda_stream) {
+    tsp_status_t st = check_call(plan, S, D);
+    if (st != TSP_OK) return st;
+    if (!X || !Wg || !Wu || !Wd || !Y) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(Y)) return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes(plan, S, TSP_WS_FORWARD))
+        return TSP_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    Profiler prof(plan, stream);
+    st = launch_gate_up(plan, X, Wg, Wu, plan->workspace, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    st = launch_down(plan, plan->workspace, Wd, Y, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, const void* Wg_host, const void* Wu_host,
+                                  const void* Wd_host, void* Y_host, int64_t S, int D, void* cuda_stream) {
+    tsp_status_t st = check_call(plan, S, D);
+    if (st != TSP_OK) return st;
+    if (!X_host || !Wg_host || !Wu_host || !Wd_host || !Y_host) return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_host(plan, S)) return TSP_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t a = align_up(static_cast<size_t>(S) * plan->F * 2, 256);
+    const size_t xb = static_cast<size_t>(S) * plan->H * 2, x = align_up(xb, 256);
+    const size_t wb = static_cast<size_t>(plan->H) * plan->F * 2, w = align_up(wb, 256);
+    uint8_t* base = static_cast<uint8_t*>(plan->workspace);
+    uint8_t* dX = base + a;
+    uint8_t* dY = dX + x;
+    uint8_t* dWg = dY + x;
+    uint8_t* dWu = dWg + w;
+    uint8_t* dWd = dWu + w;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaMemcpyAsync(dWg, Wg_host, wb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaMemcpyAsync(dWu, Wu_host, wb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaMemcpyAsync(dWd, Wd_host, wb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    // The forward proper uses only the first `a` bytes of the workspace.
+    st = tsp_mlp_forward(plan, dX, dWg, dWu, dWd, dY, S, D, cuda_stream);
+    if (st != TSP_OK) return st;
+    if ((e = cudaMemcpyAsync(Y_host, dY, xb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
+                              const void* dY, void* dX, float* dWg, float* dWu, float* dWd, int64_t S, int D,
+                              void* cuda_stream) {
+    tsp_status_t st = check_call(plan, S, D);
+    if (st != TSP_OK) return st;
+    if (!X || !Wg || !Wu || !Wd || !dY || !dX || !dWg || !dWu || !dWd) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(dY) || !aligned16(dX) ||
+        !aligned16(dWg) || !aligned16(dWu) || !aligned16(dWd))
+        return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes(plan, S, TSP_WS_BACKWARD))
+        return TSP_ERR_WORKSPACE;
+    (void)cuda_stream;
+    return TSP_ERR_UNSUPPORTED_SHAPE;  // backward kernels are enabled in bwd_kernels.cuh
+}
+
+tsp_status_t tsp_mlp_status(tsp_mlp_plan_t* plan) {
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    int v = 0;
+    cudaError_t e = cudaMemcpy(&v, plan->status_dev, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    if (v != 0) {
+        plan->last_cuda_error = v;
+        e = cudaMemset(plan->status_dev, 0, sizeof(int));
+        if (e != cudaSuccess) return cuda_fail(plan, e);
+        return TSP_ERR_DEVICE_TIMEOUT;
+    }
+    return TSP_OK;
+}
+
+const char* tsp_mlp_error_string(tsp_status_t s) {
+    switch (s) {
+        case TSP_OK: return "ok";
+        case TSP_ERR_INVALID_ARG: return "invalid argument";
+        case TSP_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case TSP_ERR_UNSUPPORTED_DEVICE: return "unsupported device (needs compute capability 10.x)";
+        case TSP_ERR_CUDA: return "CUDA call failed";
+        case TSP_ERR_WORKSPACE: return "workspace missing or too small";
+        case TSP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int tsp_mlp_last_cuda_error(const tsp_mlp_plan_t* plan) { return plan ? plan->last_cuda_error : 0; }
+
+tsp_status_t tsp_mlp_ring_order(const tsp_mlp_plan_t* plan, int* table_host) {
+    if (!plan || !table_host) return TSP_ERR_INVALID_ARG;
+    const int D = plan->D;
+    for (int r = 0; r < D; ++r)
+        for (int t = 0; t < D; ++t) table_host[r * D + t] = (r - t + D) % D;
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_profile_begin(tsp_mlp_plan_t* plan, int max_calls) {
+    if (!plan || max_calls <= 0 || max_calls > 4096) return TSP_ERR_INVALID_ARG;
+    tsp_mlp_profile_end(plan);
+    plan->profile.resize(max_calls);
+    for (auto& c : plan->profile) {
+        c.n_kernels = 0;
+        for (auto& ev : c.ev) {
+            cudaError_t e = cudaEventCreate(&ev);
+            if (e != cudaSuccess) return cuda_fail(plan, e);
+        }
+    }
+    plan->profile_next = 0;
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_profile_read(tsp_mlp_plan_t* plan, int call_index, int* n_kernels_out, float* ms_out) {
+    if (!plan || !n_kernels_out || !ms_out) return TSP_ERR_INVALID_ARG;
+    if (call_index < 0 || call_index >= plan->profile_next) return TSP_ERR_INVALID_ARG;
+    ProfileCall& c = plan->profile[call_index];
+    *n_kernels_out = c.n_kernels;
+    for (int i = 0; i < c.n_kernels; ++i) {
+        cudaError_t e = cudaEventElapsedTime(&ms_out[i], c.ev[i], c.ev[i + 1]);
+        if (e != cudaSuccess) return cuda_fail(plan, e);
+    }
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_profile_end(tsp_mlp_plan_t* plan) {
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    for (auto& c : plan->profile)
+        for (auto& ev : c.ev) cudaEventDestroy(ev);
+    plan->profile.clear();
+    plan->profile_next = 0;
+    return TSP_OK;
+}
+
+int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass) {
+    if (!plan) return 0;
+    return pass == TSP_WS_BACKWARD ? 3 : 2;
+}
+
+}  // extern "C"
