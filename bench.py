@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the TSP gated ring MLP on B200: TFLOP/s of the sharded gated-MLP path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the path (tsp_mlp_forward, or forward + backward for the `train`
+workload) over one seeded synthetic batch, for all D ranks' token shards and all D weight
+shards on one GPU.  With N > 1 (launched by torch.distributed.run) every GPU runs the same
+single-GPU job on its own seeded batch: no collective is on the data path, so `scaling`
+is "weak" and `value` is the sum over GPUs divided by the slowest GPU's time.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU fp64 oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2604_26294_b200 import inputs as inp  # noqa: E402
+
+METRIC = "sharded gated-MLP TFLOP/s on 1 B200 and % of dense-BF16 tensor-core peak"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel
+# at the named workload, from the ncu capture summarised under profiles/.  None = not captured.
+NCU_DRAM_BYTES = {
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"burst": float(d["bf16_tflops"]), "sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"burst": FALLBACK_BF16_TFLOPS, "sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+# clock sampling during the timed region (read-only NVML queries)
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+        0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+        0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, device_index: int, period_s: float = 0.01):
+        self.period = period_s
+        self.samples = []
+        self.reason_bits = 0
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self._nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"], "samples": 0}
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit and name != "gpu_idle"]
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_seconds(host, rows):
+    """Time the fp64 oracle (as it stands) on `rows` token rows of the workload; returns seconds."""
+    from oracle import tsp_mlp_oracle as orc
+
+    Xs = inp.bf16_bits_to_f64(host.X[rows])
+    t0 = time.perf_counter()
+    orc.gated_mlp_forward(Xs, host._Wg64, host._Wu64, host._Wd64)
+    return time.perf_counter() - t0
+
+
+def prepare_oracle_weights(host):
+    host._Wg64 = inp.bf16_bits_to_f64(host.Wg)
+    host._Wu64 = inp.bf16_bits_to_f64(host.Wu)
+    host._Wd64 = inp.bf16_bits_to_f64(host.Wd)
+
+
+def oracle_baseline(wl, host, target_s=12.0):
+    """Forward oracle on a bounded row sample: calibrate on 64 rows, then size the sample for ~target_s."""
+    prepare_oracle_weights(host)
+    rows = inp.sample_rows(wl.S, wl.D)[:64]
+    t = oracle_sample_seconds(host, rows)
+    per_row = max(t / len(rows), 1e-9)
+    n = int(min(wl.S, max(64, target_s / per_row)))
+    n = max(64, (n // 64) * 64)
+    rows = np.arange(n)
+    t = oracle_sample_seconds(host, rows)
+    flops = 6.0 * n * wl.H * wl.F
+    cores = len(os.sched_getaffinity(0))
+    return {"value": flops / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"fp64 numpy forward of the first {n} of {wl.S} token rows against the full weights "
+                      f"({t:.2f} s; whole workload extrapolates to {t * wl.S / n:.1f} s)",
+            "seconds": t}
+
+
+def run_reference(args, wl):
+    """--impl reference: the CPU oracle on the host cores, rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    host = inp.make_inputs(wl.S, wl.H, wl.F, seed=0)
+    prepare_oracle_weights(host)
+    # size one step to roughly (120 s / (steps + warmup)), at least 64 rows
+    rows64 = np.arange(64)
+    per_row = max(oracle_sample_seconds(host, rows64) / 64, 1e-9)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    n = int(min(wl.S, max(64, (budget / per_row) // 64 * 64)))
+    rows = np.arange(n)
+    for _ in range(args.warmup):
+        oracle_sample_seconds(host, rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_seconds(host, rows)
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    tf = 6.0 * n * wl.H * wl.F / dt / 1e12
+    cores = len(os.sched_getaffinity(0))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tf, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "S": wl.S, "H": wl.H, "F": wl.F, "D": wl.D,
+                   "sample_rows_per_step": n},
+        "cpu_baseline": {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"each step = fp64 numpy forward of the first {n} of {wl.S} token rows"},
+        "e2e": {"value": tf, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+def run_gpu(args, wl):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2604_26294_b200 import binding as b
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    train = wl.name == "train" or args.backward
+    S, H, F, D = wl.S, wl.H, wl.F, wl.D
+    host = inp.make_inputs(S, H, F, seed=rank, with_dy=train)
+
+    def dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    Wg_h, Wu_h, Wd_h = inp.shard_columns(host.Wg, D), inp.shard_columns(host.Wu, D), inp.shard_rows(host.Wd, D)
+    X, Wg, Wu, Wd = dev(host.X), dev(Wg_h), dev(Wu_h), dev(Wd_h)
+    Y = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
+    plan = b.tsp_mlp_plan(H, F, D)
+    ws_bytes = max(b.tsp_mlp_workspace_bytes(plan, S, b.TSP_WS_BACKWARD if train else b.TSP_WS_FORWARD),
+                   b.tsp_mlp_workspace_bytes_host(plan, S))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    b.tsp_mlp_set_workspace(plan, ws)
+    if train:
+        dY = dev(host.dY)
+        dX = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
+        dWg = torch.empty(D, H, F // D, dtype=torch.float32, device="cuda")
+        dWu = torch.empty(D, H, F // D, dtype=torch.float32, device="cuda")
+        dWd = torch.empty(D, F // D, H, dtype=torch.float32, device="cuda")
+
+    def step():
+        b.tsp_mlp_forward(plan, X, Wg, Wu, Wd, Y, S, D)
+        if train:
+            b.tsp_mlp_backward(plan, X, Wg, Wu, Wd, dY, dX, dWg, dWu, dWd, S, D)
+
+    kernels_per_step = b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD) + (
+        b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_BACKWARD) if train else 0)
+    model_flops = wl.forward_flops() + (wl.backward_flops() if train else 0.0)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    assert b.tsp_mlp_status(plan) == b.TSP_OK, "device-side wait timed out during warm-up"
+
+    # ---- timed region: K steps, inputs resident in HBM ----
+    calls_per_step = 2 if train else 1
+    b.tsp_mlp_profile_begin(plan, min(4096, args.steps * calls_per_step))
+    sampler = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    sampler.stop()
+    elapsed_ms = e0.elapsed_time(e1)
+    assert b.tsp_mlp_status(plan) == b.TSP_OK, "device-side wait timed out"
+    # per-kernel durations from the events the library recorded on the launch stream inside the timed region
+    per_kernel = None
+    n_prof = min(4096, args.steps * calls_per_step)
+    fwd_calls = [b.tsp_mlp_profile_read(plan, i) for i in range(0, n_prof, calls_per_step)]
+    per_kernel = np.mean(np.asarray(fwd_calls), axis=0)
+    bwd_kernel = None
+    if train:
+        bwd_calls = [b.tsp_mlp_profile_read(plan, i) for i in range(1, n_prof, calls_per_step)]
+        bwd_kernel = np.mean(np.asarray(bwd_calls), axis=0)
+    b.tsp_mlp_profile_end(plan)
+
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * model_flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: host buffers in pinned memory, H2D + forward + D2H every step ----
+    e2e = None
+    if not train:
+        hX = torch.from_numpy(host.X.view(np.int16)).pin_memory()
+        hWg = torch.from_numpy(Wg_h.view(np.int16)).pin_memory()
+        hWu = torch.from_numpy(Wu_h.view(np.int16)).pin_memory()
+        hWd = torch.from_numpy(Wd_h.view(np.int16)).pin_memory()
+        hY = torch.empty(S, H, dtype=torch.int16).pin_memory()
+        n_e2e = max(2, min(args.steps, 8))
+        for _ in range(2):
+            b.tsp_mlp_forward_host(plan, hX, hWg, hWu, hWd, hY, S, D)
+        barrier()
+        e0.record()
+        for _ in range(n_e2e):
+            b.tsp_mlp_forward_host(plan, hX, hWg, hWu, hWd, hY, S, D)
+            torch.cuda.current_stream().synchronize()  # the caller reads Y on the host
+        e1.record()
+        barrier()
+        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item()) / n_e2e
+        h2d = hX.numel() * 2 + hWg.numel() * 2 + hWu.numel() * 2 + hWd.numel() * 2
+        e2e = {"value": world * model_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(hY.numel() * 2),
+               "ms_per_step": e2e_ms, "steps": n_e2e,
+               "call": "tsp_mlp_forward_host (pinned host X, Wg, Wu, Wd -> host Y)"}
+        # the host path must give the same bits as the device path
+        same = bool((hY.cuda() == Y.view(torch.int16)).all())
+        e2e["matches_device_path"] = same
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    # dominant kernel: the gate|up GEMM with the SwiGLU epilogue (two thirds of the forward FLOPs)
+    gate_up_ms = float(per_kernel[0])
+    gate_up_flops = 4.0 * S * H * F
+    achieved = gate_up_flops / (gate_up_ms * 1e-3) / 1e12
+    roofline = {
+        "bound": "tensor", "kernel": "gate_up_swiglu_kernel", "achieved": achieved, "peak": peaks["burst"],
+        "unit": UNIT, "frac": achieved / peaks["burst"], "peak_source": f"of {peaks['source']} (burst bf16 GEMM)",
+        "frac_of_sustained": achieved / peaks["sustained"], "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
+        "flops_per_launch": gate_up_flops, "ms_per_launch": gate_up_ms,
+        "traffic": NCU_DRAM_BYTES.get(("gate_up_swiglu_kernel", wl.name)),
+        "kernels_ms": {"gate_up_swiglu_kernel": gate_up_ms, "down_accumulate_kernel": float(per_kernel[1])},
+    }
+    if bwd_kernel is not None:
+        roofline["kernels_ms"].update({f"backward_kernel_{i}": float(v) for i, v in enumerate(bwd_kernel)})
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu = oracle_baseline(wl, host)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "pass": "forward+backward" if train else "forward", "S": S, "H": H, "F": F,
+                   "D": D, "tokens_per_rank": S // D, "shard_width": F // D, "model_flops_per_step": model_flops,
+                   "l2": "inputs larger than L2 (X+W = %.0f MB, intermediate %.0f MB)" % (
+                       (2 * S * H + 6 * H * F) / 1e6, 2 * S * F / 1e6),
+                   "parallelism": "all D ranks' shards on one GPU; replicas across GPUs"},
+        "pct_of_measured_bf16_peak": 100.0 * value / world / peaks["burst"],
+        "pct_of_nominal_bf16_peak": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
+        "clocks": sampler.summary(),
+        "e2e": e2e,
+        "gpu_launches": int(args.steps * kernels_per_step),
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    b.tsp_mlp_plan_destroy(plan)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="7b_short", choices=sorted(inp.WORKLOADS))
+    ap.add_argument("--backward", action="store_true", help="time forward + backward (as the `train` workload does)")
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = inp.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_gpu(args, wl)
+
+
+if __name__ == "__main__":
+    main()

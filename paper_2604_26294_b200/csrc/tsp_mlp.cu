@@ -184,6 +184,96 @@ tsp_status_t launch_down(tsp_mlp_plan_t* plan, const void* A, const void* Wd, vo
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
 
+tsp_status_t launch_bwd_gate(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
+                             const void* dY, void* A, void* dG, void* dU, int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
+    tsp::BwdGateParams p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 128)) return TSP_ERR_CUDA;
+    p.A = static_cast<__nv_bfloat16*>(A);
+    p.dG = static_cast<__nv_bfloat16*>(dG);
+    p.dU = static_cast<__nv_bfloat16*>(dU);
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.m_blocks = static_cast<int>(S / 128);
+    p.blocks_per_rank = static_cast<int>(S / D / 128);
+    p.jl_blocks = F_d / 128;
+    const int band_cap = static_cast<int>((32ull << 20) / (128ull * H * 2));
+    p.band = band_cap < 1 ? 1 : (band_cap > p.m_blocks ? p.m_blocks : band_cap);
+    p.num_tiles = p.m_blocks * D * p.jl_blocks;
+    p.stages = pick_stages(plan, 48 * 1024, 4);
+    p.status = plan->status_dev;
+    p.timeout_ns = plan->timeout_ns;
+    const size_t smem = p.stages * 48 * 1024 + sizeof(tsp::SharedCtl) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(tsp::bwd_gate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
+    tsp::bwd_gate_kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
+}
+
+tsp_status_t launch_bwd_dx(tsp_mlp_plan_t* plan, const void* dG, const void* dU, const void* Wg, const void* Wu, void* dX,
+                           int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
+    tsp::BwdDxPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_dg, dG, S, F, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_du, dU, S, F, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 256)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 256)) return TSP_ERR_CUDA;
+    p.dX = static_cast<__nv_bfloat16*>(dX);
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.m_blocks = static_cast<int>(S / 128);
+    p.n_blocks = H / 256;
+    p.blocks_per_rank = static_cast<int>(S / D / 128);
+    p.group = p.m_blocks < 16 ? p.m_blocks : 16;
+    p.num_tiles = p.m_blocks * p.n_blocks;
+    p.stages = pick_stages(plan, 48 * 1024, 4);
+    p.status = plan->status_dev;
+    p.timeout_ns = plan->timeout_ns;
+    const size_t smem = p.stages * 48 * 1024 + sizeof(tsp::SharedCtl) + 1024;
+    auto kernel = tsp::tile_gemm_kernel<tsp::BwdDxPolicy>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
+    kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
+}
+
+tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
+                           const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D;
+    tsp::BwdDwPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_a, A, S, F, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_dg, dG, S, F, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_du, dU, S, F, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 64)) return TSP_ERR_CUDA;
+    p.dWd = dWd; p.dWg = dWg; p.dWu = dWu;
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.j_blocks = F / 128;
+    p.n_blocks = H / 256;
+    p.num_tiles = 3 * p.j_blocks * p.n_blocks;
+    p.stages = pick_stages(plan, 48 * 1024, 4);
+    p.status = plan->status_dev;
+    p.timeout_ns = plan->timeout_ns;
+    const size_t smem = p.stages * 48 * 1024 + sizeof(tsp::SharedCtl) + 1024;
+    auto kernel = tsp::tile_gemm_kernel<tsp::BwdDwPolicy>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
+    kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------
@@ -328,8 +418,23 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
         return TSP_ERR_INVALID_ARG;
     if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes(plan, S, TSP_WS_BACKWARD))
         return TSP_ERR_WORKSPACE;
-    (void)cuda_stream;
-    return TSP_ERR_UNSUPPORTED_SHAPE;  // backward kernels are enabled in bwd_kernels.cuh
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t one = align_up(static_cast<size_t>(S) * plan->F * 2, 256);
+    uint8_t* base = static_cast<uint8_t*>(plan->workspace);
+    void* A = base;
+    void* dG = base + one;
+    void* dU = base + 2 * one;
+    Profiler prof(plan, stream);
+    st = launch_bwd_gate(plan, X, Wg, Wu, Wd, dY, A, dG, dU, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    st = launch_bwd_dx(plan, dG, dU, Wg, Wu, dX, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    st = launch_bwd_dw(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    return TSP_OK;
 }
 
 tsp_status_t tsp_mlp_status(tsp_mlp_plan_t* plan) {
