@@ -56,7 +56,7 @@ def test_more_tiles_than_sms():
 
 
 def test_gradients_agree_across_D():
-    S, H, F = 1024, 512, 2048
+    S, H, F = 2048, 512, 2048
     host = inp.make_inputs(S, H, F, seed=3, with_dy=True)
     outs = {D: _grads(DeviceProblem(S, H, F, D, host=host, with_dy=True)) for D in (1, 2, 4, 8, 16)}
     for D, got in outs.items():

@@ -50,7 +50,7 @@ def test_more_tiles_than_sms():
 
 
 def test_results_agree_across_D():
-    S, H, F = 1024, 512, 2048
+    S, H, F = 2048, 512, 2048
     host = inp.make_inputs(S, H, F, seed=3)
     outs = {}
     for D in (1, 2, 4, 8, 16):

@@ -1,0 +1,111 @@
+"""Parity at the 7B-shaped sizes, in the launch configuration bench.py times.
+
+The fp64 oracle cannot finish these sizes in seconds, so it is evaluated on sampled outputs it can
+compute one by one: token rows of Y / dX (one random row inside every 128-row tile of every rank)
+and intermediate columns of the weight gradients (every shard is hit).
+"""
+import numpy as np
+import pytest
+
+from oracle import tsp_mlp_oracle as orc
+from paper_2604_26294_b200 import build
+from paper_2604_26294_b200 import inputs as inp
+from tests.helpers import DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
+
+pytestmark = pytest.mark.gpu
+
+TOL_ORACLE = 1e-2
+TOL_ACROSS_D = 5e-3
+TOL_ROW = 0.08
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build_library()
+
+
+def _weights64(host):
+    return inp.bf16_bits_to_f64(host.Wg), inp.bf16_bits_to_f64(host.Wu), inp.bf16_bits_to_f64(host.Wd)
+
+
+def _check_forward_rows(prob, Y, rows, w64):
+    import torch
+
+    got = tensor_to_f64(Y[torch.from_numpy(rows).cuda()])
+    ref = orc.forward_rows(inp.bf16_bits_to_f64(prob.host.X[rows]), *w64, np.arange(len(rows)))
+    assert np.all(np.isfinite(got))
+    assert rel_fro(got, ref) <= TOL_ORACLE, rel_fro(got, ref)
+    assert worst_row_error(got, ref) <= TOL_ROW, worst_row_error(got, ref)
+
+
+def test_7b_short_forward_sampled_rows():
+    wl = inp.WORKLOADS["7b_short"]
+    prob = DeviceProblem(wl.S, wl.H, wl.F, wl.D, seed=0)
+    Y = prob.forward()
+    import torch
+
+    assert bool(torch.isfinite(Y.float()).all())
+    _check_forward_rows(prob, Y, inp.sample_rows(wl.S, wl.D), _weights64(prob.host))
+
+
+def test_7b_long_forward_sampled_rows():
+    wl = inp.WORKLOADS["7b_long"]
+    prob = DeviceProblem(wl.S, wl.H, wl.F, wl.D, seed=0)
+    Y = prob.forward()
+    import torch
+
+    assert bool(torch.isfinite(Y.float()).all())
+    _check_forward_rows(prob, Y, inp.sample_rows(wl.S, wl.D), _weights64(prob.host))
+
+
+def test_shard_count_sweep_agrees_and_matches_oracle():
+    import torch
+
+    wl = inp.WORKLOADS["sweep_d1"]
+    host = inp.make_inputs(wl.S, wl.H, wl.F, seed=0)
+    w64 = _weights64(host)
+    rows = inp.sample_rows(wl.S, 16)
+    base = None
+    for D in (1, 2, 4, 8, 16):
+        prob = DeviceProblem(wl.S, wl.H, wl.F, D, host=host)
+        Y = prob.forward().float()
+        _check_forward_rows(prob, prob.Y, rows, w64)
+        if base is None:
+            base = Y.clone()
+        else:
+            diff = float((Y - base).norm() / base.norm())
+            assert diff <= TOL_ACROSS_D, (D, diff)
+        del prob
+        torch.cuda.empty_cache()
+
+
+def test_training_config_backward_sampled():
+    import torch
+
+    wl = inp.WORKLOADS["train"]
+    prob = DeviceProblem(wl.S, wl.H, wl.F, wl.D, seed=0, with_dy=True)
+    dX, dWg, dWu, dWd = prob.backward()
+    for t in (dX, dWg, dWu, dWd):
+        assert bool(torch.isfinite(t.float()).all())
+    host = prob.host
+    Wg64, Wu64, Wd64 = _weights64(host)
+    rows = inp.sample_rows(wl.S, wl.D)
+    ref = orc.backward_rows(inp.bf16_bits_to_f64(host.X[rows]), Wg64, Wu64, Wd64,
+                            inp.bf16_bits_to_f64(host.dY[rows]), np.arange(len(rows)))
+    got = tensor_to_f64(dX[torch.from_numpy(rows).cuda()])
+    assert rel_fro(got, ref) <= TOL_ORACLE, rel_fro(got, ref)
+    assert worst_row_error(got, ref) <= TOL_ROW
+
+    cols = inp.sample_columns(wl.F, wl.D, 64)
+    rWg, rWu, rWd = orc.backward_columns(inp.bf16_bits_to_f64(host.X), Wg64, Wu64, Wd64,
+                                         inp.bf16_bits_to_f64(host.dY), cols)
+    F_d = wl.F_d
+    k_idx = torch.from_numpy(cols // F_d).cuda()
+    j_idx = torch.from_numpy(cols % F_d).cuda()
+    gWg = tensor_to_f64(dWg[k_idx, :, j_idx]).T      # [H, len(cols)]
+    gWu = tensor_to_f64(dWu[k_idx, :, j_idx]).T
+    gWd = tensor_to_f64(dWd[k_idx, j_idx, :])        # [len(cols), H]
+    for name, g, r in (("dWg", gWg, rWg), ("dWu", gWu, rWu), ("dWd", gWd, rWd)):
+        assert g.shape == r.shape, name
+        assert rel_fro(g, r) <= TOL_ORACLE, (name, rel_fro(g, r))
+        assert worst_row_error(g.T if name != "dWd" else g, r.T if name != "dWd" else r) <= TOL_ROW, name
