@@ -188,6 +188,26 @@ def run_reference(args, wl):
 
 
 # ------------------------------------------------------------------------------------------------
+# aggregation over ranks (N > 1: independent replicas, one per GPU)
+# ------------------------------------------------------------------------------------------------
+def max_over_ranks(value_ms: float, world: int, device="cpu") -> float:
+    """Slowest rank's time: all-reduce(MAX) over the default process group (identity for world == 1)."""
+    if world <= 1:
+        return float(value_ms)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(world: int, flops_per_rank_step: float, ms_per_step: float) -> float:
+    """Aggregate over all replicas: every rank does `flops_per_rank_step` in the slowest rank's time."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
+# ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 def run_gpu(args, wl):
@@ -272,12 +292,9 @@ def run_gpu(args, wl):
         bwd_kernel = np.mean(np.asarray(bwd_calls), axis=0)
     b.tsp_mlp_profile_end(plan)
 
-    t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, world, "cuda")
     ms_per_step = elapsed_ms / args.steps
-    value = world * model_flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tflops(world, model_flops, ms_per_step)
 
     # ---- end to end: host buffers in pinned memory, H2D + forward + D2H every step ----
     e2e = None
@@ -297,12 +314,9 @@ def run_gpu(args, wl):
             torch.cuda.current_stream().synchronize()  # the caller reads Y on the host
         e1.record()
         barrier()
-        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item()) / n_e2e
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda") / n_e2e
         h2d = hX.numel() * 2 + hWg.numel() * 2 + hWu.numel() * 2 + hWd.numel() * 2
-        e2e = {"value": world * model_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+        e2e = {"value": whole_job_tflops(world, model_flops, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(hY.numel() * 2),
                "ms_per_step": e2e_ms, "steps": n_e2e,
                "call": "tsp_mlp_forward_host (pinned host X, Wg, Wu, Wd -> host Y)"}
