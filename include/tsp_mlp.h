@@ -47,7 +47,8 @@ typedef enum {
     TSP_ERR_UNSUPPORTED_DEVICE = -3, /* current device is not compute capability 10.x */
     TSP_ERR_CUDA = -4,               /* a CUDA runtime / driver call failed (see tsp_mlp_last_cuda_error) */
     TSP_ERR_WORKSPACE = -5,          /* workspace missing or smaller than tsp_mlp_workspace_bytes */
-    TSP_ERR_DEVICE_TIMEOUT = -6      /* a bounded device-side wait expired; outputs are invalid */
+    TSP_ERR_DEVICE_TIMEOUT = -6,     /* a bounded device-side wait expired; outputs are invalid */
+    TSP_ERR_STATIC_LIMIT = -7        /* tsp_mlp_forward_static: S*F*2 bytes exceed TSP_MLP_STATIC_SCRATCH_BYTES */
 } tsp_status_t;
 
 /* Which passes a workspace must serve. */
@@ -107,6 +108,39 @@ size_t tsp_mlp_workspace_bytes_host(const tsp_mlp_plan_t* plan, int64_t S);
 tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, const void* Wg_host,
                                   const void* Wu_host, const void* Wd_host, void* Y_host,
                                   int64_t S, int D, void* cuda_stream);
+
+/*
+ * tsp_mlp_forward_static - the forward pass for callers that cannot obtain device memory at call time.
+ * (The paper has no counterpart of this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: a plug-in living inside a host framework that has already claimed the whole GPU for its
+ * own pool, so that cudaMalloc fails; code on a latency-critical path that cannot accept the device-wide
+ * synchronisation an allocation implies; deployments whose rules forbid allocating after start-up.  Such
+ * a caller cannot create a plan (the plan allocates a status word) nor hand over a workspace.
+ *
+ * What it does: the same two kernels as tsp_mlp_forward, but the bf16 intermediate A = silu(G)*U [S,F]
+ * and the device status word live in a fixed array compiled into the library
+ * (TSP_MLP_STATIC_SCRATCH_BYTES + 256 bytes of device memory on every GPU that loads the library, held
+ * until the process exits).  The call performs no cudaMalloc / cudaFree and calls no allocating routine.
+ * The caller passes only inputs and outputs, all DEVICE pointers with the layouts given at the top of this
+ * file, plus optionally `timed_out_host`: a HOST int that, after `cuda_stream` has been synchronized,
+ * is 0 if the kernels completed and non-zero if a bounded device-side wait expired (Y is then invalid).
+ * Pass NULL to skip that copy.
+ *
+ * Limits and rules:
+ *   - S * F * 2 bytes must not exceed TSP_MLP_STATIC_SCRATCH_BYTES (8 MiB: e.g. S=1024, F=4096), otherwise
+ *     TSP_ERR_STATIC_LIMIT is returned and nothing is launched.  Shape rules as for tsp_mlp_plan / forward.
+ *   - The first call on each device looks up the array's device address and the device's properties (host
+ *     work only, with that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left in it.  The
+ *     entry point clears the status word on `cuda_stream` before launching; the intermediate is fully
+ *     rewritten before it is read.  Two calls that overlap on the GPU (different streams, or different
+ *     host threads) race on the array: serialize them on one stream.
+ *   - Errors: INVALID_ARG, UNSUPPORTED_SHAPE, UNSUPPORTED_DEVICE, STATIC_LIMIT, CUDA.
+ */
+#define TSP_MLP_STATIC_SCRATCH_BYTES (8u << 20)
+tsp_status_t tsp_mlp_forward_static(int H, int F, int D, const void* X, const void* Wg, const void* Wu,
+                                    const void* Wd, void* Y, int64_t S, int* timed_out_host, void* cuda_stream);
 
 /*
  * tsp_mlp_status - synchronizes nothing; reads (and clears) the plan's device status

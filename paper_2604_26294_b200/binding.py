@@ -17,6 +17,8 @@ TSP_ERR_UNSUPPORTED_DEVICE = -3
 TSP_ERR_CUDA = -4
 TSP_ERR_WORKSPACE = -5
 TSP_ERR_DEVICE_TIMEOUT = -6
+TSP_ERR_STATIC_LIMIT = -7
+TSP_MLP_STATIC_SCRATCH_BYTES = 8 << 20
 TSP_WS_FORWARD = 0
 TSP_WS_BACKWARD = 1
 
@@ -33,6 +35,8 @@ SIGNATURES = {
     "tsp_mlp_forward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_forward_host": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_backward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_mlp_forward_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, _P,
+                                              ctypes.c_int64, ctypes.POINTER(ctypes.c_int), _P]),
     "tsp_mlp_status": (ctypes.c_int, [_P]),
     "tsp_mlp_error_string": (ctypes.c_char_p, [ctypes.c_int]),
     "tsp_mlp_last_cuda_error": (ctypes.c_int, [_P]),
@@ -148,6 +152,18 @@ def tsp_mlp_backward(plan, X, Wg, Wu, Wd, dY, dX, dWg, dWu, dWd, S: int, D: int,
     _check(load_library().tsp_mlp_backward(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(dY), _ptr(dX),
                                            _ptr(dWg), _ptr(dWu), _ptr(dWd), S, D, _stream_handle(stream)),
            "tsp_mlp_backward", plan)
+
+
+def tsp_mlp_forward_static(H: int, F: int, D: int, X, Wg, Wu, Wd, Y, S: int, timed_out=None, stream=None) -> None:
+    """Forward pass that allocates nothing: for callers that cannot get device memory at call time.
+
+    The intermediate lives in a fixed array inside the library (S*F*2 bytes <= TSP_MLP_STATIC_SCRATCH_BYTES).
+    `timed_out`: optional ``ctypes.c_int`` filled (after a stream synchronize) with 0, or non-zero if a
+    device-side wait expired.  Calls that overlap on the GPU race on the shared array.
+    """
+    ref = ctypes.byref(timed_out) if timed_out is not None else None
+    _check(load_library().tsp_mlp_forward_static(H, F, D, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(Y), S, ref,
+                                                 _stream_handle(stream)), "tsp_mlp_forward_static")
 
 
 def tsp_mlp_status(plan) -> int:

@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -274,6 +275,56 @@ tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, 
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Fixed scratch for tsp_mlp_forward_static: part of the library image, so every GPU that loads the
+// library holds these bytes until the process exits.  First 256 bytes: device status word; the rest:
+// the bf16 intermediate A = silu(G)*U [S, F].  In host code the array's name is only a stand-in for
+// the symbol, not a device address: the address is fetched once per device with cudaGetSymbolAddress.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kStaticHeaderBytes = 256;
+constexpr size_t kStaticScratchBytes = TSP_MLP_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticHeaderBytes + kStaticScratchBytes];
+
+struct StaticDeviceState {
+    bool ready;
+    unsigned char* scratch;  // device address of g_static_scratch on this device
+    int sm_count;
+    int max_smem;
+    EncodeTiledFn encode;
+};
+constexpr int kMaxStaticDevices = 64;
+StaticDeviceState g_static_state[kMaxStaticDevices];
+std::mutex g_static_mutex;
+
+// Once per device, with that device current.  Allocates nothing.
+tsp_status_t static_device_setup(int dev, StaticDeviceState** out) {
+    if (dev < 0 || dev >= kMaxStaticDevices) return TSP_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDeviceState& st = g_static_state[dev];
+    if (!st.ready) {
+        int major = 0, sms = 0, smem = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TSP_ERR_CUDA;
+        if (major != 10) return TSP_ERR_UNSUPPORTED_DEVICE;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TSP_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return TSP_ERR_CUDA;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess || !fn)
+            return TSP_ERR_CUDA;
+        unsigned char* ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || !ptr)
+            return TSP_ERR_CUDA;
+        st.scratch = ptr;
+        st.sm_count = sms;
+        st.max_smem = smem;
+        st.encode = reinterpret_cast<EncodeTiledFn>(fn);
+        st.ready = true;
+    }
+    *out = &st;
+    return TSP_OK;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------
@@ -437,6 +488,49 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
     return TSP_OK;
 }
 
+tsp_status_t tsp_mlp_forward_static(int H, int F, int D, const void* X, const void* Wg, const void* Wu,
+                                    const void* Wd, void* Y, int64_t S, int* timed_out_host, void* cuda_stream) {
+    if (H <= 0 || F <= 0 || D <= 0 || D > 64 || S <= 0) return TSP_ERR_INVALID_ARG;
+    if (F % D != 0 || (F / D) % 128 != 0 || H % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (S % D != 0 || (S / D) % 128 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X || !Wg || !Wu || !Wd || !Y) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(Y)) return TSP_ERR_INVALID_ARG;
+    // the intermediate must fit the fixed scratch: S * F bf16 elements
+    if (static_cast<unsigned long long>(S) * static_cast<unsigned long long>(F) * 2ull > kStaticScratchBytes)
+        return TSP_ERR_STATIC_LIMIT;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return TSP_ERR_CUDA;
+    StaticDeviceState* sd = nullptr;
+    tsp_status_t st = static_device_setup(dev, &sd);
+    if (st != TSP_OK) return st;
+
+    // A plan-shaped bundle on the host stack (no device memory behind it) so the ordinary launch code is reused.
+    tsp_mlp_plan_t tmp{};
+    tmp.H = H; tmp.F = F; tmp.D = D;
+    tmp.device = dev;
+    tmp.sm_count = sd->sm_count;
+    tmp.max_smem = sd->max_smem;
+    tmp.status_dev = reinterpret_cast<int*>(sd->scratch);
+    tmp.workspace = sd->scratch + kStaticHeaderBytes;
+    tmp.workspace_bytes = kStaticScratchBytes;
+    tmp.last_cuda_error = 0;
+    tmp.timeout_ns = 2000ull * 1000 * 1000;
+    tmp.encode = sd->encode;
+    tmp.profile_next = 0;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // The array keeps what the previous call left: the status word has to start at zero.
+    if (cudaMemsetAsync(sd->scratch, 0, kStaticHeaderBytes, stream) != cudaSuccess) return TSP_ERR_CUDA;
+    st = launch_gate_up(&tmp, X, Wg, Wu, tmp.workspace, S, stream);
+    if (st != TSP_OK) return st;
+    st = launch_down(&tmp, tmp.workspace, Wd, Y, S, stream);
+    if (st != TSP_OK) return st;
+    if (timed_out_host &&
+        cudaMemcpyAsync(timed_out_host, sd->scratch, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return TSP_ERR_CUDA;
+    return TSP_OK;
+}
+
 tsp_status_t tsp_mlp_status(tsp_mlp_plan_t* plan) {
     if (!plan) return TSP_ERR_INVALID_ARG;
     int v = 0;
@@ -460,6 +554,7 @@ const char* tsp_mlp_error_string(tsp_status_t s) {
         case TSP_ERR_CUDA: return "CUDA call failed";
         case TSP_ERR_WORKSPACE: return "workspace missing or too small";
         case TSP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case TSP_ERR_STATIC_LIMIT: return "problem too large for the fixed scratch of tsp_mlp_forward_static (S*F*2 bytes > TSP_MLP_STATIC_SCRATCH_BYTES)";
     }
     return "unknown status";
 }
