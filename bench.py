@@ -298,7 +298,7 @@ def run_gpu(args, wl):
 
     # ---- end to end: host buffers in pinned memory, H2D + forward + D2H every step ----
     e2e = None
-    if not train:
+    if not train and not args.no_e2e:
         hX = torch.from_numpy(host.X.view(np.int16)).pin_memory()
         hWg = torch.from_numpy(Wg_h.view(np.int16)).pin_memory()
         hWu = torch.from_numpy(Wu_h.view(np.int16)).pin_memory()
@@ -381,6 +381,7 @@ def main():
     ap.add_argument("--backward", action="store_true", help="time forward + backward (as the `train` workload does)")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()
     wl = inp.WORKLOADS[args.workload]
     if args.impl == "reference":

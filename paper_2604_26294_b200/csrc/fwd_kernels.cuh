@@ -26,6 +26,7 @@ struct GateUpParams {
     int blocks_per_rank; // (S/D) / 128
     int jl_blocks;       // (F/D) / 128
     int band;            // token blocks per band (their X rows stay L2-resident while the shards stream)
+    int shared_order;    // 0: ranks of a band follow the ring (different shards at a time); 1: same column block for all
     int num_tiles;
     int stages;
     int* status;
@@ -50,7 +51,7 @@ __device__ __forceinline__ GateUpTile gate_up_tile(const GateUpParams& p, int ti
     o.jl = rem / band_sz;
     o.mb = band_start + rem % band_sz;
     o.r = o.mb / p.blocks_per_rank;
-    o.k = (o.r - t % p.D + p.D) % p.D;
+    o.k = p.shared_order ? t : (o.r - t + p.D) % p.D;
     return o;
 }
 

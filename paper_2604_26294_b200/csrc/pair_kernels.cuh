@@ -1,0 +1,662 @@
+// CTA-pair (tcgen05 cta_group::2) versions of the kernels: two CTAs of a 2-CTA cluster, on the two SMs of a TPC,
+// work on one 256-row tile.  Each CTA loads its own 128 rows of the A operand and its own half of the B operand
+// (half of N), the leader CTA issues one M=256 MMA per k-step that reads both CTAs' shared memory and writes
+// 128 accumulator rows into each CTA's tensor memory.  Per SM this moves 32 KB per k-block instead of 48 KB.
+//
+// Synchronisation (all mbarriers are bounded-wait):
+//   full[s]       leader's only: the leader's producer arrives with the byte count of BOTH CTAs; both CTAs' TMA
+//                 loads complete on it (peer loads signal the leader's barrier through the cta_group::2 form).
+//   empty[s]      one per CTA: the leader's MMA thread commits to its own and to the peer's (two plain commits).
+//   tmem_full[b]  one per CTA, committed by the leader to both.
+//   tmem_empty[b] leader's only: 256 arrivals = the epilogue threads of both CTAs (the peer arrives remotely).
+// No load in this file names more than one destination CTA.
+#pragma once
+#include "bwd_kernels.cuh"
+#include "fwd_kernels.cuh"
+
+namespace tsp {
+
+// ------------------------------------------------------------------ cluster / pair PTX
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta_rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory; the completion may signal a barrier of the peer CTA.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
+                                                 int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 "
+        "[%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_dst), "l"(map), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr)
+                 : "memory");
+}
+
+constexpr uint32_t kPairStageBytes = 32 * 1024;  // per CTA: 128 rows of A (16 KB) + half of B (<= 16 KB)
+constexpr uint32_t kPairABytes = 16 * 1024;
+
+__device__ __forceinline__ void pair_load_kmajor(uint32_t smem, const CUtensorMap* map, uint32_t bar, int k0, int row0,
+                                                 int z) {
+    tma_load_3d_pair(smem, map, bar, k0, row0, z);
+}
+__device__ __forceinline__ void pair_load_mnmajor(uint32_t smem, const CUtensorMap* map, uint32_t bar, int mn0, int k0,
+                                                  int z, int chunks) {
+    for (int c = 0; c < chunks; ++c) tma_load_3d_pair(smem + c * 8192, map, bar, mn0 + c * 64, k0, z);
+}
+
+template <bool kAMn, bool kBMn>
+__device__ __forceinline__ void pair_issue_kblock(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem, uint32_t idesc,
+                                                  bool accumulate_first) {
+    const uint64_t a_desc = make_smem_desc_sw128(a_smem, kAMn ? 8192u : 0u, 1024u);
+    const uint64_t b_desc = make_smem_desc_sw128(b_smem, kBMn ? 8192u : 0u, 1024u);
+    constexpr uint64_t a_step = (kAMn ? 2048u : 32u) >> 4;
+    constexpr uint64_t b_step = (kBMn ? 2048u : 32u) >> 4;
+#pragma unroll
+    for (int kk = 0; kk < kBK / kUmmaK; ++kk)
+        umma_bf16_pair(d_tmem, a_desc + kk * a_step, b_desc + kk * b_step, idesc, (accumulate_first || kk > 0) ? 1u : 0u);
+}
+
+// All threads of both CTAs call.  n_acc accumulator barrier pairs.
+__device__ __forceinline__ void pair_setup(SharedCtl* ctl, int stages, int n_acc) {
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+            ctl->issued[s] = 0;
+        }
+        for (int b = 0; b < n_acc; ++b) {
+            mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[b]), 2 * kEpilogueThreads);
+        }
+        mbar_init(smem_u32(&ctl->teardown), 1);
+        ctl->abort = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(&ctl->tmem_base), kTmemCols);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    cluster_sync_all();
+    tc_fence_after_sync();
+}
+
+__device__ __forceinline__ void pair_teardown(SharedCtl* ctl, const WaitCtx& w) {
+    const int warp = threadIdx.x >> 5;
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*w.abort) {
+        // error path: give copies and MMAs still in flight time to land before shared / tensor memory is released
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+    }
+    cluster_sync_all();
+    tc_fence_after_sync();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc_pair(ctl->tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Generic pair kernel: tile = 256 rows (128 per CTA) x 256 columns, one K loop, two accumulator buffers.
+// Policy: Params{num_tiles, stages, status, timeout_ns}, Tile decode(p, tile), k_blocks(p),
+//         load(p, tile, kb, cta, sa, sb, bar), kAMn, kBMn, epilogue(p, tile, cta, row, t_row).
+// ------------------------------------------------------------------------------------------------
+template <class Policy>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
+pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_1024(smem_raw);
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + p.stages * kPairStageBytes);
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta = cluster_ctarank();
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+    pair_setup(ctl, p.stages, 2);
+    const uint32_t tmem_base = ctl->tmem_base;
+    WaitCtx w{&ctl->abort, p.status, p.timeout_ns};
+    // The K loop is outer() x inner() k-blocks; the policy maps (outer, inner) to coordinates without divisions.
+    const int n_outer = Policy::outer(p), n_inner = Policy::inner(p);
+    const int k_blocks = n_outer * n_inner;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            Policy::prefetch(p);
+            PipeState ps;
+            bool ok = true;
+            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs) {
+                const typename Policy::Tile tl = Policy::decode(p, tile);
+                for (int o = 0; o < n_outer && ok; ++o) {
+                    const int sel = Policy::select(p, tl, o);  // shard (or rank) met at outer step o
+                    for (int i = 0; i < n_inner; ++i) {
+                        if (!(ok = wait_bar(smem_u32(&ctl->empty[ps.stage]), ps.phase ^ 1u, w, kErrWaitEmpty))) break;
+                        const uint32_t bar = map_to_cta(smem_u32(&ctl->full[ps.stage]), 0);
+                        const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
+                        if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), 2 * kPairStageBytes);
+                        Policy::load(p, tl, sel, i, cta, sa, sb, bar);
+                        ps.advance(p.stages);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && cta == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(256, 256, Policy::kAMn, Policy::kBMn);
+            PipeState ps;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
+                const int buf = it & 1;
+                if (!(ok = wait_bar(smem_u32(&ctl->tmem_empty[buf]), ((it >> 1) & 1) ^ 1u, w, kErrWaitTmemEmpty))) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * 256;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
+                    pair_issue_kblock<Policy::kAMn, Policy::kBMn>(d_tmem, sa, sb, idesc, kb > 0);
+                    const uint32_t e = smem_u32(&ctl->empty[ps.stage]);
+                    umma_commit_pair(e);
+                    umma_commit_pair(map_to_cta(e, 1));
+                    ps.advance(p.stages);
+                }
+                if (ok) {
+                    const uint32_t f = smem_u32(&ctl->tmem_full[buf]);
+                    umma_commit_pair(f);
+                    umma_commit_pair(map_to_cta(f, 1));
+                }
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        bool ok = true;
+        int it = 0;
+        for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
+            const typename Policy::Tile tl = Policy::decode(p, tile);
+            const int buf = it & 1;
+            if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[buf]), (it >> 1) & 1, w, kErrWaitTmemFull))) break;
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
+            Policy::epilogue(p, tl, cta, row, t_row);
+            tc_fence_before_sync();
+            mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[buf]), 0));
+        }
+    }
+    pair_teardown(ctl, w);
+}
+
+// ---- store helpers ---------------------------------------------------------------------------------
+__device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t_row) {
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+        uint32_t v[32];
+        tmem_ld32(t_row + c * 32, v);
+        tmem_ld_wait();
+        uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            dst[q] = make_uint4(pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])),
+                                pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
+                                pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
+                                pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
+        }
+    }
+}
+
+// ---- gate | up + SwiGLU: tile = 256 tokens x 128 intermediate columns; CTA 0 loads the Wg half of B, CTA 1 the Wu half
+struct PairGateUpPolicy {
+    static constexpr bool kAMn = false, kBMn = true;
+    struct Params {
+        CUtensorMap map_x, map_wg, map_wu;  // boxes (64,128), (64,64), (64,64)
+        __nv_bfloat16* A;
+        int S, H, F, D, F_d;
+        int m_tiles, tiles_per_rank, jl_blocks, band, shared_order;
+        int num_tiles, stages;
+        int* status;
+        unsigned long long timeout_ns;
+    };
+    struct Tile {
+        int mt, k, jl;
+    };
+    __device__ static __forceinline__ int outer(const Params&) { return 1; }
+    __device__ static __forceinline__ int inner(const Params& p) { return p.H / kBK; }
+    __device__ static __forceinline__ int select(const Params&, const Tile& tl, int) { return tl.k; }
+    __device__ static __forceinline__ void prefetch(const Params& p) {
+        tma_prefetch_desc(&p.map_x);
+        tma_prefetch_desc(&p.map_wg);
+        tma_prefetch_desc(&p.map_wu);
+    }
+    // band of token tiles -> step t -> column block of the shard -> token tile
+    __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
+        const int per_band = p.band * p.D * p.jl_blocks;
+        const int band_idx = tile / per_band;
+        const int band_start = band_idx * p.band;
+        const int band_sz = min(p.band, p.m_tiles - band_start);
+        int rem = tile - band_idx * per_band;
+        const int t = rem / (p.jl_blocks * band_sz);
+        rem -= t * p.jl_blocks * band_sz;
+        Tile o;
+        o.jl = rem / band_sz;
+        o.mt = band_start + rem % band_sz;
+        const int r = o.mt / p.tiles_per_rank;
+        o.k = p.shared_order ? t : (r - t + p.D) % p.D;
+        return o;
+    }
+    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int k, int kb, uint32_t cta,
+                                                uint32_t sa, uint32_t sb, uint32_t bar) {
+        pair_load_kmajor(sa, &p.map_x, bar, kb * kBK, tl.mt * 256 + cta * 128, 0);
+        pair_load_mnmajor(sb, cta == 0 ? &p.map_wg : &p.map_wu, bar, tl.jl * 128, kb * kBK, k, 2);
+    }
+    __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
+        __nv_bfloat16* out = p.A + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F +
+                             static_cast<size_t>(tl.k) * p.F_d + tl.jl * 128;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            uint32_t g[32], u[32];
+            tmem_ld32(t_row + c * 32, g);
+            tmem_ld32(t_row + 128 + c * 32, u);
+            tmem_ld_wait();
+            uint32_t packed[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+                packed[i] = pack_bf16x2(g0 * sigmoid_fast(g0) * __uint_as_float(u[2 * i]),
+                                        g1 * sigmoid_fast(g1) * __uint_as_float(u[2 * i + 1]));
+            }
+            uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+        }
+    }
+};
+
+// ---- down projection: tile = 256 tokens x 256 hidden; K = F in ring order --------------------------
+struct PairDownPolicy {
+    static constexpr bool kAMn = false, kBMn = true;
+    struct Params {
+        CUtensorMap map_a, map_wd;  // boxes (64,128), (64,64)
+        __nv_bfloat16* Y;
+        int S, H, F, D, F_d;
+        int m_tiles, n_blocks, tiles_per_rank, group;
+        int num_tiles, stages;
+        int* status;
+        unsigned long long timeout_ns;
+    };
+    struct Tile {
+        int mt, nb, r;
+    };
+    __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
+    __device__ static __forceinline__ int inner(const Params& p) { return p.F_d / kBK; }
+    // shard held at ring step t: k = (r - t) mod D
+    __device__ static __forceinline__ int select(const Params& p, const Tile& tl, int t) {
+        const int k = tl.r - t;
+        return k < 0 ? k + p.D : k;
+    }
+    __device__ static __forceinline__ void prefetch(const Params& p) {
+        tma_prefetch_desc(&p.map_a);
+        tma_prefetch_desc(&p.map_wd);
+    }
+    __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
+        const int per_group = p.group * p.n_blocks;
+        const int g = tile / per_group;
+        const int g_start = g * p.group;
+        const int g_sz = min(p.group, p.m_tiles - g_start);
+        const int rem = tile - g * per_group;
+        Tile o;
+        o.nb = rem / g_sz;
+        o.mt = g_start + rem % g_sz;
+        o.r = o.mt / p.tiles_per_rank;
+        return o;
+    }
+    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
+                                                uint32_t sa, uint32_t sb, uint32_t bar) {
+        const int f0 = k * p.F_d + i * kBK;
+        pair_load_kmajor(sa, &p.map_a, bar, f0, tl.mt * 256 + cta * 128, 0);
+        pair_load_mnmajor(sb, &p.map_wd, bar, tl.nb * 256 + cta * 128, f0, 0, 2);
+    }
+    __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
+        store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
+    }
+};
+
+// ---- dX: tile = 256 tokens x 256 hidden; K = 2F (dG Wg^T then dU Wu^T per 64-slice), ring order ------
+struct PairDxPolicy {
+    static constexpr bool kAMn = false, kBMn = false;
+    struct Params {
+        CUtensorMap map_dg, map_du, map_wg, map_wu;  // boxes (64,128) all
+        __nv_bfloat16* dX;
+        int S, H, F, D, F_d;
+        int m_tiles, n_blocks, tiles_per_rank, group;
+        int num_tiles, stages;
+        int* status;
+        unsigned long long timeout_ns;
+    };
+    using Tile = PairDownPolicy::Tile;
+    __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
+    __device__ static __forceinline__ int inner(const Params& p) { return 2 * (p.F_d / kBK); }
+    __device__ static __forceinline__ int select(const Params& p, const Tile& tl, int t) {
+        const int k = tl.r - t;
+        return k < 0 ? k + p.D : k;
+    }
+    __device__ static __forceinline__ void prefetch(const Params& p) {
+        tma_prefetch_desc(&p.map_dg);
+        tma_prefetch_desc(&p.map_du);
+        tma_prefetch_desc(&p.map_wg);
+        tma_prefetch_desc(&p.map_wu);
+    }
+    __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
+        const int per_group = p.group * p.n_blocks;
+        const int g = tile / per_group;
+        const int g_start = g * p.group;
+        const int g_sz = min(p.group, p.m_tiles - g_start);
+        const int rem = tile - g * per_group;
+        Tile o;
+        o.nb = rem / g_sz;
+        o.mt = g_start + rem % g_sz;
+        o.r = o.mt / p.tiles_per_rank;
+        return o;
+    }
+    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
+                                                uint32_t sa, uint32_t sb, uint32_t bar) {
+        const int j0 = (i >> 1) * kBK;
+        const bool up = i & 1;
+        pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sb, up ? &p.map_wu : &p.map_wg, bar, j0, tl.nb * 256 + cta * 128, k);
+    }
+    __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
+        store_bf16_row256(p.dX + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
+    }
+};
+
+// ---- weight gradients: tile = 256 intermediate columns x 256 hidden; K = all S tokens ------------------
+struct PairDwPolicy {
+    static constexpr bool kAMn = true, kBMn = true;
+    struct Params {
+        CUtensorMap map_a, map_dg, map_du, map_dy, map_x;  // boxes (64,64) all
+        float* dWd;
+        float* dWg;
+        float* dWu;
+        int S, H, F, D, F_d, S_loc;
+        int j_tiles, n_blocks, j_tiles_per_shard;
+        int num_tiles, stages;
+        int* status;
+        unsigned long long timeout_ns;
+    };
+    struct Tile {
+        int which, jt, nb, k;
+    };
+    __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
+    __device__ static __forceinline__ int inner(const Params& p) { return p.S_loc / kBK; }
+    // shard k meets the ranks in the order r = (k + t) mod D
+    __device__ static __forceinline__ int select(const Params& p, const Tile& tl, int t) {
+        const int r = tl.k + t;
+        return r >= p.D ? r - p.D : r;
+    }
+    __device__ static __forceinline__ void prefetch(const Params& p) {
+        tma_prefetch_desc(&p.map_a);
+        tma_prefetch_desc(&p.map_dg);
+        tma_prefetch_desc(&p.map_du);
+        tma_prefetch_desc(&p.map_dy);
+        tma_prefetch_desc(&p.map_x);
+    }
+    __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
+        Tile o;
+        const int per_which = p.j_tiles * p.n_blocks;
+        o.which = tile / per_which;
+        const int rem = tile - o.which * per_which;
+        o.jt = rem / p.n_blocks;
+        o.nb = rem - o.jt * p.n_blocks;
+        o.k = o.jt / p.j_tiles_per_shard;
+        return o;
+    }
+    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int r, int i, uint32_t cta,
+                                                uint32_t sa, uint32_t sb, uint32_t bar) {
+        const int s0 = r * p.S_loc + i * kBK;
+        const CUtensorMap* ma = tl.which == 0 ? &p.map_a : (tl.which == 1 ? &p.map_dg : &p.map_du);
+        const CUtensorMap* mb = tl.which == 0 ? &p.map_dy : &p.map_x;
+        pair_load_mnmajor(sa, ma, bar, tl.jt * 256 + cta * 128, s0, 0, 2);
+        pair_load_mnmajor(sb, mb, bar, tl.nb * 256 + cta * 128, s0, 0, 2);
+    }
+    __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
+        const int j = tl.jt * 256 + cta * 128 + row;  // global intermediate index of this lane
+        const int F_d = p.F_d;
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+            uint32_t v[32];
+            tmem_ld32(t_row + c * 32, v);
+            tmem_ld_wait();
+            const int h0 = tl.nb * 256 + c * 32;
+            if (tl.which == 0) {
+                float4* dst = reinterpret_cast<float4*>(p.dWd + static_cast<size_t>(j) * p.H + h0);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                         __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+            } else {
+                float* base = (tl.which == 1 ? p.dWg : p.dWu) + static_cast<size_t>(tl.k) * p.H * F_d + (j - tl.k * F_d);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) base[static_cast<size_t>(h0 + i) * F_d] = __uint_as_float(v[i]);
+            }
+        }
+    }
+};
+
+// ------------------------------------------------------------------------------------------------
+// Pair version of bwd_gate_kernel: tile = 256 tokens x 128 intermediate columns.
+// Tensor memory per CTA: columns 0..255 G | U, columns 256..383 / 384..511 dA (alternating per tile).
+// ------------------------------------------------------------------------------------------------
+struct PairBwdGateParams {
+    CUtensorMap map_x, map_dy;    // (H, S, 1) box (64,128)
+    CUtensorMap map_wg, map_wu;   // (F/D, H, D) box (64,64)
+    CUtensorMap map_wd;           // (H, F, 1) box (64,64): 64 intermediate rows per CTA
+    __nv_bfloat16* A;
+    __nv_bfloat16* dG;
+    __nv_bfloat16* dU;
+    int S, H, F, D;
+    int m_tiles, tiles_per_rank, jl_blocks, band, shared_order;
+    int num_tiles, stages;
+    int* status;
+    unsigned long long timeout_ns;
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
+pair_bwd_gate_kernel(const __grid_constant__ PairBwdGateParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_1024(smem_raw);
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + p.stages * kPairStageBytes);
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta = cluster_ctarank();
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    constexpr uint32_t kBytesDA = kPairABytes + 64 * 128, kBytesGU = kPairABytes + 128 * 128;
+
+    pair_setup(ctl, p.stages, 3);
+    const uint32_t tmem_base = ctl->tmem_base;
+    WaitCtx w{&ctl->abort, p.status, p.timeout_ns};
+    const int k_blocks = p.H / kBK;
+    const int F_d = p.F / p.D;
+
+    auto decode = [&](int tile, int& mt, int& k, int& jl) {
+        const int per_band = p.band * p.D * p.jl_blocks;
+        const int band_idx = tile / per_band;
+        const int band_start = band_idx * p.band;
+        const int band_sz = min(p.band, p.m_tiles - band_start);
+        int rem = tile - band_idx * per_band;
+        const int t = rem / (p.jl_blocks * band_sz);
+        rem -= t * p.jl_blocks * band_sz;
+        jl = rem / band_sz;
+        mt = band_start + rem % band_sz;
+        const int r = mt / p.tiles_per_rank;
+        k = p.shared_order ? t : (r - t + p.D) % p.D;
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&p.map_x);
+            tma_prefetch_desc(&p.map_dy);
+            tma_prefetch_desc(&p.map_wg);
+            tma_prefetch_desc(&p.map_wu);
+            tma_prefetch_desc(&p.map_wd);
+            PipeState ps;
+            bool ok = true;
+            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs) {
+                int mt, k, jl;
+                decode(tile, mt, k, jl);
+                for (int kb = 0; kb < 2 * k_blocks; ++kb) {
+                    if (!(ok = wait_bar(smem_u32(&ctl->empty[ps.stage]), ps.phase ^ 1u, w, kErrWaitEmpty))) break;
+                    const uint32_t bar = map_to_cta(smem_u32(&ctl->full[ps.stage]), 0);
+                    const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
+                    if (kb < k_blocks) {  // dA = dY Wd_k^T ; each CTA brings 64 of the 128 intermediate rows of Wd
+                        if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), 2 * kBytesDA);
+                        pair_load_kmajor(sa, &p.map_dy, bar, kb * kBK, mt * 256 + cta * 128, 0);
+                        pair_load_kmajor(sb, &p.map_wd, bar, kb * kBK, k * F_d + jl * 128 + cta * 64, 0);
+                    } else {              // G | U: CTA 0 brings the Wg columns, CTA 1 the Wu columns
+                        const int h0 = (kb - k_blocks) * kBK;
+                        if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), 2 * kBytesGU);
+                        pair_load_kmajor(sa, &p.map_x, bar, h0, mt * 256 + cta * 128, 0);
+                        pair_load_mnmajor(sb, cta == 0 ? &p.map_wg : &p.map_wu, bar, jl * 128, h0, k, 2);
+                    }
+                    ps.advance(p.stages);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && cta == 0) {
+            constexpr uint32_t idesc_da = make_idesc_bf16(256, 128, false, false);
+            constexpr uint32_t idesc_gu = make_idesc_bf16(256, 256, false, true);
+            PipeState ps;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
+                const int slot = it & 1;
+                if (!(ok = wait_bar(smem_u32(&ctl->tmem_empty[slot]), ((it >> 1) & 1) ^ 1u, w, kErrWaitTmemEmpty))) break;
+                tc_fence_after_sync();
+                const uint32_t d_da = tmem_base + 256 + slot * 128;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
+                    pair_issue_kblock<false, false>(d_da, sa, sb, idesc_da, kb > 0);
+                    const uint32_t e = smem_u32(&ctl->empty[ps.stage]);
+                    umma_commit_pair(e);
+                    umma_commit_pair(map_to_cta(e, 1));
+                    ps.advance(p.stages);
+                }
+                if (!ok) break;
+                if (!(ok = wait_bar(smem_u32(&ctl->tmem_empty[2]), (it & 1) ^ 1u, w, kErrWaitTmemEmpty))) break;
+                tc_fence_after_sync();
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
+                    pair_issue_kblock<false, true>(tmem_base, sa, sb, idesc_gu, kb > 0);
+                    const uint32_t e = smem_u32(&ctl->empty[ps.stage]);
+                    umma_commit_pair(e);
+                    umma_commit_pair(map_to_cta(e, 1));
+                    ps.advance(p.stages);
+                }
+                if (ok) {
+                    const uint32_t f = smem_u32(&ctl->tmem_full[slot]);
+                    umma_commit_pair(f);
+                    umma_commit_pair(map_to_cta(f, 1));
+                }
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        bool ok = true;
+        int it = 0;
+        for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
+            int mt, k, jl;
+            decode(tile, mt, k, jl);
+            const int slot = it & 1;
+            if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[slot]), (it >> 1) & 1, w, kErrWaitTmemFull))) break;
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            const size_t off = static_cast<size_t>(mt * 256 + cta * 128 + row) * p.F + static_cast<size_t>(k) * F_d + jl * 128;
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+                uint32_t g[16], u[16], da[16];
+                tmem_ld16(t_row + c * 16, g);
+                tmem_ld16(t_row + 128 + c * 16, u);
+                tmem_ld16(t_row + 256 + slot * 128 + c * 16, da);
+                tmem_ld_wait();
+                uint32_t pa[8], pg[8], pu[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float va[2], vg[2], vu[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float gg = __uint_as_float(g[2 * i + e]);
+                        const float uu = __uint_as_float(u[2 * i + e]);
+                        const float dd = __uint_as_float(da[2 * i + e]);
+                        const float s = sigmoid_fast(gg);
+                        const float sg = gg * s;
+                        va[e] = sg * uu;
+                        vu[e] = dd * sg;
+                        vg[e] = dd * uu * (s * (1.0f + gg * (1.0f - s)));
+                    }
+                    pa[i] = pack_bf16x2(va[0], va[1]);
+                    pg[i] = pack_bf16x2(vg[0], vg[1]);
+                    pu[i] = pack_bf16x2(vu[0], vu[1]);
+                }
+                uint4* oa = reinterpret_cast<uint4*>(p.A + off + c * 16);
+                uint4* og = reinterpret_cast<uint4*>(p.dG + off + c * 16);
+                uint4* ou = reinterpret_cast<uint4*>(p.dU + off + c * 16);
+                oa[0] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
+                oa[1] = make_uint4(pa[4], pa[5], pa[6], pa[7]);
+                og[0] = make_uint4(pg[0], pg[1], pg[2], pg[3]);
+                og[1] = make_uint4(pg[4], pg[5], pg[6], pg[7]);
+                ou[0] = make_uint4(pu[0], pu[1], pu[2], pu[3]);
+                ou[1] = make_uint4(pu[4], pu[5], pu[6], pu[7]);
+            }
+            tc_fence_before_sync();
+            mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[2]), 0));
+            mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[slot]), 0));
+        }
+    }
+    pair_teardown(ctl, w);
+}
+
+}  // namespace tsp

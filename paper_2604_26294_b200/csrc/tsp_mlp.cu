@@ -14,6 +14,7 @@
 #include "../../include/tsp_mlp.h"
 #include "bwd_kernels.cuh"
 #include "fwd_kernels.cuh"
+#include "pair_kernels.cuh"
 
 namespace {
 
@@ -46,6 +47,12 @@ struct tsp_mlp_plan {
     EncodeTiledFn encode;
     std::vector<ProfileCall> profile;
     int profile_next;
+    // tunables (environment overrides read at plan creation; 0 = default)
+    int use_pairs;      // CTA-pair (cta_group::2) kernels where the shape allows
+    int band;           // token tiles per band in the gate|up tile order
+    int shared_order;   // gate|up tile order: 1 = all ranks of a band on the same shard column block
+    int group;          // token tiles per group in the down / dX tile order
+    int pair_stages;
 };
 
 namespace {
@@ -127,6 +134,12 @@ struct Profiler {
     }
 };
 
+// Token tiles (of 256 rows) per band of the gate|up tile order.
+int gate_band(const tsp_mlp_plan_t* plan, int m_tiles) {
+    int band = plan->band > 0 ? plan->band : 8;   // 8 tiles of 256 tokens: 16 MB of X at H = 4096
+    return band > m_tiles ? m_tiles : band;
+}
+
 // ---------------------------------------------------------------------------------------------
 // launches
 // ---------------------------------------------------------------------------------------------
@@ -143,8 +156,9 @@ tsp_status_t launch_gate_up(tsp_mlp_plan_t* plan, const void* X, const void* Wg,
     p.m_blocks = static_cast<int>(S / 128);
     p.blocks_per_rank = static_cast<int>(S / D / 128);
     p.jl_blocks = F_d / 128;
-    const int band_cap = static_cast<int>((64ull << 20) / (128ull * H * 2));
-    p.band = band_cap < 1 ? 1 : (band_cap > p.m_blocks ? p.m_blocks : band_cap);
+    p.band = 2 * gate_band(plan, (p.m_blocks + 1) / 2);   // same band, counted in 128-token blocks
+    if (p.band > p.m_blocks) p.band = p.m_blocks;
+    p.shared_order = plan->shared_order;
     p.num_tiles = p.m_blocks * D * p.jl_blocks;
     p.stages = pick_stages(plan, 48 * 1024, 4);
     p.status = plan->status_dev;
@@ -202,8 +216,8 @@ tsp_status_t launch_bwd_gate(tsp_mlp_plan_t* plan, const void* X, const void* Wg
     p.m_blocks = static_cast<int>(S / 128);
     p.blocks_per_rank = static_cast<int>(S / D / 128);
     p.jl_blocks = F_d / 128;
-    const int band_cap = static_cast<int>((32ull << 20) / (128ull * H * 2));
-    p.band = band_cap < 1 ? 1 : (band_cap > p.m_blocks ? p.m_blocks : band_cap);
+    p.band = 2 * gate_band(plan, (p.m_blocks + 1) / 2);
+    if (p.band > p.m_blocks) p.band = p.m_blocks;
     p.num_tiles = p.m_blocks * D * p.jl_blocks;
     p.stages = pick_stages(plan, 48 * 1024, 4);
     p.status = plan->status_dev;
@@ -274,6 +288,134 @@ tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, 
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
+
+
+// ---------------------------------------------------------------------------------------------
+// CTA-pair launches (tile = 256 rows per pair).  Chosen when (S/D) % 256 == 0 (and (F/D) % 256 == 0 for dW).
+// ---------------------------------------------------------------------------------------------
+template <class Params>
+void fill_common(tsp_mlp_plan_t* plan, Params& p, int num_tiles) {
+    p.num_tiles = num_tiles;
+    p.stages = pick_stages(plan, tsp::kPairStageBytes, plan->pair_stages > 0 ? plan->pair_stages : 6);
+    p.status = plan->status_dev;
+    p.timeout_ns = plan->timeout_ns;
+}
+
+template <class Kernel, class Params>
+tsp_status_t launch_pair(tsp_mlp_plan_t* plan, Kernel kernel, const Params& p, cudaStream_t stream) {
+    const size_t smem = p.stages * tsp::kPairStageBytes + sizeof(tsp::SharedCtl) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    const int pairs_avail = plan->sm_count / 2;
+    const int pairs = p.num_tiles < pairs_avail ? p.num_tiles : pairs_avail;
+    kernel<<<2 * pairs, tsp::kNumThreads, smem, stream>>>(p);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
+}
+
+tsp_status_t launch_gate_up_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A, int64_t S,
+                                 cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
+    tsp::PairGateUpPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    p.A = static_cast<__nv_bfloat16*>(A);
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.F_d = F_d;
+    p.m_tiles = static_cast<int>(S / 256);
+    p.tiles_per_rank = static_cast<int>(S / D / 256);
+    p.jl_blocks = F_d / 128;
+    p.band = gate_band(plan, p.m_tiles);
+    p.shared_order = plan->shared_order;
+    fill_common(plan, p, p.m_tiles * D * p.jl_blocks);
+    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairGateUpPolicy>, p, stream);
+}
+
+tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* Wd, void* Y, int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D;
+    tsp::PairDownPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_a, A, S, F, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 64)) return TSP_ERR_CUDA;
+    p.Y = static_cast<__nv_bfloat16*>(Y);
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D; p.F_d = F / D;
+    p.m_tiles = static_cast<int>(S / 256);
+    p.n_blocks = H / 256;
+    p.tiles_per_rank = static_cast<int>(S / D / 256);
+    const int group = plan->group > 0 ? plan->group : 8;
+    p.group = p.m_tiles < group ? p.m_tiles : group;
+    fill_common(plan, p, p.m_tiles * p.n_blocks);
+    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownPolicy>, p, stream);
+}
+
+tsp_status_t launch_bwd_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
+                                  const void* dY, void* A, void* dG, void* dU, int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
+    tsp::PairBwdGateParams p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 64)) return TSP_ERR_CUDA;
+    p.A = static_cast<__nv_bfloat16*>(A);
+    p.dG = static_cast<__nv_bfloat16*>(dG);
+    p.dU = static_cast<__nv_bfloat16*>(dU);
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.m_tiles = static_cast<int>(S / 256);
+    p.tiles_per_rank = static_cast<int>(S / D / 256);
+    p.jl_blocks = F_d / 128;
+    p.band = gate_band(plan, p.m_tiles);
+    p.shared_order = plan->shared_order;
+    fill_common(plan, p, p.m_tiles * D * p.jl_blocks);
+    return launch_pair(plan, tsp::pair_bwd_gate_kernel, p, stream);
+}
+
+tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void* dU, const void* Wg, const void* Wu,
+                                void* dX, int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
+    tsp::PairDxPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_dg, dG, S, F, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_du, dU, S, F, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 128)) return TSP_ERR_CUDA;
+    p.dX = static_cast<__nv_bfloat16*>(dX);
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D; p.F_d = F_d;
+    p.m_tiles = static_cast<int>(S / 256);
+    p.n_blocks = H / 256;
+    p.tiles_per_rank = static_cast<int>(S / D / 256);
+    const int group = plan->group > 0 ? plan->group : 8;
+    p.group = p.m_tiles < group ? p.m_tiles : group;
+    fill_common(plan, p, p.m_tiles * p.n_blocks);
+    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDxPolicy>, p, stream);
+}
+
+tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
+                                const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D;
+    tsp::PairDwPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_a, A, S, F, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_dg, dG, S, F, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_du, dU, S, F, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 64)) return TSP_ERR_CUDA;
+    p.dWd = dWd; p.dWg = dWg; p.dWu = dWu;
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.F_d = F / D;
+    p.S_loc = static_cast<int>(S / D);
+    p.j_tiles = F / 256;
+    p.j_tiles_per_shard = p.F_d / 256;
+    p.n_blocks = H / 256;
+    fill_common(plan, p, 3 * p.j_tiles * p.n_blocks);
+    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDwPolicy>, p, stream);
+}
+
+bool pairs_for_tokens(const tsp_mlp_plan_t* plan, int64_t S) { return plan->use_pairs && (S / plan->D) % 256 == 0; }
+bool pairs_for_dw(const tsp_mlp_plan_t* plan) { return plan->use_pairs && (plan->F / plan->D) % 256 == 0; }
 
 // ---------------------------------------------------------------------------------------------
 // Fixed scratch for tsp_mlp_forward_static: part of the library image, so every GPU that loads the
@@ -362,6 +504,15 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
         const long ms = std::atol(t);
         if (ms > 0) plan->timeout_ns = static_cast<unsigned long long>(ms) * 1000 * 1000;
     }
+    auto env_int = [](const char* name, int dflt) {
+        const char* v = std::getenv(name);
+        return v ? std::atoi(v) : dflt;
+    };
+    plan->use_pairs = env_int("TSP_MLP_PAIR", 1);
+    plan->band = env_int("TSP_MLP_BAND", 0);
+    plan->shared_order = env_int("TSP_MLP_GATE_ORDER", 1);
+    plan->group = env_int("TSP_MLP_GROUP", 0);
+    plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
@@ -421,10 +572,13 @@ tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg
         return TSP_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     Profiler prof(plan, stream);
-    st = launch_gate_up(plan, X, Wg, Wu, plan->workspace, S, stream);
+    const bool pairs = pairs_for_tokens(plan, S);
+    st = pairs ? launch_gate_up_pair(plan, X, Wg, Wu, plan->workspace, S, stream)
+               : launch_gate_up(plan, X, Wg, Wu, plan->workspace, S, stream);
     if (st != TSP_OK) return st;
     prof.mark();
-    st = launch_down(plan, plan->workspace, Wd, Y, S, stream);
+    st = pairs ? launch_down_pair(plan, plan->workspace, Wd, Y, S, stream)
+               : launch_down(plan, plan->workspace, Wd, Y, S, stream);
     if (st != TSP_OK) return st;
     prof.mark();
     return TSP_OK;
@@ -476,13 +630,17 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
     void* dG = base + one;
     void* dU = base + 2 * one;
     Profiler prof(plan, stream);
-    st = launch_bwd_gate(plan, X, Wg, Wu, Wd, dY, A, dG, dU, S, stream);
+    const bool pairs = pairs_for_tokens(plan, S);
+    st = pairs ? launch_bwd_gate_pair(plan, X, Wg, Wu, Wd, dY, A, dG, dU, S, stream)
+               : launch_bwd_gate(plan, X, Wg, Wu, Wd, dY, A, dG, dU, S, stream);
     if (st != TSP_OK) return st;
     prof.mark();
-    st = launch_bwd_dx(plan, dG, dU, Wg, Wu, dX, S, stream);
+    st = pairs ? launch_bwd_dx_pair(plan, dG, dU, Wg, Wu, dX, S, stream)
+               : launch_bwd_dx(plan, dG, dU, Wg, Wu, dX, S, stream);
     if (st != TSP_OK) return st;
     prof.mark();
-    st = launch_bwd_dw(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream);
+    st = pairs_for_dw(plan) ? launch_bwd_dw_pair(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream)
+                            : launch_bwd_dw(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream);
     if (st != TSP_OK) return st;
     prof.mark();
     return TSP_OK;
