@@ -36,6 +36,8 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel
 # at the named workload, from the ncu capture summarised under profiles/.  None = not captured.
 NCU_DRAM_BYTES = {
+    ("gate_up", "7b_short"): 1.0717e9 + 0.2282e9,   # profiles/ncu_full_pair_kernels_7b_train.txt (same shapes)
+    ("gate_up", "train"): 1.0717e9 + 0.2282e9,
 }
 
 
@@ -334,13 +336,17 @@ def run_gpu(args, wl):
     gate_up_ms = float(per_kernel[0])
     gate_up_flops = 4.0 * S * H * F
     achieved = gate_up_flops / (gate_up_ms * 1e-3) / 1e12
+    pairs = (S // D) % 256 == 0 and os.environ.get("TSP_MLP_PAIR", "1") != "0"
+    gate_up_name = "pair_gemm_kernel<PairGateUpPolicy>" if pairs else "gate_up_swiglu_kernel"
+    down_name = "pair_gemm_kernel<PairDownPolicy>" if pairs else "down_accumulate_kernel"
     roofline = {
-        "bound": "tensor", "kernel": "gate_up_swiglu_kernel", "achieved": achieved, "peak": peaks["burst"],
+        "bound": "tensor", "kernel": gate_up_name, "achieved": achieved, "peak": peaks["burst"],
         "unit": UNIT, "frac": achieved / peaks["burst"], "peak_source": f"of {peaks['source']} (burst bf16 GEMM)",
         "frac_of_sustained": achieved / peaks["sustained"], "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
         "flops_per_launch": gate_up_flops, "ms_per_launch": gate_up_ms,
-        "traffic": NCU_DRAM_BYTES.get(("gate_up_swiglu_kernel", wl.name)),
-        "kernels_ms": {"gate_up_swiglu_kernel": gate_up_ms, "down_accumulate_kernel": float(per_kernel[1])},
+        "traffic": NCU_DRAM_BYTES.get(("gate_up", wl.name)) if pairs else None,
+        "algorithmic_bytes_per_launch": 2.0 * S * H + 4.0 * H * F + 2.0 * S * F,
+        "kernels_ms": {gate_up_name: gate_up_ms, down_name: float(per_kernel[1])},
     }
     if bwd_kernel is not None:
         roofline["kernels_ms"].update({f"backward_kernel_{i}": float(v) for i, v in enumerate(bwd_kernel)})
