@@ -259,14 +259,15 @@ def run_gpu(args, wl):
         if train:
             b.tsp_mlp_backward(plan, X, Wg, Wu, Wd, dY, dX, dWg, dWu, dWd, S, D)
 
-    kernels_per_step = b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD) + (
-        b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_BACKWARD) if train else 0)
     model_flops = wl.forward_flops() + (wl.backward_flops() if train else 0.0)
 
     for _ in range(max(3, args.warmup)):
         step()
     barrier()
     assert b.tsp_mlp_status(plan) == b.TSP_OK, "device-side wait timed out during warm-up"
+    # counted after a call has been made: the backward count depends on the shape-dependent path taken
+    kernels_per_step = b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD) + (
+        b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_BACKWARD) if train else 0)
 
     # ---- timed region: K steps, inputs resident in HBM ----
     calls_per_step = 2 if train else 1

@@ -67,7 +67,7 @@ tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan);
 
 /*
  * Workspace: scratch for the bf16 intermediate A = silu(G)*U [S,F] (forward) and for
- * A, dG, dU [S,F] each (backward).  tsp_mlp_workspace_bytes returns the size needed
+ * A, dG, dU [S,F] in bf16 plus dA [S,F] in fp32 (backward).  tsp_mlp_workspace_bytes returns the size needed
  * for S tokens (`pass` = TSP_WS_FORWARD or TSP_WS_BACKWARD; backward covers forward);
  * 0 on bad arguments.  tsp_mlp_set_workspace hands a caller-owned device buffer
  * (256-byte aligned) to the plan; it must stay valid while calls using it are in flight.
@@ -89,8 +89,8 @@ tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg
  * tsp_mlp_backward - gradients of the forward above for upstream dY (the backward
  * pass mirrors the forward weight movement; the partial weight gradients every rank
  * produces for shard k are summed to the owner, Sections 4.3.4 and 4.7).  G and U are
- * recomputed from X; dA = dY Wd^T; dU = dA*silu(G); dG = dA*U*silu'(G); A, dG, dU are
- * rounded once to bf16 into the workspace.  dX [S,H] bf16 accumulates over shards in
+ * recomputed from X; dA = dY Wd^T (kept in fp32); dU = dA*silu(G); dG = dA*U*silu'(G);
+ * A, dG, dU are rounded once to bf16 into the workspace.  dX [S,H] bf16 accumulates over shards in
  * ring order; dWg, dWu [D][H][F/D] and dWd [D][F/D][H] are fp32 and contract over all S
  * tokens, rank order r = (k + t) mod D.
  */
@@ -171,7 +171,9 @@ tsp_status_t tsp_mlp_profile_begin(tsp_mlp_plan_t* plan, int max_calls);
 tsp_status_t tsp_mlp_profile_read(tsp_mlp_plan_t* plan, int call_index, int* n_kernels_out, float* ms_out);
 tsp_status_t tsp_mlp_profile_end(tsp_mlp_plan_t* plan);
 
-/* Number of kernels one forward (pass=TSP_WS_FORWARD) or backward call launches. */
+/* Number of kernels one forward call launches (pass=TSP_WS_FORWARD: 2), or that the most recent
+ * tsp_mlp_backward on this plan launched (pass=TSP_WS_BACKWARD: 4 when (S/D) % 256 == 0 and F % 256 == 0,
+ * else 3; 3 before the first backward call). */
 int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass);
 
 #ifdef __cplusplus

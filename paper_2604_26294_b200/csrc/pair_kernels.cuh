@@ -242,12 +242,18 @@ __device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t
     }
 }
 
-// ---- gate | up + SwiGLU: tile = 256 tokens x 128 intermediate columns; CTA 0 loads the Wg half of B, CTA 1 the Wu half
-struct PairGateUpPolicy {
+// ---- gate | up + SwiGLU: tile = 256 tokens x 128 intermediate columns; CTA 0 loads the Wg half of B, CTA 1 the Wu half.
+// kBackward = false: epilogue writes A = silu(G) * U.
+// kBackward = true : epilogue also reads dA (fp32, from the dA GEMM) and writes A, dG = dA*U*silu'(G), dU = dA*silu(G).
+template <bool kBackward>
+struct PairGateUpPolicyT {
     static constexpr bool kAMn = false, kBMn = true;
     struct Params {
         CUtensorMap map_x, map_wg, map_wu;  // boxes (64,128), (64,64), (64,64)
         __nv_bfloat16* A;
+        const float* dA;      // [S, F] fp32 (backward only)
+        __nv_bfloat16* dG;    // [S, F] (backward only)
+        __nv_bfloat16* dU;    // [S, F] (backward only)
         int S, H, F, D, F_d;
         int m_tiles, tiles_per_rank, jl_blocks, band, shared_order;
         int num_tiles, stages;
@@ -287,25 +293,125 @@ struct PairGateUpPolicy {
         pair_load_mnmajor(sb, cta == 0 ? &p.map_wg : &p.map_wu, bar, tl.jl * 128, kb * kBK, k, 2);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        __nv_bfloat16* out = p.A + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F +
-                             static_cast<size_t>(tl.k) * p.F_d + tl.jl * 128;
+        const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F + static_cast<size_t>(tl.k) * p.F_d +
+                           tl.jl * 128;
+        if constexpr (!kBackward) {
+            __nv_bfloat16* out = p.A + off;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            uint32_t g[32], u[32];
-            tmem_ld32(t_row + c * 32, g);
-            tmem_ld32(t_row + 128 + c * 32, u);
-            tmem_ld_wait();
-            uint32_t packed[16];
+            for (int c = 0; c < 4; ++c) {
+                uint32_t g[32], u[32];
+                tmem_ld32(t_row + c * 32, g);
+                tmem_ld32(t_row + 128 + c * 32, u);
+                tmem_ld_wait();
+                uint32_t packed[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-                packed[i] = pack_bf16x2(g0 * sigmoid_fast(g0) * __uint_as_float(u[2 * i]),
-                                        g1 * sigmoid_fast(g1) * __uint_as_float(u[2 * i + 1]));
+                for (int i = 0; i < 16; ++i) {
+                    const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+                    packed[i] = pack_bf16x2(g0 * sigmoid_fast(g0) * __uint_as_float(u[2 * i]),
+                                            g1 * sigmoid_fast(g1) * __uint_as_float(u[2 * i + 1]));
+                }
+                uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
             }
-            uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+        } else {
+            const float4* da_row = reinterpret_cast<const float4*>(p.dA + off);
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+                float4 da4[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                for (int q = 0; q < 4; ++q) da4[q] = __ldg(da_row + c * 4 + q);   // issued before the tensor-memory loads
+                uint32_t g[16], u[16];
+                tmem_ld16(t_row + c * 16, g);
+                tmem_ld16(t_row + 128 + c * 16, u);
+                tmem_ld_wait();
+                const float* da = reinterpret_cast<const float*>(da4);
+                uint32_t pa[8], pg[8], pu[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float va[2], vg[2], vu[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float gg = __uint_as_float(g[2 * i + e]);
+                        const float uu = __uint_as_float(u[2 * i + e]);
+                        const float dd = da[2 * i + e];
+                        const float sgm = sigmoid_fast(gg);
+                        const float sg = gg * sgm;                          // silu(G)
+                        va[e] = sg * uu;                                    // A
+                        vu[e] = dd * sg;                                    // dU = dA * silu(G)
+                        vg[e] = dd * uu * (sgm * (1.0f + gg * (1.0f - sgm)));  // dG = dA * U * silu'(G)
+                    }
+                    pa[i] = pack_bf16x2(va[0], va[1]);
+                    pg[i] = pack_bf16x2(vg[0], vg[1]);
+                    pu[i] = pack_bf16x2(vu[0], vu[1]);
+                }
+                uint4* oa = reinterpret_cast<uint4*>(p.A + off + c * 16);
+                uint4* og = reinterpret_cast<uint4*>(p.dG + off + c * 16);
+                uint4* ou = reinterpret_cast<uint4*>(p.dU + off + c * 16);
+                oa[0] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
+                oa[1] = make_uint4(pa[4], pa[5], pa[6], pa[7]);
+                og[0] = make_uint4(pg[0], pg[1], pg[2], pg[3]);
+                og[1] = make_uint4(pg[4], pg[5], pg[6], pg[7]);
+                ou[0] = make_uint4(pu[0], pu[1], pu[2], pu[3]);
+                ou[1] = make_uint4(pu[4], pu[5], pu[6], pu[7]);
+            }
+        }
+    }
+};
+using PairGateUpPolicy = PairGateUpPolicyT<false>;
+using PairGateBwdPolicy = PairGateUpPolicyT<true>;
+
+// ---- dA = dY Wd^T (fp32 out): tile = 256 tokens x 256 intermediate columns; K = H ---------------------
+struct PairDaPolicy {
+    static constexpr bool kAMn = false, kBMn = false;
+    struct Params {
+        CUtensorMap map_dy, map_wd;  // (H, S, 1) box (64,128); (H, F, 1) box (64,128)
+        float* dA;                   // [S, F] fp32
+        int S, H, F, D;
+        int m_tiles, j_tiles, band;
+        int num_tiles, stages;
+        int* status;
+        unsigned long long timeout_ns;
+    };
+    struct Tile {
+        int mt, jt;
+    };
+    __device__ static __forceinline__ int outer(const Params&) { return 1; }
+    __device__ static __forceinline__ int inner(const Params& p) { return p.H / kBK; }
+    __device__ static __forceinline__ int select(const Params&, const Tile&, int) { return 0; }
+    __device__ static __forceinline__ void prefetch(const Params& p) {
+        tma_prefetch_desc(&p.map_dy);
+        tma_prefetch_desc(&p.map_wd);
+    }
+    // band of token tiles -> intermediate tile -> token tile (the dY rows of a band stay in L2 while Wd streams)
+    __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
+        const int per_band = p.band * p.j_tiles;
+        const int band_idx = tile / per_band;
+        const int band_start = band_idx * p.band;
+        const int band_sz = min(p.band, p.m_tiles - band_start);
+        const int rem = tile - band_idx * per_band;
+        Tile o;
+        o.jt = rem / band_sz;
+        o.mt = band_start + rem % band_sz;
+        return o;
+    }
+    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int, int kb, uint32_t cta, uint32_t sa,
+                                                uint32_t sb, uint32_t bar) {
+        pair_load_kmajor(sa, &p.map_dy, bar, kb * kBK, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sb, &p.map_wd, bar, kb * kBK, tl.jt * 256 + cta * 128, 0);
+    }
+    __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
+        float4* dst = reinterpret_cast<float4*>(p.dA + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F + tl.jt * 256);
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+            uint32_t v[32];
+            tmem_ld32(t_row + c * 32, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                dst[c * 8 + q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                             __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
         }
     }
 };
@@ -480,183 +586,5 @@ struct PairDwPolicy {
         }
     }
 };
-
-// ------------------------------------------------------------------------------------------------
-// Pair version of bwd_gate_kernel: tile = 256 tokens x 128 intermediate columns.
-// Tensor memory per CTA: columns 0..255 G | U, columns 256..383 / 384..511 dA (alternating per tile).
-// ------------------------------------------------------------------------------------------------
-struct PairBwdGateParams {
-    CUtensorMap map_x, map_dy;    // (H, S, 1) box (64,128)
-    CUtensorMap map_wg, map_wu;   // (F/D, H, D) box (64,64)
-    CUtensorMap map_wd;           // (H, F, 1) box (64,64): 64 intermediate rows per CTA
-    __nv_bfloat16* A;
-    __nv_bfloat16* dG;
-    __nv_bfloat16* dU;
-    int S, H, F, D;
-    int m_tiles, tiles_per_rank, jl_blocks, band, shared_order;
-    int num_tiles, stages;
-    int* status;
-    unsigned long long timeout_ns;
-};
-
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
-pair_bwd_gate_kernel(const __grid_constant__ PairBwdGateParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = align_1024(smem_raw);
-    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + p.stages * kPairStageBytes);
-    const uint32_t smem_base = smem_u32(smem);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t cta = cluster_ctarank();
-    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    constexpr uint32_t kBytesDA = kPairABytes + 64 * 128, kBytesGU = kPairABytes + 128 * 128;
-
-    pair_setup(ctl, p.stages, 3);
-    const uint32_t tmem_base = ctl->tmem_base;
-    WaitCtx w{&ctl->abort, p.status, p.timeout_ns};
-    const int k_blocks = p.H / kBK;
-    const int F_d = p.F / p.D;
-
-    auto decode = [&](int tile, int& mt, int& k, int& jl) {
-        const int per_band = p.band * p.D * p.jl_blocks;
-        const int band_idx = tile / per_band;
-        const int band_start = band_idx * p.band;
-        const int band_sz = min(p.band, p.m_tiles - band_start);
-        int rem = tile - band_idx * per_band;
-        const int t = rem / (p.jl_blocks * band_sz);
-        rem -= t * p.jl_blocks * band_sz;
-        jl = rem / band_sz;
-        mt = band_start + rem % band_sz;
-        const int r = mt / p.tiles_per_rank;
-        k = p.shared_order ? t : (r - t + p.D) % p.D;
-    };
-
-    if (warp == 0) {
-        if (lane == 0) {
-            tma_prefetch_desc(&p.map_x);
-            tma_prefetch_desc(&p.map_dy);
-            tma_prefetch_desc(&p.map_wg);
-            tma_prefetch_desc(&p.map_wu);
-            tma_prefetch_desc(&p.map_wd);
-            PipeState ps;
-            bool ok = true;
-            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs) {
-                int mt, k, jl;
-                decode(tile, mt, k, jl);
-                for (int kb = 0; kb < 2 * k_blocks; ++kb) {
-                    if (!(ok = wait_bar(smem_u32(&ctl->empty[ps.stage]), ps.phase ^ 1u, w, kErrWaitEmpty))) break;
-                    const uint32_t bar = map_to_cta(smem_u32(&ctl->full[ps.stage]), 0);
-                    const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
-                    if (kb < k_blocks) {  // dA = dY Wd_k^T ; each CTA brings 64 of the 128 intermediate rows of Wd
-                        if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), 2 * kBytesDA);
-                        pair_load_kmajor(sa, &p.map_dy, bar, kb * kBK, mt * 256 + cta * 128, 0);
-                        pair_load_kmajor(sb, &p.map_wd, bar, kb * kBK, k * F_d + jl * 128 + cta * 64, 0);
-                    } else {              // G | U: CTA 0 brings the Wg columns, CTA 1 the Wu columns
-                        const int h0 = (kb - k_blocks) * kBK;
-                        if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), 2 * kBytesGU);
-                        pair_load_kmajor(sa, &p.map_x, bar, h0, mt * 256 + cta * 128, 0);
-                        pair_load_mnmajor(sb, cta == 0 ? &p.map_wg : &p.map_wu, bar, jl * 128, h0, k, 2);
-                    }
-                    ps.advance(p.stages);
-                }
-            }
-        }
-    } else if (warp == 1) {
-        if (lane == 0 && cta == 0) {
-            constexpr uint32_t idesc_da = make_idesc_bf16(256, 128, false, false);
-            constexpr uint32_t idesc_gu = make_idesc_bf16(256, 256, false, true);
-            PipeState ps;
-            bool ok = true;
-            int it = 0;
-            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
-                const int slot = it & 1;
-                if (!(ok = wait_bar(smem_u32(&ctl->tmem_empty[slot]), ((it >> 1) & 1) ^ 1u, w, kErrWaitTmemEmpty))) break;
-                tc_fence_after_sync();
-                const uint32_t d_da = tmem_base + 256 + slot * 128;
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
-                    tc_fence_after_sync();
-                    const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
-                    pair_issue_kblock<false, false>(d_da, sa, sb, idesc_da, kb > 0);
-                    const uint32_t e = smem_u32(&ctl->empty[ps.stage]);
-                    umma_commit_pair(e);
-                    umma_commit_pair(map_to_cta(e, 1));
-                    ps.advance(p.stages);
-                }
-                if (!ok) break;
-                if (!(ok = wait_bar(smem_u32(&ctl->tmem_empty[2]), (it & 1) ^ 1u, w, kErrWaitTmemEmpty))) break;
-                tc_fence_after_sync();
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
-                    tc_fence_after_sync();
-                    const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
-                    pair_issue_kblock<false, true>(tmem_base, sa, sb, idesc_gu, kb > 0);
-                    const uint32_t e = smem_u32(&ctl->empty[ps.stage]);
-                    umma_commit_pair(e);
-                    umma_commit_pair(map_to_cta(e, 1));
-                    ps.advance(p.stages);
-                }
-                if (ok) {
-                    const uint32_t f = smem_u32(&ctl->tmem_full[slot]);
-                    umma_commit_pair(f);
-                    umma_commit_pair(map_to_cta(f, 1));
-                }
-            }
-        }
-    } else {
-        const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;
-        bool ok = true;
-        int it = 0;
-        for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
-            int mt, k, jl;
-            decode(tile, mt, k, jl);
-            const int slot = it & 1;
-            if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[slot]), (it >> 1) & 1, w, kErrWaitTmemFull))) break;
-            tc_fence_after_sync();
-            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            const size_t off = static_cast<size_t>(mt * 256 + cta * 128 + row) * p.F + static_cast<size_t>(k) * F_d + jl * 128;
-#pragma unroll 1
-            for (int c = 0; c < 8; ++c) {
-                uint32_t g[16], u[16], da[16];
-                tmem_ld16(t_row + c * 16, g);
-                tmem_ld16(t_row + 128 + c * 16, u);
-                tmem_ld16(t_row + 256 + slot * 128 + c * 16, da);
-                tmem_ld_wait();
-                uint32_t pa[8], pg[8], pu[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    float va[2], vg[2], vu[2];
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const float gg = __uint_as_float(g[2 * i + e]);
-                        const float uu = __uint_as_float(u[2 * i + e]);
-                        const float dd = __uint_as_float(da[2 * i + e]);
-                        const float s = sigmoid_fast(gg);
-                        const float sg = gg * s;
-                        va[e] = sg * uu;
-                        vu[e] = dd * sg;
-                        vg[e] = dd * uu * (s * (1.0f + gg * (1.0f - s)));
-                    }
-                    pa[i] = pack_bf16x2(va[0], va[1]);
-                    pg[i] = pack_bf16x2(vg[0], vg[1]);
-                    pu[i] = pack_bf16x2(vu[0], vu[1]);
-                }
-                uint4* oa = reinterpret_cast<uint4*>(p.A + off + c * 16);
-                uint4* og = reinterpret_cast<uint4*>(p.dG + off + c * 16);
-                uint4* ou = reinterpret_cast<uint4*>(p.dU + off + c * 16);
-                oa[0] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
-                oa[1] = make_uint4(pa[4], pa[5], pa[6], pa[7]);
-                og[0] = make_uint4(pg[0], pg[1], pg[2], pg[3]);
-                og[1] = make_uint4(pg[4], pg[5], pg[6], pg[7]);
-                ou[0] = make_uint4(pu[0], pu[1], pu[2], pu[3]);
-                ou[1] = make_uint4(pu[4], pu[5], pu[6], pu[7]);
-            }
-            tc_fence_before_sync();
-            mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[2]), 0));
-            mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[slot]), 0));
-        }
-    }
-    pair_teardown(ctl, w);
-}
 
 }  // namespace tsp

@@ -53,6 +53,7 @@ struct tsp_mlp_plan {
     int shared_order;   // gate|up tile order: 1 = all ranks of a band on the same shard column block
     int group;          // token tiles per group in the down / dX tile order
     int pair_stages;
+    int last_backward_kernels;  // kernels launched by the most recent tsp_mlp_backward (3 or 4)
 };
 
 namespace {
@@ -313,15 +314,20 @@ tsp_status_t launch_pair(tsp_mlp_plan_t* plan, Kernel kernel, const Params& p, c
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
 
-tsp_status_t launch_gate_up_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A, int64_t S,
-                                 cudaStream_t stream) {
+template <bool kBackward>
+tsp_status_t launch_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A,
+                              const float* dA, void* dG, void* dU, int64_t S, cudaStream_t stream) {
+    using Policy = tsp::PairGateUpPolicyT<kBackward>;
     const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
-    tsp::PairGateUpPolicy::Params p;
+    typename Policy::Params p;
     std::memset(&p, 0, sizeof(p));
     if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
     if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
     if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
     p.A = static_cast<__nv_bfloat16*>(A);
+    p.dA = dA;
+    p.dG = static_cast<__nv_bfloat16*>(dG);
+    p.dU = static_cast<__nv_bfloat16*>(dU);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.F_d = F_d;
     p.m_tiles = static_cast<int>(S / 256);
@@ -330,7 +336,28 @@ tsp_status_t launch_gate_up_pair(tsp_mlp_plan_t* plan, const void* X, const void
     p.band = gate_band(plan, p.m_tiles);
     p.shared_order = plan->shared_order;
     fill_common(plan, p, p.m_tiles * D * p.jl_blocks);
-    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairGateUpPolicy>, p, stream);
+    return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
+}
+
+tsp_status_t launch_gate_up_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A, int64_t S,
+                                 cudaStream_t stream) {
+    return launch_gate_pair<false>(plan, X, Wg, Wu, A, nullptr, nullptr, nullptr, S, stream);
+}
+
+// dA = dY Wd^T in fp32 (needs F % 256 == 0)
+tsp_status_t launch_da_pair(tsp_mlp_plan_t* plan, const void* dY, const void* Wd, float* dA, int64_t S, cudaStream_t stream) {
+    const int H = plan->H, F = plan->F, D = plan->D;
+    tsp::PairDaPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 128)) return TSP_ERR_CUDA;
+    p.dA = dA;
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.m_tiles = static_cast<int>(S / 256);
+    p.j_tiles = F / 256;
+    p.band = gate_band(plan, p.m_tiles);
+    fill_common(plan, p, p.m_tiles * p.j_tiles);
+    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDaPolicy>, p, stream);
 }
 
 tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* Wd, void* Y, int64_t S, cudaStream_t stream) {
@@ -348,29 +375,6 @@ tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* W
     p.group = p.m_tiles < group ? p.m_tiles : group;
     fill_common(plan, p, p.m_tiles * p.n_blocks);
     return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownPolicy>, p, stream);
-}
-
-tsp_status_t launch_bwd_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
-                                  const void* dY, void* A, void* dG, void* dU, int64_t S, cudaStream_t stream) {
-    const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
-    tsp::PairBwdGateParams p;
-    std::memset(&p, 0, sizeof(p));
-    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
-    if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 128)) return TSP_ERR_CUDA;
-    if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
-    if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
-    if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 64)) return TSP_ERR_CUDA;
-    p.A = static_cast<__nv_bfloat16*>(A);
-    p.dG = static_cast<__nv_bfloat16*>(dG);
-    p.dU = static_cast<__nv_bfloat16*>(dU);
-    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
-    p.m_tiles = static_cast<int>(S / 256);
-    p.tiles_per_rank = static_cast<int>(S / D / 256);
-    p.jl_blocks = F_d / 128;
-    p.band = gate_band(plan, p.m_tiles);
-    p.shared_order = plan->shared_order;
-    fill_common(plan, p, p.m_tiles * D * p.jl_blocks);
-    return launch_pair(plan, tsp::pair_bwd_gate_kernel, p, stream);
 }
 
 tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void* dU, const void* Wg, const void* Wu,
@@ -513,6 +517,7 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->shared_order = env_int("TSP_MLP_GATE_ORDER", 1);
     plan->group = env_int("TSP_MLP_GROUP", 0);
     plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
+    plan->last_backward_kernels = 3;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
@@ -543,7 +548,7 @@ tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan) {
 size_t tsp_mlp_workspace_bytes(const tsp_mlp_plan_t* plan, int64_t S, int pass) {
     if (!plan || S <= 0 || (pass != TSP_WS_FORWARD && pass != TSP_WS_BACKWARD)) return 0;
     const size_t one = align_up(static_cast<size_t>(S) * plan->F * 2, 256);
-    return pass == TSP_WS_BACKWARD ? 3 * one : one;
+    return pass == TSP_WS_BACKWARD ? 5 * one : one;   // A, dG, dU in bf16 and dA in fp32
 }
 
 size_t tsp_mlp_workspace_bytes_host(const tsp_mlp_plan_t* plan, int64_t S) {
@@ -631,8 +636,16 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
     void* dU = base + 2 * one;
     Profiler prof(plan, stream);
     const bool pairs = pairs_for_tokens(plan, S);
-    st = pairs ? launch_bwd_gate_pair(plan, X, Wg, Wu, Wd, dY, A, dG, dU, S, stream)
-               : launch_bwd_gate(plan, X, Wg, Wu, Wd, dY, A, dG, dU, S, stream);
+    if (pairs && plan->F % 256 == 0) {
+        // dA in fp32 by a full-rate GEMM, then the gate|up GEMM whose epilogue consumes it
+        float* dA = reinterpret_cast<float*>(base + 3 * one);
+        st = launch_da_pair(plan, dY, Wd, dA, S, stream);
+        if (st != TSP_OK) return st;
+        prof.mark();
+        st = launch_gate_pair<true>(plan, X, Wg, Wu, A, dA, dG, dU, S, stream);
+    } else {
+        st = launch_bwd_gate(plan, X, Wg, Wu, Wd, dY, A, dG, dU, S, stream);
+    }
     if (st != TSP_OK) return st;
     prof.mark();
     st = pairs ? launch_bwd_dx_pair(plan, dG, dU, Wg, Wu, dX, S, stream)
@@ -643,6 +656,7 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
                             : launch_bwd_dw(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream);
     if (st != TSP_OK) return st;
     prof.mark();
+    plan->last_backward_kernels = (pairs && plan->F % 256 == 0) ? 4 : 3;
     return TSP_OK;
 }
 
@@ -765,7 +779,7 @@ tsp_status_t tsp_mlp_profile_end(tsp_mlp_plan_t* plan) {
 
 int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass) {
     if (!plan) return 0;
-    return pass == TSP_WS_BACKWARD ? 3 : 2;
+    return pass == TSP_WS_BACKWARD ? plan->last_backward_kernels : 2;
 }
 
 }  // extern "C"
