@@ -149,6 +149,15 @@ tsp_status_t tsp_mlp_forward_static(int H, int F, int D, const void* X, const vo
  */
 tsp_status_t tsp_mlp_status(tsp_mlp_plan_t* plan);
 
+/*
+ * tsp_mlp_selftest_wait_expiry - exercise the bounded-wait error path (no counterpart in the paper).
+ * Launches one warp that waits, for at most `limit_ms` (1..1000), on a barrier nothing arrives on.  The
+ * wait expires, the kernel sets the plan's status word and returns normally; after a synchronize,
+ * tsp_mlp_status reports TSP_ERR_DEVICE_TIMEOUT (and clears the word) and the plan stays usable.
+ * Nothing faults, traps or hangs.
+ */
+tsp_status_t tsp_mlp_selftest_wait_expiry(tsp_mlp_plan_t* plan, int limit_ms, void* cuda_stream);
+
 /* Static, never-null description of a status code. */
 const char* tsp_mlp_error_string(tsp_status_t status);
 /* The cudaError_t / CUresult value of the last failed CUDA call on this plan (0 if none). */

@@ -37,6 +37,7 @@ SIGNATURES = {
     "tsp_mlp_backward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_forward_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, _P,
                                               ctypes.c_int64, ctypes.POINTER(ctypes.c_int), _P]),
+    "tsp_mlp_selftest_wait_expiry": (ctypes.c_int, [_P, ctypes.c_int, _P]),
     "tsp_mlp_status": (ctypes.c_int, [_P]),
     "tsp_mlp_error_string": (ctypes.c_char_p, [ctypes.c_int]),
     "tsp_mlp_last_cuda_error": (ctypes.c_int, [_P]),
@@ -164,6 +165,12 @@ def tsp_mlp_forward_static(H: int, F: int, D: int, X, Wg, Wu, Wd, Y, S: int, tim
     ref = ctypes.byref(timed_out) if timed_out is not None else None
     _check(load_library().tsp_mlp_forward_static(H, F, D, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(Y), S, ref,
                                                  _stream_handle(stream)), "tsp_mlp_forward_static")
+
+
+def tsp_mlp_selftest_wait_expiry(plan, limit_ms: int = 20, stream=None) -> None:
+    """Make one bounded device-side wait expire on purpose (sets the plan's status word; harmless)."""
+    _check(load_library().tsp_mlp_selftest_wait_expiry(plan, limit_ms, _stream_handle(stream)),
+           "tsp_mlp_selftest_wait_expiry", plan)
 
 
 def tsp_mlp_status(plan) -> int:

@@ -20,7 +20,8 @@ constexpr int kEpilogueThreads = 128;
 constexpr uint32_t kTmemCols = 512;
 
 // Error codes written to the device status word (first one wins).
-constexpr int kErrWaitEmpty = 1, kErrWaitFull = 2, kErrWaitTmemEmpty = 3, kErrWaitTmemFull = 4, kErrTeardown = 5;
+constexpr int kErrWaitEmpty = 1, kErrWaitFull = 2, kErrWaitTmemEmpty = 3, kErrWaitTmemFull = 4, kErrTeardown = 5,
+              kErrSelfTest = 6;
 
 struct __align__(16) SharedCtl {
     uint64_t full[kMaxStages];
@@ -150,6 +151,24 @@ __device__ __forceinline__ void cta_teardown(SharedCtl* ctl, int stages, const W
         __syncwarp();
         tmem_dealloc(ctl->tmem_base, kTmemCols);
     }
+}
+
+// One warp waits, with the usual bound, on a barrier that nothing ever arrives on: the wait expires, the status
+// word is set and the kernel returns normally.  Proves the error path without faulting or hanging anything.
+__global__ void wait_expiry_selftest_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        WaitCtx w{&abort_flag, status, limit_ns};
+        wait_bar(smem_u32(&bar), 0, w, kErrSelfTest);
+    }
+    __syncthreads();
 }
 
 // ---- epilogue helpers ---------------------------------------------------------------------------

@@ -717,6 +717,14 @@ tsp_status_t tsp_mlp_status(tsp_mlp_plan_t* plan) {
     return TSP_OK;
 }
 
+tsp_status_t tsp_mlp_selftest_wait_expiry(tsp_mlp_plan_t* plan, int limit_ms, void* cuda_stream) {
+    if (!plan || limit_ms <= 0 || limit_ms > 1000) return TSP_ERR_INVALID_ARG;
+    tsp::wait_expiry_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        plan->status_dev, static_cast<unsigned long long>(limit_ms) * 1000 * 1000);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
+}
+
 const char* tsp_mlp_error_string(tsp_status_t s) {
     switch (s) {
         case TSP_OK: return "ok";
