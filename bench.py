@@ -243,8 +243,11 @@ def run_gpu(args, wl):
     X, Wg, Wu, Wd = dev(host.X), dev(Wg_h), dev(Wu_h), dev(Wd_h)
     Y = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
     plan = b.tsp_mlp_plan(H, F, D)
+    staged = args.mode == "staged"
     ws_bytes = max(b.tsp_mlp_workspace_bytes(plan, S, b.TSP_WS_BACKWARD if train else b.TSP_WS_FORWARD),
-                   b.tsp_mlp_workspace_bytes_host(plan, S))
+                   b.tsp_mlp_workspace_bytes_host(plan, S),
+                   b.tsp_mlp_workspace_bytes_staged(plan, S) if staged else 0)
+    copy_stream = torch.cuda.Stream() if staged else None
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     b.tsp_mlp_set_workspace(plan, ws)
     if train:
@@ -255,7 +258,10 @@ def run_gpu(args, wl):
         dWd = torch.empty(D, F // D, H, dtype=torch.float32, device="cuda")
 
     def step():
-        b.tsp_mlp_forward(plan, X, Wg, Wu, Wd, Y, S, D)
+        if staged:
+            b.tsp_mlp_forward_staged(plan, X, Wg, Wu, Wd, Y, S, D, torch.cuda.current_stream(), copy_stream)
+        else:
+            b.tsp_mlp_forward(plan, X, Wg, Wu, Wd, Y, S, D)
         if train:
             b.tsp_mlp_backward(plan, X, Wg, Wu, Wd, dY, dX, dWg, dWu, dWd, S, D)
 
@@ -266,7 +272,7 @@ def run_gpu(args, wl):
     barrier()
     assert b.tsp_mlp_status(plan) == b.TSP_OK, "device-side wait timed out during warm-up"
     # counted after a call has been made: the backward count depends on the shape-dependent path taken
-    kernels_per_step = b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD) + (
+    kernels_per_step = (2 * D if staged else b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD)) + (
         b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_BACKWARD) if train else 0)
 
     # ---- timed region: K steps, inputs resident in HBM ----
@@ -301,7 +307,7 @@ def run_gpu(args, wl):
 
     # ---- end to end: host buffers in pinned memory, H2D + forward + D2H every step ----
     e2e = None
-    if not train and not args.no_e2e:
+    if not train and not args.no_e2e and not staged:
         hX = torch.from_numpy(host.X.view(np.int16)).pin_memory()
         hWg = torch.from_numpy(Wg_h.view(np.int16)).pin_memory()
         hWu = torch.from_numpy(Wu_h.view(np.int16)).pin_memory()
@@ -333,6 +339,22 @@ def run_gpu(args, wl):
         return
 
     peaks = measured_peaks()
+    if staged:
+        # staged mode records one interval for the whole call; no per-kernel split
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "pass": "forward", "mode": "staged (ring copies on a side stream)",
+                       "S": S, "H": H, "F": F, "D": D, "ring_copy_bytes_per_step": (D - 1) * 6 * H * F},
+            "clocks": sampler.summary(), "gpu_launches": int(args.steps * kernels_per_step),
+            "e2e": None, "roofline": None, "cpu_baseline": None,
+        }
+        print(json.dumps(line), flush=True)
+        b.tsp_mlp_plan_destroy(plan)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     # dominant kernel: the gate|up GEMM with the SwiGLU epilogue (two thirds of the forward FLOPs)
     gate_up_ms = float(per_kernel[0])
     gate_up_flops = 4.0 * S * H * F
@@ -386,6 +408,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="7b_short", choices=sorted(inp.WORKLOADS))
     ap.add_argument("--backward", action="store_true", help="time forward + backward (as the `train` workload does)")
+    ap.add_argument("--mode", default="direct", choices=["direct", "staged"],
+                    help="staged: Algorithm 2 step by step with the shard transfer emulated on a side stream")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")

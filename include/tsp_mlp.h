@@ -110,6 +110,25 @@ tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, cons
                                   int64_t S, int D, void* cuda_stream);
 
 /*
+ * tsp_mlp_forward_staged - Algorithm 2 executed step by step, with the ring transfer stood in for by
+ * device-to-device copies on a second stream (Section 4.9: send/receive on a dedicated communication
+ * stream while the default stream computes; wait only when the next shard is needed).
+ * For t = 0..D-1: the copy stream moves every rank's current (Wg, Wu, Wd) buffers into the next rank's
+ * receive buffers (send to (p+1) mod D, receive from (p-1) mod D; two buffer sets alternate), while the
+ * compute stream runs step t for all ranks: the gate|up GEMM with the SwiGLU epilogue into a [S, F/D]
+ * scratch, then the down projection of that shard added into an fp32 [S, H] accumulator; the last step
+ * rounds the accumulator to bf16 Y.  Events order "received" before "compute t+1" and "computed t-1"
+ * before the buffers are overwritten.  Same result as tsp_mlp_forward up to fp32 summation order
+ * (per-shard partial sums are formed first).  Needs (S/D) % 256 == 0, two distinct streams, and a
+ * workspace of tsp_mlp_workspace_bytes_staged(plan, S) bytes (scratch, accumulator, 2 x 3 receive buffers
+ * of the size of one weight matrix).  2*D kernels and at most 6*(D-1) copies per call.
+ */
+size_t tsp_mlp_workspace_bytes_staged(const tsp_mlp_plan_t* plan, int64_t S);
+tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu,
+                                    const void* Wd, void* Y, int64_t S, int D, void* compute_stream,
+                                    void* copy_stream);
+
+/*
  * tsp_mlp_forward_static - the forward pass for callers that cannot obtain device memory at call time.
  * (The paper has no counterpart of this entry point; it exists for integration reasons only.)
  *

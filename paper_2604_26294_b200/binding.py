@@ -35,6 +35,8 @@ SIGNATURES = {
     "tsp_mlp_forward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_forward_host": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_backward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_mlp_workspace_bytes_staged": (ctypes.c_size_t, [_P, ctypes.c_int64]),
+    "tsp_mlp_forward_staged": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P, _P]),
     "tsp_mlp_forward_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, _P,
                                               ctypes.c_int64, ctypes.POINTER(ctypes.c_int), _P]),
     "tsp_mlp_selftest_wait_expiry": (ctypes.c_int, [_P, ctypes.c_int, _P]),
@@ -153,6 +155,17 @@ def tsp_mlp_backward(plan, X, Wg, Wu, Wd, dY, dX, dWg, dWu, dWd, S: int, D: int,
     _check(load_library().tsp_mlp_backward(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(dY), _ptr(dX),
                                            _ptr(dWg), _ptr(dWu), _ptr(dWd), S, D, _stream_handle(stream)),
            "tsp_mlp_backward", plan)
+
+
+def tsp_mlp_workspace_bytes_staged(plan, S: int) -> int:
+    return int(load_library().tsp_mlp_workspace_bytes_staged(plan, S))
+
+
+def tsp_mlp_forward_staged(plan, X, Wg, Wu, Wd, Y, S: int, D: int, compute_stream=None, copy_stream=None) -> None:
+    """Algorithm 2 step by step with the shard transfer emulated by copies on `copy_stream`."""
+    _check(load_library().tsp_mlp_forward_staged(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(Y), S, D,
+                                                 _stream_handle(compute_stream), _stream_handle(copy_stream)),
+           "tsp_mlp_forward_staged", plan)
 
 
 def tsp_mlp_forward_static(H: int, F: int, D: int, X, Wg, Wu, Wd, Y, S: int, timed_out=None, stream=None) -> None:

@@ -256,6 +256,8 @@ struct PairGateUpPolicyT {
         __nv_bfloat16* dU;    // [S, F] (backward only)
         int S, H, F, D, F_d;
         int m_tiles, tiles_per_rank, jl_blocks, band, shared_order;
+        int rank_indexed;     // staged mode: one ring step per launch; the weight tensors hold, at index r, the
+                              // shard rank r currently has in its receive buffer, and A is [S, F/D]
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -273,7 +275,8 @@ struct PairGateUpPolicyT {
     }
     // band of token tiles -> step t -> column block of the shard -> token tile
     __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
-        const int per_band = p.band * p.D * p.jl_blocks;
+        const int steps = p.rank_indexed ? 1 : p.D;
+        const int per_band = p.band * steps * p.jl_blocks;
         const int band_idx = tile / per_band;
         const int band_start = band_idx * p.band;
         const int band_sz = min(p.band, p.m_tiles - band_start);
@@ -284,7 +287,7 @@ struct PairGateUpPolicyT {
         o.jl = rem / band_sz;
         o.mt = band_start + rem % band_sz;
         const int r = o.mt / p.tiles_per_rank;
-        o.k = p.shared_order ? t : (r - t + p.D) % p.D;
+        o.k = p.rank_indexed ? r : (p.shared_order ? t : (r - t + p.D) % p.D);
         return o;
     }
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int k, int kb, uint32_t cta,
@@ -293,8 +296,9 @@ struct PairGateUpPolicyT {
         pair_load_mnmajor(sb, cta == 0 ? &p.map_wg : &p.map_wu, bar, tl.jl * 128, kb * kBK, k, 2);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F + static_cast<size_t>(tl.k) * p.F_d +
-                           tl.jl * 128;
+        // p.F is the row pitch of A: F in direct mode, F/D in staged mode (where the shard offset is dropped)
+        const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F +
+                           (p.rank_indexed ? 0 : static_cast<size_t>(tl.k) * p.F_d) + tl.jl * 128;
         if constexpr (!kBackward) {
             __nv_bfloat16* out = p.A + off;
 #pragma unroll 1
@@ -462,6 +466,82 @@ struct PairDownPolicy {
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
+    }
+};
+
+// ---- staged mode, one ring step: Y_acc (fp32) += A_step Wd_cur, K = F/D.  The weights of rank r are read from
+// index r of the receive buffer.  mode 0: first step (store), 1: middle (add), 2: last (add, round to bf16 Y),
+// 3: only step (D = 1: round to bf16 Y directly).
+struct PairDownStagedPolicy {
+    static constexpr bool kAMn = false, kBMn = true;
+    struct Params {
+        CUtensorMap map_a, map_wd;  // A_step (F/D, S, 1) box (64,128); Wd buffers (H, F/D, D) box (64,64)
+        float* Yacc;                // [S, H] fp32
+        __nv_bfloat16* Y;           // [S, H]
+        int S, H, F_d, D, mode;
+        int m_tiles, n_blocks, tiles_per_rank, group;
+        int num_tiles, stages;
+        int* status;
+        unsigned long long timeout_ns;
+    };
+    using Tile = PairDownPolicy::Tile;
+    __device__ static __forceinline__ int outer(const Params&) { return 1; }
+    __device__ static __forceinline__ int inner(const Params& p) { return p.F_d / kBK; }
+    __device__ static __forceinline__ int select(const Params&, const Tile& tl, int) { return tl.r; }
+    __device__ static __forceinline__ void prefetch(const Params& p) {
+        tma_prefetch_desc(&p.map_a);
+        tma_prefetch_desc(&p.map_wd);
+    }
+    __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
+        const int per_group = p.group * p.n_blocks;
+        const int g = tile / per_group;
+        const int g_start = g * p.group;
+        const int g_sz = min(p.group, p.m_tiles - g_start);
+        const int rem = tile - g * per_group;
+        Tile o;
+        o.nb = rem / g_sz;
+        o.mt = g_start + rem % g_sz;
+        o.r = o.mt / p.tiles_per_rank;
+        return o;
+    }
+    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int r, int i, uint32_t cta, uint32_t sa,
+                                                uint32_t sb, uint32_t bar) {
+        pair_load_kmajor(sa, &p.map_a, bar, i * kBK, tl.mt * 256 + cta * 128, 0);
+        pair_load_mnmajor(sb, &p.map_wd, bar, tl.nb * 256 + cta * 128, i * kBK, r, 2);
+    }
+    __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
+        const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256;
+        float4* acc = reinterpret_cast<float4*>(p.Yacc + off);
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+            float4 prev[8];
+            if (p.mode == 1 || p.mode == 2) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) prev[q] = acc[c * 8 + q];
+            }
+            uint32_t v[32];
+            tmem_ld32(t_row + c * 32, v);
+            tmem_ld_wait();
+            float f[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
+            if (p.mode == 1 || p.mode == 2) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    f[4 * q] += prev[q].x; f[4 * q + 1] += prev[q].y; f[4 * q + 2] += prev[q].z; f[4 * q + 3] += prev[q].w;
+                }
+            }
+            if (p.mode <= 1) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc[c * 8 + q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+            } else {
+                uint4* dst = reinterpret_cast<uint4*>(p.Y + off + c * 32);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    dst[q] = make_uint4(pack_bf16x2(f[8 * q], f[8 * q + 1]), pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
+                                        pack_bf16x2(f[8 * q + 4], f[8 * q + 5]), pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+            }
+        }
     }
 };
 

@@ -54,6 +54,7 @@ struct tsp_mlp_plan {
     int group;          // token tiles per group in the down / dX tile order
     int pair_stages;
     int last_backward_kernels;  // kernels launched by the most recent tsp_mlp_backward (3 or 4)
+    std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
 };
 
 namespace {
@@ -540,6 +541,7 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
 tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan) {
     if (!plan) return TSP_ERR_INVALID_ARG;
     tsp_mlp_profile_end(plan);
+    for (auto& ev : plan->staged_events) cudaEventDestroy(ev);
     if (plan->status_dev) cudaFree(plan->status_dev);
     delete plan;
     return TSP_OK;
@@ -614,6 +616,129 @@ tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, cons
     st = tsp_mlp_forward(plan, dX, dWg, dWu, dWd, dY, S, D, cuda_stream);
     if (st != TSP_OK) return st;
     if ((e = cudaMemcpyAsync(Y_host, dY, xb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    return TSP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// STAGED mode: Algorithm 2 step by step.  Every ring step is its own pair of launches on the compute
+// stream; meanwhile the copy stream moves each rank's current shard buffers into the next rank's
+// receive buffers (the stand-in for AsyncRingSendRecv); events implement Wait() and the buffer swap.
+// ---------------------------------------------------------------------------------------------
+size_t tsp_mlp_workspace_bytes_staged(const tsp_mlp_plan_t* plan, int64_t S) {
+    if (!plan || S <= 0) return 0;
+    const size_t a_step = align_up(static_cast<size_t>(S) * (plan->F / plan->D) * 2, 256);
+    const size_t y_acc = align_up(static_cast<size_t>(S) * plan->H * 4, 256);
+    const size_t w = align_up(static_cast<size_t>(plan->H) * plan->F * 2, 256);  // one matrix, all D receive buffers
+    return a_step + y_acc + 2 * 3 * w;
+}
+
+tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu,
+                                    const void* Wd, void* Y, int64_t S, int D, void* compute_stream,
+                                    void* copy_stream) {
+    tsp_status_t st = check_call(plan, S, D);
+    if (st != TSP_OK) return st;
+    if (!X || !Wg || !Wu || !Wd || !Y) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(Y)) return TSP_ERR_INVALID_ARG;
+    if (compute_stream == copy_stream) return TSP_ERR_INVALID_ARG;
+    if ((S / D) % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_staged(plan, S)) return TSP_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(compute_stream), xs = static_cast<cudaStream_t>(copy_stream);
+    const int H = plan->H, F = plan->F, F_d = F / D;
+    const size_t a_step_bytes = align_up(static_cast<size_t>(S) * F_d * 2, 256);
+    const size_t y_acc_bytes = align_up(static_cast<size_t>(S) * H * 4, 256);
+    const size_t w = align_up(static_cast<size_t>(H) * F * 2, 256);
+    const size_t shard_bytes = static_cast<size_t>(H) * F_d * 2;
+    uint8_t* base = static_cast<uint8_t*>(plan->workspace);
+    void* A_step = base;
+    float* Yacc = reinterpret_cast<float*>(base + a_step_bytes);
+    uint8_t* rb = base + a_step_bytes + y_acc_bytes;  // receive buffers [parity][matrix][rank]
+    auto recv = [&](int parity, int m) { return rb + (static_cast<size_t>(parity) * 3 + m) * w; };
+    const void* own[3] = {Wg, Wu, Wd};
+
+    const size_t need_events = 2 * static_cast<size_t>(D) + 2;
+    while (plan->staged_events.size() < need_events) {
+        cudaEvent_t ev;
+        cudaError_t e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail(plan, e);
+        plan->staged_events.push_back(ev);
+    }
+    auto ev_recv = [&](int t) { return plan->staged_events[2 * t]; };
+    auto ev_done = [&](int t) { return plan->staged_events[2 * t + 1]; };
+    cudaError_t e;
+    // the copy stream starts after whatever precedes this call on the compute stream
+    cudaEvent_t ev_start = plan->staged_events[2 * D];
+    if ((e = cudaEventRecord(ev_start, cs)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaStreamWaitEvent(xs, ev_start, 0)) != cudaSuccess) return cuda_fail(plan, e);
+
+    Profiler prof(plan, cs);
+    for (int t = 0; t < D; ++t) {
+        // ---- AsyncRingSendRecv for step t + 1: rank r's primed buffers <- rank (r-1)'s current buffers
+        if (t < D - 1) {
+            // the primed buffers (parity (t+1)&1) were last read by the compute of step t-1
+            if (t >= 1 && (e = cudaStreamWaitEvent(xs, ev_done(t - 1), 0)) != cudaSuccess) return cuda_fail(plan, e);
+            for (int m = 0; m < 3; ++m) {
+                const uint8_t* cur = t == 0 ? static_cast<const uint8_t*>(own[m]) : recv(t & 1, m);
+                uint8_t* dst = recv((t + 1) & 1, m);
+                // ranks 1..D-1 receive from ranks 0..D-2 (one contiguous block), rank 0 from rank D-1
+                if (D > 1) {
+                    if ((e = cudaMemcpyAsync(dst + shard_bytes, cur, shard_bytes * (D - 1), cudaMemcpyDeviceToDevice, xs)) !=
+                        cudaSuccess)
+                        return cuda_fail(plan, e);
+                }
+                if ((e = cudaMemcpyAsync(dst, cur + shard_bytes * (D - 1), shard_bytes, cudaMemcpyDeviceToDevice, xs)) !=
+                    cudaSuccess)
+                    return cuda_fail(plan, e);
+            }
+            if ((e = cudaEventRecord(ev_recv(t + 1), xs)) != cudaSuccess) return cuda_fail(plan, e);
+        }
+        // ---- compute of step t with the current buffers
+        if (t >= 1 && (e = cudaStreamWaitEvent(cs, ev_recv(t), 0)) != cudaSuccess) return cuda_fail(plan, e);  // Wait()
+        const void* cur_g = t == 0 ? Wg : recv(t & 1, 0);
+        const void* cur_u = t == 0 ? Wu : recv(t & 1, 1);
+        const void* cur_d = t == 0 ? Wd : recv(t & 1, 2);
+        {
+            using Policy = tsp::PairGateUpPolicyT<false>;
+            Policy::Params p;
+            std::memset(&p, 0, sizeof(p));
+            if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+            if (!encode_sharded(plan, &p.map_wg, cur_g, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+            if (!encode_sharded(plan, &p.map_wu, cur_u, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+            p.A = static_cast<__nv_bfloat16*>(A_step);
+            p.S = static_cast<int>(S); p.H = H; p.F = F_d; p.D = D; p.F_d = F_d;
+            p.m_tiles = static_cast<int>(S / 256);
+            p.tiles_per_rank = static_cast<int>(S / D / 256);
+            p.jl_blocks = F_d / 128;
+            p.band = gate_band(plan, p.m_tiles);
+            p.rank_indexed = 1;
+            fill_common(plan, p, p.m_tiles * p.jl_blocks);
+            st = launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, cs);
+            if (st != TSP_OK) return st;
+        }
+        {
+            tsp::PairDownStagedPolicy::Params p;
+            std::memset(&p, 0, sizeof(p));
+            if (!encode_matrix(plan, &p.map_a, A_step, S, F_d, 64, 128)) return TSP_ERR_CUDA;
+            if (!encode_sharded(plan, &p.map_wd, cur_d, D, F_d, H, 64, 64)) return TSP_ERR_CUDA;
+            p.Yacc = Yacc;
+            p.Y = static_cast<__nv_bfloat16*>(Y);
+            p.S = static_cast<int>(S); p.H = H; p.F_d = F_d; p.D = D;
+            p.mode = D == 1 ? 3 : (t == 0 ? 0 : (t == D - 1 ? 2 : 1));
+            p.m_tiles = static_cast<int>(S / 256);
+            p.n_blocks = H / 256;
+            p.tiles_per_rank = static_cast<int>(S / D / 256);
+            const int group = plan->group > 0 ? plan->group : 8;
+            p.group = p.m_tiles < group ? p.m_tiles : group;
+            fill_common(plan, p, p.m_tiles * p.n_blocks);
+            st = launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownStagedPolicy>, p, cs);
+            if (st != TSP_OK) return st;
+        }
+        if ((e = cudaEventRecord(ev_done(t), cs)) != cudaSuccess) return cuda_fail(plan, e);
+    }
+    prof.mark();
+    // later work on the copy stream must not overtake this call: join it back
+    cudaEvent_t ev_end = plan->staged_events[2 * D + 1];
+    if ((e = cudaEventRecord(ev_end, xs)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaStreamWaitEvent(cs, ev_end, 0)) != cudaSuccess) return cuda_fail(plan, e);
     return TSP_OK;
 }
 
