@@ -54,6 +54,7 @@ struct tsp_mlp_plan {
     int group;          // token tiles per group in the down / dX tile order
     int pair_stages;
     int last_backward_kernels;  // kernels launched by the most recent tsp_mlp_backward (3 or 4)
+    int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
 };
 
@@ -519,6 +520,7 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->group = env_int("TSP_MLP_GROUP", 0);
     plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
     plan->last_backward_kernels = 3;
+    plan->phase_mask = env_int("TSP_MLP_PHASES", 3);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
@@ -580,13 +582,17 @@ tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     Profiler prof(plan, stream);
     const bool pairs = pairs_for_tokens(plan, S);
-    st = pairs ? launch_gate_up_pair(plan, X, Wg, Wu, plan->workspace, S, stream)
-               : launch_gate_up(plan, X, Wg, Wu, plan->workspace, S, stream);
-    if (st != TSP_OK) return st;
+    if (plan->phase_mask & 1) {
+        st = pairs ? launch_gate_up_pair(plan, X, Wg, Wu, plan->workspace, S, stream)
+                   : launch_gate_up(plan, X, Wg, Wu, plan->workspace, S, stream);
+        if (st != TSP_OK) return st;
+    }
     prof.mark();
-    st = pairs ? launch_down_pair(plan, plan->workspace, Wd, Y, S, stream)
-               : launch_down(plan, plan->workspace, Wd, Y, S, stream);
-    if (st != TSP_OK) return st;
+    if (plan->phase_mask & 2) {
+        st = pairs ? launch_down_pair(plan, plan->workspace, Wd, Y, S, stream)
+                   : launch_down(plan, plan->workspace, Wd, Y, S, stream);
+        if (st != TSP_OK) return st;
+    }
     prof.mark();
     return TSP_OK;
 }
