@@ -604,6 +604,7 @@ struct PairDwPolicy {
         float* dWu;
         int S, H, F, D, F_d, S_loc;
         int j_tiles, n_blocks, j_tiles_per_shard;
+        int n_group;   // hidden blocks per group: their columns of X / dY stay in L2 while the [S,F] operand streams
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -626,12 +627,18 @@ struct PairDwPolicy {
         tma_prefetch_desc(&p.map_x);
     }
     __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
+        // family (dWd, dWg, dWu) -> group of hidden blocks -> intermediate tile -> hidden block of the group
         Tile o;
         const int per_which = p.j_tiles * p.n_blocks;
         o.which = tile / per_which;
-        const int rem = tile - o.which * per_which;
-        o.jt = rem / p.n_blocks;
-        o.nb = rem - o.jt * p.n_blocks;
+        int rem = tile - o.which * per_which;
+        const int per_group = p.j_tiles * p.n_group;
+        const int g = rem / per_group;
+        const int g_start = g * p.n_group;
+        const int g_sz = min(p.n_group, p.n_blocks - g_start);
+        rem -= g * per_group;
+        o.jt = rem / g_sz;
+        o.nb = g_start + rem - o.jt * g_sz;
         o.k = o.jt / p.j_tiles_per_shard;
         return o;
     }

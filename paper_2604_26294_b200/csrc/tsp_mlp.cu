@@ -54,6 +54,8 @@ struct tsp_mlp_plan {
     int group;          // token tiles per group in the down / dX tile order
     int pair_stages;
     int last_backward_kernels;  // kernels launched by the most recent tsp_mlp_backward (3 or 4)
+    int dw_group;               // hidden blocks per group in the dW tile order
+    int dx_group;               // token tiles per group in the dX tile order
     int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
 };
@@ -139,7 +141,10 @@ struct Profiler {
 
 // Token tiles (of 256 rows) per band of the gate|up tile order.
 int gate_band(const tsp_mlp_plan_t* plan, int m_tiles) {
-    int band = plan->band > 0 ? plan->band : 8;   // 8 tiles of 256 tokens: 16 MB of X at H = 4096
+    // default: the band's rows of X (256 * band * H * 2 bytes) take about 32 MB, a quarter of L2, so they stay
+    // resident while the weights stream past once per band (16 tiles at H = 4096)
+    int band = plan->band > 0 ? plan->band : static_cast<int>((32ull << 20) / (512ull * plan->H));
+    if (band < 1) band = 1;
     return band > m_tiles ? m_tiles : band;
 }
 
@@ -393,7 +398,7 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
     p.m_tiles = static_cast<int>(S / 256);
     p.n_blocks = H / 256;
     p.tiles_per_rank = static_cast<int>(S / D / 256);
-    const int group = plan->group > 0 ? plan->group : 8;
+    const int group = plan->dx_group > 0 ? plan->dx_group : 8;
     p.group = p.m_tiles < group ? p.m_tiles : group;
     fill_common(plan, p, p.m_tiles * p.n_blocks);
     return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDxPolicy>, p, stream);
@@ -416,6 +421,10 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     p.j_tiles = F / 256;
     p.j_tiles_per_shard = p.F_d / 256;
     p.n_blocks = H / 256;
+    // hidden blocks are taken in groups whose columns of X / dY (S * 512 bytes per block) fit in about 32 MB of L2
+    int n_group = plan->dw_group > 0 ? plan->dw_group : static_cast<int>((32ull << 20) / (512ull * static_cast<size_t>(S)));
+    if (n_group < 1) n_group = 1;
+    p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
     fill_common(plan, p, 3 * p.j_tiles * p.n_blocks);
     return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDwPolicy>, p, stream);
 }
@@ -521,6 +530,8 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
     plan->last_backward_kernels = 3;
     plan->phase_mask = env_int("TSP_MLP_PHASES", 3);
+    plan->dw_group = env_int("TSP_MLP_DW_GROUP", 0);
+    plan->dx_group = env_int("TSP_MLP_DX_GROUP", 0);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
