@@ -62,6 +62,8 @@ WORKLOADS = {
     "sweep_d8": Workload("sweep_d8", S=16384, H=4096, F=14336, D=8),
     "sweep_d16": Workload("sweep_d16", S=16384, H=4096, F=14336, D=16),
     "train": Workload("train", S=8192, H=4096, F=14336, D=8),
+    # the paper's own 7B-class MLP: expansion factor 4, intermediate width 4 * 4096 (reference-model table)
+    "7b_paper": Workload("7b_paper", S=8192, H=4096, F=16384, D=8),
 }
 
 

@@ -46,6 +46,9 @@ def test_tiny_config_full_compare():
     (512, 512, 1536, 4),
     (1536, 768, 1280, 2),
     (2048, 256, 2048, 16),
+    (2304, 256, 1536, 3),    # D = 3, pair path incl. the split backward (F % 256 == 0) and pair dW (512 per shard)
+    (2304, 256, 1152, 3),    # D = 3, pair tokens but 384-wide shards: single-CTA dW, fused single-CTA gate kernel
+    (3840, 512, 1280, 5),    # D = 5
 ])
 def test_multi_tile_shapes_full_compare(S, H, F, D):
     _check_full(S, H, F, D, seed=1)

@@ -39,6 +39,9 @@ def test_tiny_config_full_compare():
     (512, 512, 1536, 4),     # several tiles, 3 column blocks per shard
     (1536, 768, 1280, 2),    # H = 3 x 256, 5 column blocks per shard, 12 token blocks
     (2048, 256, 2048, 16),   # D = 16 with the narrowest shard (128)
+    (2304, 256, 1152, 3),    # D = 3: 768 tokens and 384 columns per rank, 9 pair tiles (odd), 3 column blocks
+    (3840, 512, 1280, 5),    # D = 5: 15 pair tiles, band / group sizes do not divide the tile counts
+    (384, 256, 384, 3),      # D = 3 on the single-CTA path (128 tokens per rank)
 ])
 def test_multi_tile_shapes_full_compare(S, H, F, D):
     _check_full(S, H, F, D, seed=1)

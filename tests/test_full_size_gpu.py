@@ -48,6 +48,14 @@ def test_7b_short_forward_sampled_rows():
     _check_forward_rows(prob, Y, inp.sample_rows(wl.S, wl.D), _weights64(prob.host))
 
 
+def test_paper_7b_shape_forward_sampled_rows():
+    # the paper's own MLP shape: intermediate width 4 * h = 16384 (2048 per shard at D = 8)
+    wl = inp.WORKLOADS["7b_paper"]
+    prob = DeviceProblem(wl.S, wl.H, wl.F, wl.D, seed=0)
+    Y = prob.forward()
+    _check_forward_rows(prob, Y, inp.sample_rows(wl.S, wl.D), _weights64(prob.host))
+
+
 def test_7b_long_forward_sampled_rows():
     wl = inp.WORKLOADS["7b_long"]
     prob = DeviceProblem(wl.S, wl.H, wl.F, wl.D, seed=0)
