@@ -224,6 +224,108 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
     pair_teardown(ctl, w);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Wide pair kernel for the long-K GEMMs: tile = 256 rows x 512 columns, ONE accumulator set that fills all 512
+// tensor-memory columns.  Per k-block each CTA loads 128 rows of A once (16 KB) and two half-B blocks (2 x 16 KB);
+// the leader issues two N = 256 MMAs per k-step that share the A descriptor.  Compared with the 256 x 256 tile this
+// moves 48 KB instead of 64 KB per CTA pair and tile-k-block from L2, and a wave of 74 pairs spans twice the columns,
+// which halves the DRAM re-reads of the row operand.  The price: the epilogue no longer overlaps the next main
+// loop (the two column halves are released separately, so the first half of the next tile starts early); worth it
+// when K is long (down projection, dX, dW).
+// Policy additionally provides load_wide(p, tile, sel, i, cta, sa, sb, bar) and epilogue_half(p, tile, cta, row, t_row, h).
+// ------------------------------------------------------------------------------------------------
+constexpr uint32_t kWideStageBytes = 48 * 1024;
+
+template <class Policy>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
+pair_wide_kernel(const __grid_constant__ typename Policy::Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_1024(smem_raw);
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + p.stages * kWideStageBytes);
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta = cluster_ctarank();
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+    pair_setup(ctl, p.stages, 2);   // tmem_empty[h]: column half h drained; tmem_full[0]: whole tile accumulated
+    const uint32_t tmem_base = ctl->tmem_base;
+    WaitCtx w{&ctl->abort, p.status, p.timeout_ns};
+    const int n_outer = Policy::outer(p), n_inner = Policy::inner(p);
+    const int k_blocks = n_outer * n_inner;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            Policy::prefetch(p);
+            PipeState ps;
+            bool ok = true;
+            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs) {
+                const typename Policy::Tile tl = Policy::decode(p, tile);
+                for (int o = 0; o < n_outer && ok; ++o) {
+                    const int sel = Policy::select(p, tl, o);
+                    for (int i = 0; i < n_inner; ++i) {
+                        if (!(ok = wait_bar(smem_u32(&ctl->empty[ps.stage]), ps.phase ^ 1u, w, kErrWaitEmpty))) break;
+                        const uint32_t bar = map_to_cta(smem_u32(&ctl->full[ps.stage]), 0);
+                        const uint32_t sa = smem_base + ps.stage * kWideStageBytes, sb = sa + kPairABytes;
+                        if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), 2 * kWideStageBytes);
+                        Policy::load_wide(p, tl, sel, i, cta, sa, sb, bar);
+                        ps.advance(p.stages);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && cta == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(256, 256, Policy::kAMn, Policy::kBMn);
+            PipeState ps;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
+                for (int kb = 0; kb < k_blocks && ok; ++kb) {
+                    if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_base + ps.stage * kWideStageBytes, sb = sa + kPairABytes;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (kb == 0) {  // the previous tile's epilogue must have drained this half
+                            if (!(ok = wait_bar(smem_u32(&ctl->tmem_empty[h]), (it & 1) ^ 1u, w, kErrWaitTmemEmpty))) break;
+                            tc_fence_after_sync();
+                        }
+                        pair_issue_kblock<Policy::kAMn, Policy::kBMn>(tmem_base + h * 256, sa, sb + h * 16384, idesc, kb > 0);
+                    }
+                    if (!ok) break;
+                    const uint32_t e = smem_u32(&ctl->empty[ps.stage]);
+                    umma_commit_pair(e);
+                    umma_commit_pair(map_to_cta(e, 1));
+                    ps.advance(p.stages);
+                }
+                if (ok) {
+                    const uint32_t f = smem_u32(&ctl->tmem_full[0]);
+                    umma_commit_pair(f);
+                    umma_commit_pair(map_to_cta(f, 1));
+                }
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        bool ok = true;
+        int it = 0;
+        for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
+            const typename Policy::Tile tl = Policy::decode(p, tile);
+            if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[0]), it & 1, w, kErrWaitTmemFull))) break;
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                Policy::epilogue_half(p, tl, cta, row, t_row + h * 256, h);
+                tc_fence_before_sync();
+                mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[h]), 0));
+            }
+        }
+    }
+    pair_teardown(ctl, w);
+}
+
 // ---- store helpers ---------------------------------------------------------------------------------
 __device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t_row) {
 #pragma unroll 1
@@ -467,6 +569,18 @@ struct PairDownPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
     }
+    // wide tile: tl.nb counts 512-column blocks
+    __device__ static __forceinline__ void load_wide(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
+                                                     uint32_t sa, uint32_t sb, uint32_t bar) {
+        const int f0 = k * p.F_d + i * kBK;
+        pair_load_kmajor(sa, &p.map_a, bar, f0, tl.mt * 256 + cta * 128, 0);
+        pair_load_mnmajor(sb, &p.map_wd, bar, tl.nb * 512 + cta * 128, f0, 0, 2);
+        pair_load_mnmajor(sb + 16384, &p.map_wd, bar, tl.nb * 512 + 256 + cta * 128, f0, 0, 2);
+    }
+    __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
+                                                         uint32_t t_row, int h) {
+        store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 512 + h * 256, t_row);
+    }
 };
 
 // ---- staged mode, one ring step: Y_acc (fp32) += A_step Wd_cur, K = F/D.  The weights of rank r are read from
@@ -592,6 +706,19 @@ struct PairDxPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_bf16_row256(p.dX + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
     }
+    __device__ static __forceinline__ void load_wide(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
+                                                     uint32_t sa, uint32_t sb, uint32_t bar) {
+        const int j0 = (i >> 1) * kBK;
+        const bool up = i & 1;
+        const CUtensorMap* mw = up ? &p.map_wu : &p.map_wg;
+        pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sb, mw, bar, j0, tl.nb * 512 + cta * 128, k);
+        pair_load_kmajor(sb + 16384, mw, bar, j0, tl.nb * 512 + 256 + cta * 128, k);
+    }
+    __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
+                                                         uint32_t t_row, int h) {
+        store_bf16_row256(p.dX + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 512 + h * 256, t_row);
+    }
 };
 
 // ---- weight gradients: tile = 256 intermediate columns x 256 hidden; K = all S tokens ------------------
@@ -650,7 +777,9 @@ struct PairDwPolicy {
         pair_load_mnmajor(sa, ma, bar, tl.jt * 256 + cta * 128, s0, 0, 2);
         pair_load_mnmajor(sb, mb, bar, tl.nb * 256 + cta * 128, s0, 0, 2);
     }
-    __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
+    // writes the 256 hidden columns starting at h_base for this lane's intermediate index
+    __device__ static __forceinline__ void store_cols(const Params& p, const Tile& tl, uint32_t cta, int row,
+                                                      uint32_t t_row, int h_base) {
         const int j = tl.jt * 256 + cta * 128 + row;  // global intermediate index of this lane
         const int F_d = p.F_d;
 #pragma unroll 1
@@ -658,7 +787,7 @@ struct PairDwPolicy {
             uint32_t v[32];
             tmem_ld32(t_row + c * 32, v);
             tmem_ld_wait();
-            const int h0 = tl.nb * 256 + c * 32;
+            const int h0 = h_base + c * 32;
             if (tl.which == 0) {
                 float4* dst = reinterpret_cast<float4*>(p.dWd + static_cast<size_t>(j) * p.H + h0);
 #pragma unroll
@@ -671,6 +800,22 @@ struct PairDwPolicy {
                 for (int i = 0; i < 32; ++i) base[static_cast<size_t>(h0 + i) * F_d] = __uint_as_float(v[i]);
             }
         }
+    }
+    __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
+        store_cols(p, tl, cta, row, t_row, tl.nb * 256);
+    }
+    __device__ static __forceinline__ void load_wide(const Params& p, const Tile& tl, int r, int i, uint32_t cta,
+                                                     uint32_t sa, uint32_t sb, uint32_t bar) {
+        const int s0 = r * p.S_loc + i * kBK;
+        const CUtensorMap* ma = tl.which == 0 ? &p.map_a : (tl.which == 1 ? &p.map_dg : &p.map_du);
+        const CUtensorMap* mb = tl.which == 0 ? &p.map_dy : &p.map_x;
+        pair_load_mnmajor(sa, ma, bar, tl.jt * 256 + cta * 128, s0, 0, 2);
+        pair_load_mnmajor(sb, mb, bar, tl.nb * 512 + cta * 128, s0, 0, 2);
+        pair_load_mnmajor(sb + 16384, mb, bar, tl.nb * 512 + 256 + cta * 128, s0, 0, 2);
+    }
+    __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
+                                                         uint32_t t_row, int h) {
+        store_cols(p, tl, cta, row, t_row, tl.nb * 512 + h * 256);
     }
 };
 

@@ -56,6 +56,7 @@ struct tsp_mlp_plan {
     int last_backward_kernels;  // kernels launched by the most recent tsp_mlp_backward (3 or 4)
     int dw_group;               // hidden blocks per group in the dW tile order
     int dx_group;               // token tiles per group in the dX tile order
+    int wide_mask;              // 256 x 512 tiles for: bit 0 down, bit 1 dX, bit 2 dW (env TSP_MLP_WIDE)
     int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
 };
@@ -301,12 +302,39 @@ tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, 
 // ---------------------------------------------------------------------------------------------
 // CTA-pair launches (tile = 256 rows per pair).  Chosen when (S/D) % 256 == 0 (and (F/D) % 256 == 0 for dW).
 // ---------------------------------------------------------------------------------------------
+// 256 x 512 tiles move a quarter less data per FLOP but halve the tile count: take them only when the last round of
+// tiles over the CTA pairs stays about as full as with 256 x 256 tiles (wave quantisation costs more than they gain).
+bool use_wide(const tsp_mlp_plan_t* plan, int bit, int H, int narrow_tiles, int k_blocks) {
+    if (H % 512 != 0) return false;
+    if (plan->wide_mask >= 0) return (plan->wide_mask & bit) != 0;
+    if (k_blocks < 200) return false;   // short K loops cannot amortise the epilogue that no longer overlaps
+    const int pairs = plan->sm_count / 2;
+    auto fill = [pairs](int tiles) {
+        const int rounds = (tiles + pairs - 1) / pairs;
+        return static_cast<double>(tiles) / (static_cast<double>(rounds) * pairs);
+    };
+    return fill(narrow_tiles / 2) >= fill(narrow_tiles) - 0.03;
+}
+
 template <class Params>
 void fill_common(tsp_mlp_plan_t* plan, Params& p, int num_tiles) {
     p.num_tiles = num_tiles;
     p.stages = pick_stages(plan, tsp::kPairStageBytes, plan->pair_stages > 0 ? plan->pair_stages : 6);
     p.status = plan->status_dev;
     p.timeout_ns = plan->timeout_ns;
+}
+
+template <class Kernel, class Params>
+tsp_status_t launch_pair_wide(tsp_mlp_plan_t* plan, Kernel kernel, Params& p, cudaStream_t stream) {
+    p.stages = pick_stages(plan, tsp::kWideStageBytes, 4);
+    const size_t smem = p.stages * tsp::kWideStageBytes + sizeof(tsp::SharedCtl) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    const int pairs_avail = plan->sm_count / 2;
+    const int pairs = p.num_tiles < pairs_avail ? p.num_tiles : pairs_avail;
+    kernel<<<2 * pairs, tsp::kNumThreads, smem, stream>>>(p);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
 
 template <class Kernel, class Params>
@@ -380,6 +408,11 @@ tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* W
     p.tiles_per_rank = static_cast<int>(S / D / 256);
     const int group = plan->group > 0 ? plan->group : 8;
     p.group = p.m_tiles < group ? p.m_tiles : group;
+    if (use_wide(plan, 1, H, p.m_tiles * p.n_blocks, F / 64)) {   // 256 x 512 tiles
+        p.n_blocks = H / 512;
+        fill_common(plan, p, p.m_tiles * p.n_blocks);
+        return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDownPolicy>, p, stream);
+    }
     fill_common(plan, p, p.m_tiles * p.n_blocks);
     return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownPolicy>, p, stream);
 }
@@ -400,6 +433,11 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
     p.tiles_per_rank = static_cast<int>(S / D / 256);
     const int group = plan->dx_group > 0 ? plan->dx_group : 8;
     p.group = p.m_tiles < group ? p.m_tiles : group;
+    if (use_wide(plan, 2, H, p.m_tiles * p.n_blocks, 2 * F / 64)) {
+        p.n_blocks = H / 512;
+        fill_common(plan, p, p.m_tiles * p.n_blocks);
+        return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDxPolicy>, p, stream);
+    }
     fill_common(plan, p, p.m_tiles * p.n_blocks);
     return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDxPolicy>, p, stream);
 }
@@ -424,6 +462,13 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     // hidden blocks are taken in groups whose columns of X / dY (S * 512 bytes per block) fit in about 32 MB of L2
     int n_group = plan->dw_group > 0 ? plan->dw_group : static_cast<int>((32ull << 20) / (512ull * static_cast<size_t>(S)));
     if (n_group < 1) n_group = 1;
+    if (use_wide(plan, 4, H, 3 * p.j_tiles * p.n_blocks, static_cast<int>(S / 64))) {
+        p.n_blocks = H / 512;
+        n_group = (n_group + 1) / 2;
+        p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
+        fill_common(plan, p, 3 * p.j_tiles * p.n_blocks);
+        return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDwPolicy>, p, stream);
+    }
     p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
     fill_common(plan, p, 3 * p.j_tiles * p.n_blocks);
     return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDwPolicy>, p, stream);
@@ -530,6 +575,7 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
     plan->last_backward_kernels = 3;
     plan->phase_mask = env_int("TSP_MLP_PHASES", 3);
+    plan->wide_mask = env_int("TSP_MLP_WIDE", -1);   // -1: decide per launch from the tile counts
     plan->dw_group = env_int("TSP_MLP_DW_GROUP", 0);
     plan->dx_group = env_int("TSP_MLP_DX_GROUP", 0);
     void* fn = nullptr;

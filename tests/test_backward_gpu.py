@@ -54,6 +54,25 @@ def test_multi_tile_shapes_full_compare(S, H, F, D):
     _check_full(S, H, F, D, seed=1)
 
 
+def test_wide_tiles_forced(monkeypatch):
+    # 256 x 512 tiles for the down projection, dX and dW (normally chosen from the tile counts; forced here)
+    monkeypatch.setenv("TSP_MLP_WIDE", "7")
+    S, H, F, D = 1024, 1024, 1024, 2
+    prob = DeviceProblem(S, H, F, D, seed=8, with_dy=True)
+    Y = tensor_to_f64(prob.forward())
+    X, Wg, Wu, Wd, dY = prob.f64()
+    assert rel_fro(Y, orc.gated_mlp_forward(X, Wg, Wu, Wd)) <= TOL_ORACLE
+    got = _grads(prob)
+    ref = orc.gated_mlp_backward(X, Wg, Wu, Wd, dY)
+    for name, g, r in zip(("dX", "dWg", "dWu", "dWd"), got, ref):
+        assert rel_fro(g, r) <= TOL_ORACLE, (name, rel_fro(g, r))
+        assert worst_row_error(g, r) <= TOL_ROW, name
+    monkeypatch.setenv("TSP_MLP_WIDE", "0")
+    narrow = _grads(DeviceProblem(S, H, F, D, host=prob.host, with_dy=True))
+    for g, n in zip(got, narrow):
+        assert rel_fro(g, n) <= 1e-6     # same accumulation order, same bits expected
+
+
 def test_more_tiles_than_sms():
     _check_full(20480, 256, 512, 4, seed=2)
 
