@@ -66,6 +66,18 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out);
 tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan);
 
 /*
+ * tsp_mlp_set_activation - choose the gate activation sigma of Algorithm 2 ("Activation sigma"; the paper
+ * names SwiGLU as the example of a gated MLP).  TSP_ACT_SILU (default): sigma(z) = z / (1 + e^-z);
+ * TSP_ACT_GELU: sigma(z) = z * Phi(z), Phi the standard normal CDF (erf form, not the tanh approximation);
+ * TSP_ACT_RELU: sigma(z) = max(z, 0), with sigma'(0) = 0 in the backward pass.  Applies to every later
+ * forward / backward / staged call on the plan.  Error: INVALID_ARG for any other value.
+ */
+#define TSP_ACT_SILU 0
+#define TSP_ACT_GELU 1
+#define TSP_ACT_RELU 2
+tsp_status_t tsp_mlp_set_activation(tsp_mlp_plan_t* plan, int activation);
+
+/*
  * Workspace: scratch for the bf16 intermediate A = silu(G)*U [S,F] (forward) and for
  * A, dG, dU [S,F] in bf16 plus dA [S,F] in fp32 (backward).  tsp_mlp_workspace_bytes returns the size needed
  * for S tokens (`pass` = TSP_WS_FORWARD or TSP_WS_BACKWARD; backward covers forward);

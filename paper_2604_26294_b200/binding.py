@@ -19,6 +19,9 @@ TSP_ERR_WORKSPACE = -5
 TSP_ERR_DEVICE_TIMEOUT = -6
 TSP_ERR_STATIC_LIMIT = -7
 TSP_MLP_STATIC_SCRATCH_BYTES = 8 << 20
+TSP_ACT_SILU = 0
+TSP_ACT_GELU = 1
+TSP_ACT_RELU = 2
 TSP_WS_FORWARD = 0
 TSP_WS_BACKWARD = 1
 
@@ -29,6 +32,7 @@ _P = ctypes.c_void_p
 SIGNATURES = {
     "tsp_mlp_plan": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(_P)]),
     "tsp_mlp_plan_destroy": (ctypes.c_int, [_P]),
+    "tsp_mlp_set_activation": (ctypes.c_int, [_P, ctypes.c_int]),
     "tsp_mlp_workspace_bytes": (ctypes.c_size_t, [_P, ctypes.c_int64, ctypes.c_int]),
     "tsp_mlp_workspace_bytes_host": (ctypes.c_size_t, [_P, ctypes.c_int64]),
     "tsp_mlp_set_workspace": (ctypes.c_int, [_P, _P, ctypes.c_size_t]),
@@ -125,6 +129,11 @@ def tsp_mlp_plan(H: int, F: int, D: int):
 
 def tsp_mlp_plan_destroy(plan) -> None:
     _check(load_library().tsp_mlp_plan_destroy(plan), "tsp_mlp_plan_destroy")
+
+
+def tsp_mlp_set_activation(plan, activation: int) -> None:
+    """Gate activation: TSP_ACT_SILU (default), TSP_ACT_GELU (erf form) or TSP_ACT_RELU."""
+    _check(load_library().tsp_mlp_set_activation(plan, activation), "tsp_mlp_set_activation")
 
 
 def tsp_mlp_workspace_bytes(plan, S: int, backward: int = TSP_WS_FORWARD) -> int:

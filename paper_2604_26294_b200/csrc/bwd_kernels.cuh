@@ -38,6 +38,7 @@ struct BwdGateParams {
     __nv_bfloat16* dU;    // [S, F]
     int S, H, F, D;
     int m_blocks, blocks_per_rank, jl_blocks, band, num_tiles, stages;
+    int act;              // gate activation
     int* status;
     unsigned long long timeout_ns;
 };
@@ -170,11 +171,11 @@ __global__ void __launch_bounds__(kNumThreads, 1) bwd_gate_kernel(const __grid_c
                         const float gg = __uint_as_float(g[2 * i + e]);
                         const float uu = __uint_as_float(u[2 * i + e]);
                         const float dd = __uint_as_float(da[2 * i + e]);
-                        const float s = sigmoid_fast(gg);
-                        const float sg = gg * s;                       // silu(G)
+                        float sg, ds;
+                        gate_act_grad(gg, p.act, sg, ds);              // sigma(G), sigma'(G)
                         va[e] = sg * uu;                               // A
-                        vu[e] = dd * sg;                               // dU = dA * silu(G)
-                        vg[e] = dd * uu * (s * (1.0f + gg * (1.0f - s)));  // dG = dA * U * silu'(G)
+                        vu[e] = dd * sg;                               // dU = dA * sigma(G)
+                        vg[e] = dd * uu * ds;                          // dG = dA * U * sigma'(G)
                     }
                     pa[i] = pack_bf16x2(va[0], va[1]);
                     pg[i] = pack_bf16x2(vg[0], vg[1]);

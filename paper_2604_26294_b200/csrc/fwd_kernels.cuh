@@ -27,6 +27,7 @@ struct GateUpParams {
     int jl_blocks;       // (F/D) / 128
     int band;            // token blocks per band (their X rows stay L2-resident while the shards stream)
     int shared_order;    // 0: ranks of a band follow the ring (different shards at a time); 1: same column block for all
+    int act;             // gate activation (kActSilu / kActGelu / kActRelu)
     int num_tiles;
     int stages;
     int* status;
@@ -137,8 +138,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) gate_up_swiglu_kernel(const __
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-                    const float a0 = g0 * sigmoid_fast(g0) * __uint_as_float(u[2 * i]);
-                    const float a1 = g1 * sigmoid_fast(g1) * __uint_as_float(u[2 * i + 1]);
+                    const float a0 = gate_act(g0, p.act) * __uint_as_float(u[2 * i]);
+                    const float a1 = gate_act(g1, p.act) * __uint_as_float(u[2 * i + 1]);
                     packed[i] = pack_bf16x2(a0, a1);
                 }
                 uint4* dst = reinterpret_cast<uint4*>(out + c * 32);

@@ -182,4 +182,29 @@ __device__ __forceinline__ float sigmoid_fast(float z) {
     return __fdividef(1.0f, 1.0f + __expf(fminf(-z, 80.0f)));
 }
 
+// Gate activations sigma of Algorithm 2 ("Activation sigma"): 0 = SiLU (SwiGLU), 1 = GELU, exact erf form (GeGLU),
+// 2 = ReLU (ReGLU).  `act` is uniform over the launch, so the branch does not diverge.
+constexpr int kActSilu = 0, kActGelu = 1, kActRelu = 2;
+
+__device__ __forceinline__ float gate_act(float z, int act) {
+    if (act == kActSilu) return z * sigmoid_fast(z);
+    if (act == kActGelu) return 0.5f * z * (1.0f + erff(z * 0.70710678118654752f));
+    return fmaxf(z, 0.0f);
+}
+// value and derivative of the activation
+__device__ __forceinline__ void gate_act_grad(float z, int act, float& val, float& der) {
+    if (act == kActSilu) {
+        const float s = sigmoid_fast(z);
+        val = z * s;
+        der = s * (1.0f + z * (1.0f - s));
+    } else if (act == kActGelu) {
+        const float cdf = 0.5f * (1.0f + erff(z * 0.70710678118654752f));
+        val = z * cdf;
+        der = cdf + z * 0.3989422804014327f * __expf(-0.5f * z * z);
+    } else {
+        val = fmaxf(z, 0.0f);
+        der = z > 0.0f ? 1.0f : 0.0f;
+    }
+}
+
 }  // namespace tsp

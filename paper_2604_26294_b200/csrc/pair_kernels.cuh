@@ -358,6 +358,7 @@ struct PairGateUpPolicyT {
         __nv_bfloat16* dU;    // [S, F] (backward only)
         int S, H, F, D, F_d;
         int m_tiles, tiles_per_rank, jl_blocks, band, shared_order;
+        int act;              // gate activation
         int rank_indexed;     // staged mode: one ring step per launch; the weight tensors hold, at index r, the
                               // shard rank r currently has in its receive buffer, and A is [S, F/D]
         int num_tiles, stages;
@@ -413,8 +414,8 @@ struct PairGateUpPolicyT {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-                    packed[i] = pack_bf16x2(g0 * sigmoid_fast(g0) * __uint_as_float(u[2 * i]),
-                                            g1 * sigmoid_fast(g1) * __uint_as_float(u[2 * i + 1]));
+                    packed[i] = pack_bf16x2(gate_act(g0, p.act) * __uint_as_float(u[2 * i]),
+                                            gate_act(g1, p.act) * __uint_as_float(u[2 * i + 1]));
                 }
                 uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
 #pragma unroll
@@ -442,11 +443,11 @@ struct PairGateUpPolicyT {
                         const float gg = __uint_as_float(g[2 * i + e]);
                         const float uu = __uint_as_float(u[2 * i + e]);
                         const float dd = da[2 * i + e];
-                        const float sgm = sigmoid_fast(gg);
-                        const float sg = gg * sgm;                          // silu(G)
+                        float sg, ds;
+                        gate_act_grad(gg, p.act, sg, ds);                   // sigma(G), sigma'(G)
                         va[e] = sg * uu;                                    // A
-                        vu[e] = dd * sg;                                    // dU = dA * silu(G)
-                        vg[e] = dd * uu * (sgm * (1.0f + gg * (1.0f - sgm)));  // dG = dA * U * silu'(G)
+                        vu[e] = dd * sg;                                    // dU = dA * sigma(G)
+                        vg[e] = dd * uu * ds;                               // dG = dA * U * sigma'(G)
                     }
                     pa[i] = pack_bf16x2(va[0], va[1]);
                     pg[i] = pack_bf16x2(vg[0], vg[1]);
@@ -556,7 +557,9 @@ struct PairDownPolicy {
         const int rem = tile - g * per_group;
         Tile o;
         o.nb = rem / g_sz;
-        o.mt = g_start + rem % g_sz;
+        // token tiles are taken from the last to the first: the producer kernel wrote the last rows most recently,
+        // so they are the ones still in L2
+        o.mt = p.m_tiles - 1 - (g_start + rem % g_sz);
         o.r = o.mt / p.tiles_per_rank;
         return o;
     }
@@ -614,7 +617,9 @@ struct PairDownStagedPolicy {
         const int rem = tile - g * per_group;
         Tile o;
         o.nb = rem / g_sz;
-        o.mt = g_start + rem % g_sz;
+        // token tiles are taken from the last to the first: the producer kernel wrote the last rows most recently,
+        // so they are the ones still in L2
+        o.mt = p.m_tiles - 1 - (g_start + rem % g_sz);
         o.r = o.mt / p.tiles_per_rank;
         return o;
     }
@@ -692,7 +697,9 @@ struct PairDxPolicy {
         const int rem = tile - g * per_group;
         Tile o;
         o.nb = rem / g_sz;
-        o.mt = g_start + rem % g_sz;
+        // token tiles are taken from the last to the first: the producer kernel wrote the last rows most recently,
+        // so they are the ones still in L2
+        o.mt = p.m_tiles - 1 - (g_start + rem % g_sz);
         o.r = o.mt / p.tiles_per_rank;
         return o;
     }

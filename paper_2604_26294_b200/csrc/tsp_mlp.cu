@@ -56,6 +56,7 @@ struct tsp_mlp_plan {
     int last_backward_kernels;  // kernels launched by the most recent tsp_mlp_backward (3 or 4)
     int dw_group;               // hidden blocks per group in the dW tile order
     int dx_group;               // token tiles per group in the dX tile order
+    int act;                    // gate activation (TSP_ACT_*)
     int wide_mask;              // 256 x 512 tiles for: bit 0 down, bit 1 dX, bit 2 dW (env TSP_MLP_WIDE)
     int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
@@ -168,6 +169,7 @@ tsp_status_t launch_gate_up(tsp_mlp_plan_t* plan, const void* X, const void* Wg,
     p.band = 2 * gate_band(plan, (p.m_blocks + 1) / 2);   // same band, counted in 128-token blocks
     if (p.band > p.m_blocks) p.band = p.m_blocks;
     p.shared_order = plan->shared_order;
+    p.act = plan->act;
     p.num_tiles = p.m_blocks * D * p.jl_blocks;
     p.stages = pick_stages(plan, 48 * 1024, 4);
     p.status = plan->status_dev;
@@ -227,6 +229,7 @@ tsp_status_t launch_bwd_gate(tsp_mlp_plan_t* plan, const void* X, const void* Wg
     p.jl_blocks = F_d / 128;
     p.band = 2 * gate_band(plan, (p.m_blocks + 1) / 2);
     if (p.band > p.m_blocks) p.band = p.m_blocks;
+    p.act = plan->act;
     p.num_tiles = p.m_blocks * D * p.jl_blocks;
     p.stages = pick_stages(plan, 48 * 1024, 4);
     p.status = plan->status_dev;
@@ -370,6 +373,7 @@ tsp_status_t launch_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* W
     p.jl_blocks = F_d / 128;
     p.band = gate_band(plan, p.m_tiles);
     p.shared_order = plan->shared_order;
+    p.act = plan->act;
     fill_common(plan, p, p.m_tiles * D * p.jl_blocks);
     return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
 }
@@ -575,6 +579,7 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
     plan->last_backward_kernels = 3;
     plan->phase_mask = env_int("TSP_MLP_PHASES", 3);
+    plan->act = TSP_ACT_SILU;
     plan->wide_mask = env_int("TSP_MLP_WIDE", -1);   // -1: decide per launch from the tile counts
     plan->dw_group = env_int("TSP_MLP_DW_GROUP", 0);
     plan->dx_group = env_int("TSP_MLP_DX_GROUP", 0);
@@ -625,6 +630,13 @@ tsp_status_t tsp_mlp_set_workspace(tsp_mlp_plan_t* plan, void* dev_ptr, size_t b
     if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return TSP_ERR_INVALID_ARG;
     plan->workspace = dev_ptr;
     plan->workspace_bytes = dev_ptr ? bytes : 0;
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_set_activation(tsp_mlp_plan_t* plan, int activation) {
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    if (activation != TSP_ACT_SILU && activation != TSP_ACT_GELU && activation != TSP_ACT_RELU) return TSP_ERR_INVALID_ARG;
+    plan->act = activation;
     return TSP_OK;
 }
 
@@ -773,6 +785,7 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
             p.jl_blocks = F_d / 128;
             p.band = gate_band(plan, p.m_tiles);
             p.rank_indexed = 1;
+            p.act = plan->act;
             fill_common(plan, p, p.m_tiles * p.jl_blocks);
             st = launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, cs);
             if (st != TSP_OK) return st;

@@ -44,7 +44,7 @@ class DeviceProblem:
         self.dY = bf16_tensor(h.dY) if h.dY is not None else None
         self.Y = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
 
-    def forward(self):
+    def forward(self, act=None):
         """Run tsp_mlp_forward through the binding; returns Y (torch bf16 on the GPU)."""
         import torch
 
@@ -52,6 +52,8 @@ class DeviceProblem:
 
         plan = b.tsp_mlp_plan(self.H, self.F, self.D)
         try:
+            if act is not None:
+                b.tsp_mlp_set_activation(plan, act)
             ws = torch.empty(b.tsp_mlp_workspace_bytes(plan, self.S, b.TSP_WS_FORWARD), dtype=torch.uint8, device="cuda")
             b.tsp_mlp_set_workspace(plan, ws)
             self.Y.fill_(float("nan"))
@@ -63,7 +65,7 @@ class DeviceProblem:
             b.tsp_mlp_plan_destroy(plan)
         return self.Y
 
-    def backward(self):
+    def backward(self, act=None):
         """Run tsp_mlp_backward; returns dX (bf16), dWg, dWu, dWd (fp32) torch tensors."""
         import torch
 
@@ -72,6 +74,8 @@ class DeviceProblem:
         S, H, F, D = self.S, self.H, self.F, self.D
         plan = b.tsp_mlp_plan(H, F, D)
         try:
+            if act is not None:
+                b.tsp_mlp_set_activation(plan, act)
             ws = torch.empty(b.tsp_mlp_workspace_bytes(plan, S, b.TSP_WS_BACKWARD), dtype=torch.uint8, device="cuda")
             b.tsp_mlp_set_workspace(plan, ws)
             dX = torch.full((S, H), float("nan"), dtype=torch.bfloat16, device="cuda")

@@ -1,0 +1,49 @@
+"""The gate activation sigma of Algorithm 2 as a plan parameter: SiLU (default), GELU, ReLU."""
+import numpy as np
+import pytest
+
+from oracle import tsp_mlp_oracle as orc
+from paper_2604_26294_b200 import binding as b
+from paper_2604_26294_b200 import build
+from paper_2604_26294_b200 import inputs as inp
+from tests.helpers import DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
+
+pytestmark = pytest.mark.gpu
+
+TOL_ORACLE = 1e-2
+ACTS = {"silu": b.TSP_ACT_SILU, "gelu": b.TSP_ACT_GELU, "relu": b.TSP_ACT_RELU}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build_library()
+
+
+@pytest.mark.parametrize("name", ["gelu", "relu", "silu"])
+@pytest.mark.parametrize("S,H,F,D", [(256, 256, 768, 2), (1536, 768, 1280, 2)])   # single-CTA path, CTA-pair path
+def test_forward_and_backward_match_oracle(name, S, H, F, D):
+    prob = DeviceProblem(S, H, F, D, seed=31, with_dy=True)
+    X, Wg, Wu, Wd, dY = prob.f64()
+    Y = tensor_to_f64(prob.forward(ACTS[name]))
+    ref = orc.gated_mlp_forward(X, Wg, Wu, Wd, name)
+    assert rel_fro(Y, ref) <= TOL_ORACLE, rel_fro(Y, ref)
+    assert worst_row_error(Y, ref) <= 0.08
+    dX, dWg, dWu, dWd = prob.backward(ACTS[name])
+    got = (tensor_to_f64(dX), inp.unshard_columns(tensor_to_f64(dWg)), inp.unshard_columns(tensor_to_f64(dWu)),
+           inp.unshard_rows(tensor_to_f64(dWd)))
+    refs = orc.gated_mlp_backward(X, Wg, Wu, Wd, dY, name)
+    for n, g, r in zip(("dX", "dWg", "dWu", "dWd"), got, refs):
+        assert rel_fro(g, r) <= TOL_ORACLE, (name, n, rel_fro(g, r))
+
+
+def test_activations_differ_and_bad_value_is_refused():
+    prob = DeviceProblem(256, 256, 768, 2, seed=32)
+    ys = {n: tensor_to_f64(prob.forward(a)).copy() for n, a in ACTS.items()}
+    assert rel_fro(ys["gelu"], ys["silu"]) > 0.05 and rel_fro(ys["relu"], ys["silu"]) > 0.05
+    plan = b.tsp_mlp_plan(256, 768, 2)
+    try:
+        with pytest.raises(b.TspError) as err:
+            b.tsp_mlp_set_activation(plan, 7)
+        assert err.value.code == b.TSP_ERR_INVALID_ARG
+    finally:
+        b.tsp_mlp_plan_destroy(plan)

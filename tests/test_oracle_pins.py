@@ -269,3 +269,90 @@ def test_output_scale_under_benchmark_distribution():
     Y = orc.gated_mlp_forward(X, Wg, Wu, Wd)
     assert abs(Y.std() - math.sqrt(second_moment)) < 0.03
     assert abs(math.sqrt(second_moment) - 0.596) < 2e-3
+
+
+# ---------------------------------------------------------------------------------------
+# other gate activations (Algorithm 2 takes a generic "Activation sigma")
+# ---------------------------------------------------------------------------------------
+def _brute_forward_act(X, Wg, Wu, Wd, act):
+    def sigma(g):
+        if act == "gelu":
+            return g * 0.5 * (1.0 + math.erf(g / math.sqrt(2.0)))
+        if act == "relu":
+            return g if g > 0 else 0.0
+        return g * _sig(g)
+    S, H, F = len(X), len(X[0]), len(Wd)
+    Y = [[0.0] * H for _ in range(S)]
+    for s in range(S):
+        a = []
+        for j in range(F):
+            g = math.fsum(X[s][h] * Wg[h][j] for h in range(H))
+            u = math.fsum(X[s][h] * Wu[h][j] for h in range(H))
+            a.append(sigma(g) * u)
+        for h in range(H):
+            Y[s][h] = math.fsum(a[j] * Wd[j][h] for j in range(F))
+    return Y
+
+
+@pytest.mark.parametrize("act", ["silu", "gelu", "relu"])
+def test_forward_brute_force_every_activation(act):
+    S, H, F = 5, 6, 7
+    X, Wg, Wu, Wd = _rand(S, H), _rand(H, F) / 2, _rand(H, F) / 2, _rand(F, H)
+    Y = orc.gated_mlp_forward(X, Wg, Wu, Wd, act)
+    Yb = np.array(_brute_forward_act(X.tolist(), Wg.tolist(), Wu.tolist(), Wd.tolist(), act))
+    np.testing.assert_allclose(Y, Yb, rtol=1e-12, atol=1e-13)
+
+
+def test_gelu_golden_values_and_identities(golden_dir):
+    with open(os.path.join(golden_dir, "gelu_closed_forms.txt")) as f:
+        rows = [[float(v) for v in ln.split()] for ln in f if ln.strip() and not ln.startswith("#")]
+    assert len(rows) >= 5
+    for z, g, gp in rows:
+        assert abs(float(orc.gelu(np.array([z]))[0]) - g) < 1e-13
+        assert abs(float(orc.gelu_prime(np.array([z]))[0]) - gp) < 1e-13
+    z = np.linspace(-8, 8, 161)
+    np.testing.assert_allclose(orc.gelu(-z), orc.gelu(z) - z, atol=1e-13)
+    np.testing.assert_allclose(orc.gelu_prime(-z), 1.0 - orc.gelu_prime(z), atol=1e-13)
+    e = 1e-6
+    np.testing.assert_allclose(orc.gelu_prime(z), (orc.gelu(z + e) - orc.gelu(z - e)) / (2 * e), atol=1e-8)
+
+
+def test_relu_values():
+    z = np.array([-2.0, -0.0, 0.0, 0.5, 3.0])
+    assert np.array_equal(orc.relu(z), np.array([0.0, 0.0, 0.0, 0.5, 3.0]))
+    assert np.array_equal(orc.relu_prime(z), np.array([0.0, 0.0, 0.0, 1.0, 1.0]))
+
+
+@pytest.mark.parametrize("act", ["gelu", "relu"])
+def test_gradients_finite_differences_other_activations(act):
+    S, H, F = 6, 5, 7
+    X, Wg, Wu, Wd, dY = _rand(S, H), _rand(H, F) / 2, _rand(H, F) / 2, _rand(F, H) / 2, _rand(S, H)
+    grads = orc.gated_mlp_backward(X, Wg, Wu, Wd, dY, act)
+    params = [X, Wg, Wu, Wd]
+    # relu is piecewise linear: keep the step far below the distance of any pre-activation to the kink
+    eps = 1e-7 if act == "relu" else 1e-5
+    assert act != "relu" or np.min(np.abs(X @ Wg)) > 1e-4
+    for which in range(4):
+        V = _rand(*params[which].shape)
+        plus = [q.copy() for q in params]
+        minus = [q.copy() for q in params]
+        plus[which] = plus[which] + eps * V
+        minus[which] = minus[which] - eps * V
+        fd = (float(np.sum(dY * orc.gated_mlp_forward(*plus, act))) -
+              float(np.sum(dY * orc.gated_mlp_forward(*minus, act)))) / (2 * eps)
+        an = float(np.sum(grads[which] * V))
+        assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (act, which, fd, an)
+
+
+@pytest.mark.parametrize("act", ["gelu", "relu"])
+@pytest.mark.parametrize("D", [2, 4])
+def test_ring_equals_unsharded_other_activations(act, D):
+    S, H, F = 16, 6, 24
+    X, Wg, Wu, Wd, dY = _rand(S, H), _rand(H, F) / 2, _rand(H, F) / 2, _rand(F, H) / 4, _rand(S, H)
+    Yr, _ = orc.ring_gated_mlp_forward(*_split(X, Wg, Wu, Wd, D), act)
+    np.testing.assert_allclose(np.concatenate(Yr, 0), orc.gated_mlp_forward(X, Wg, Wu, Wd, act), rtol=1e-12, atol=1e-12)
+    dX, dWg, dWu, dWd = orc.gated_mlp_backward(X, Wg, Wu, Wd, dY, act)
+    rX, rWg, rWu, rWd = orc.ring_gated_mlp_backward(*_split(X, Wg, Wu, Wd, D, dY), act)
+    np.testing.assert_allclose(np.concatenate(rX, 0), dX, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(np.concatenate(rWg, 1), dWg, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(np.concatenate(rWd, 0), dWd, rtol=1e-11, atol=1e-12)
