@@ -30,13 +30,14 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Test the phase with `parity`; while it is incomplete the thread may be suspended by the hardware for up to
+// Test the phase with `parity` (acquire at cluster scope: in the CTA-pair kernels the arrivals come from the peer
+// CTA; for a kernel launched without clusters the scope degenerates to the CTA); while it is incomplete the thread may be suspended by the hardware for up to
 // `suspend_hint_ns` (it is woken when the phase completes), which keeps waiting warps off the issue ports.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t suspend_hint_ns = 20000u) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity), "r"(suspend_hint_ns)
