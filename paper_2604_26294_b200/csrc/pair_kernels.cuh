@@ -225,16 +225,31 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Wide pair kernel for the long-K GEMMs: tile = 256 rows x 512 columns, ONE accumulator set that fills all 512
-// tensor-memory columns.  Per k-block each CTA loads 128 rows of A once (16 KB) and two half-B blocks (2 x 16 KB);
-// the leader issues two N = 256 MMAs per k-step that share the A descriptor.  Compared with the 256 x 256 tile this
-// moves 48 KB instead of 64 KB per CTA pair and tile-k-block from L2, and a wave of 74 pairs spans twice the columns,
-// which halves the DRAM re-reads of the row operand.  The price: the epilogue no longer overlaps the next main
-// loop (the two column halves are released separately, so the first half of the next tile starts early); worth it
-// when K is long (down projection, dX, dW).
-// Policy additionally provides load_wide(p, tile, sel, i, cta, sa, sb, bar) and epilogue_half(p, tile, cta, row, t_row, h).
+// Mixed-width pair kernel for the long-K GEMMs.  A tile is 256 rows x 512 columns ("wide": ONE accumulator set that
+// fills all 512 tensor-memory columns) or 256 x 256 ("narrow": the first 256 columns only).  Per k-block each CTA
+// loads 128 rows of A once (16 KB) and one 16 KB half-B block per 256 columns; the leader issues one N = 256 MMA per
+// column half, sharing the A descriptor.  A wide tile moves 48 KB instead of 64 KB per CTA pair and 256x256-tile-
+// k-block from L2, and a round of 74 wide tiles spans twice the columns, which halves the DRAM re-reads of the row
+// operand.  The price: the epilogue no longer overlaps the next main loop (the two column halves are released
+// separately, so the first half of the next tile starts early); worth it when K is long.
+// The tile list holds `wide_tiles` wide tiles first, then narrow ones that fill the last round, so the 74 pairs
+// finish together (e.g. 512 narrow tiles = 3 rounds of wide tiles + 68 narrow tiles).  Tiles are numbered row-major
+// over (row tile, 256-column block); a wide tile covers two neighbouring column blocks.
+// Policy provides Tile decode_mixed(p, list_index) with Tile::halves and Tile::nb in 256-column units,
+// load_wide(p, tile, sel, i, cta, sa, sb, bar) and epilogue_half(p, tile, cta, row, t_row, h).
 // ------------------------------------------------------------------------------------------------
 constexpr uint32_t kWideStageBytes = 48 * 1024;
+
+// list index -> (row tile, first 256-column block, halves); rows are taken from the last to the first when `reverse`
+__device__ __forceinline__ void mixed_tile(int t, int wide_tiles, int n_blocks, int rows, bool reverse, int& row, int& nb,
+                                           int& halves) {
+    const bool wide = t < wide_tiles;
+    const int flat = wide ? 2 * t : 2 * wide_tiles + (t - wide_tiles);
+    row = flat / n_blocks;
+    nb = flat - row * n_blocks;
+    if (reverse) row = rows - 1 - row;
+    halves = wide ? 2 : 1;
+}
 
 template <class Policy>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
@@ -259,14 +274,15 @@ pair_wide_kernel(const __grid_constant__ typename Policy::Params p) {
             PipeState ps;
             bool ok = true;
             for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs) {
-                const typename Policy::Tile tl = Policy::decode(p, tile);
+                const typename Policy::Tile tl = Policy::decode_mixed(p, tile);
+                const uint32_t bytes = 2u * (kPairABytes + static_cast<uint32_t>(tl.halves) * 16384u);
                 for (int o = 0; o < n_outer && ok; ++o) {
                     const int sel = Policy::select(p, tl, o);
                     for (int i = 0; i < n_inner; ++i) {
                         if (!(ok = wait_bar(smem_u32(&ctl->empty[ps.stage]), ps.phase ^ 1u, w, kErrWaitEmpty))) break;
                         const uint32_t bar = map_to_cta(smem_u32(&ctl->full[ps.stage]), 0);
                         const uint32_t sa = smem_base + ps.stage * kWideStageBytes, sb = sa + kPairABytes;
-                        if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), 2 * kWideStageBytes);
+                        if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), bytes);
                         Policy::load_wide(p, tl, sel, i, cta, sa, sb, bar);
                         ps.advance(p.stages);
                     }
@@ -278,17 +294,18 @@ pair_wide_kernel(const __grid_constant__ typename Policy::Params p) {
             constexpr uint32_t idesc = make_idesc_bf16(256, 256, Policy::kAMn, Policy::kBMn);
             PipeState ps;
             bool ok = true;
-            int it = 0;
-            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
+            uint32_t uses[2] = {0u, 0u};   // how often each column half has been filled so far
+            for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs) {
+                const int halves = tile < p.wide_tiles ? 2 : 1;
                 for (int kb = 0; kb < k_blocks && ok; ++kb) {
                     if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
                     tc_fence_after_sync();
                     const uint32_t sa = smem_base + ps.stage * kWideStageBytes, sb = sa + kPairABytes;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (kb == 0) {  // the previous tile's epilogue must have drained this half
-                            if (!(ok = wait_bar(smem_u32(&ctl->tmem_empty[h]), (it & 1) ^ 1u, w, kErrWaitTmemEmpty))) break;
+                    for (int h = 0; h < halves; ++h) {
+                        if (kb == 0) {  // the previous user's epilogue must have drained this half
+                            if (!(ok = wait_bar(smem_u32(&ctl->tmem_empty[h]), (uses[h] & 1u) ^ 1u, w, kErrWaitTmemEmpty))) break;
                             tc_fence_after_sync();
+                            ++uses[h];
                         }
                         pair_issue_kblock<Policy::kAMn, Policy::kBMn>(tmem_base + h * 256, sa, sb + h * 16384, idesc, kb > 0);
                     }
@@ -311,12 +328,12 @@ pair_wide_kernel(const __grid_constant__ typename Policy::Params p) {
         bool ok = true;
         int it = 0;
         for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs, ++it) {
-            const typename Policy::Tile tl = Policy::decode(p, tile);
+            const typename Policy::Tile tl = Policy::decode_mixed(p, tile);
             if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[0]), it & 1, w, kErrWaitTmemFull))) break;
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
 #pragma unroll 1
-            for (int h = 0; h < 2; ++h) {
+            for (int h = 0; h < tl.halves; ++h) {
                 Policy::epilogue_half(p, tl, cta, row, t_row + h * 256, h);
                 tc_fence_before_sync();
                 mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[h]), 0));
@@ -531,12 +548,13 @@ struct PairDownPolicy {
         __nv_bfloat16* Y;
         int S, H, F, D, F_d;
         int m_tiles, n_blocks, tiles_per_rank, group;
+        int wide_tiles;   // mixed-width kernel: number of 256 x 512 tiles at the head of the tile list
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
     };
     struct Tile {
-        int mt, nb, r;
+        int mt, nb, r, halves;
     };
     __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
     __device__ static __forceinline__ int inner(const Params& p) { return p.F_d / kBK; }
@@ -572,17 +590,23 @@ struct PairDownPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
     }
-    // wide tile: tl.nb counts 512-column blocks
+    // mixed-width kernel: tl.nb is the first 256-column block, tl.halves the number of column blocks
+    __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
+        Tile o;
+        mixed_tile(t, p.wide_tiles, p.n_blocks, p.m_tiles, true, o.mt, o.nb, o.halves);
+        o.r = o.mt / p.tiles_per_rank;
+        return o;
+    }
     __device__ static __forceinline__ void load_wide(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
                                                      uint32_t sa, uint32_t sb, uint32_t bar) {
         const int f0 = k * p.F_d + i * kBK;
         pair_load_kmajor(sa, &p.map_a, bar, f0, tl.mt * 256 + cta * 128, 0);
-        pair_load_mnmajor(sb, &p.map_wd, bar, tl.nb * 512 + cta * 128, f0, 0, 2);
-        pair_load_mnmajor(sb + 16384, &p.map_wd, bar, tl.nb * 512 + 256 + cta * 128, f0, 0, 2);
+        for (int h = 0; h < tl.halves; ++h)
+            pair_load_mnmajor(sb + h * 16384, &p.map_wd, bar, (tl.nb + h) * 256 + cta * 128, f0, 0, 2);
     }
     __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
                                                          uint32_t t_row, int h) {
-        store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 512 + h * 256, t_row);
+        store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + (tl.nb + h) * 256, t_row);
     }
 };
 
@@ -672,6 +696,7 @@ struct PairDxPolicy {
         __nv_bfloat16* dX;
         int S, H, F, D, F_d;
         int m_tiles, n_blocks, tiles_per_rank, group;
+        int wide_tiles;
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -713,18 +738,23 @@ struct PairDxPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_bf16_row256(p.dX + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
     }
+    __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
+        Tile o;
+        mixed_tile(t, p.wide_tiles, p.n_blocks, p.m_tiles, true, o.mt, o.nb, o.halves);
+        o.r = o.mt / p.tiles_per_rank;
+        return o;
+    }
     __device__ static __forceinline__ void load_wide(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
                                                      uint32_t sa, uint32_t sb, uint32_t bar) {
         const int j0 = (i >> 1) * kBK;
         const bool up = i & 1;
         const CUtensorMap* mw = up ? &p.map_wu : &p.map_wg;
         pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.mt * 256 + cta * 128, 0);
-        pair_load_kmajor(sb, mw, bar, j0, tl.nb * 512 + cta * 128, k);
-        pair_load_kmajor(sb + 16384, mw, bar, j0, tl.nb * 512 + 256 + cta * 128, k);
+        for (int h = 0; h < tl.halves; ++h) pair_load_kmajor(sb + h * 16384, mw, bar, j0, (tl.nb + h) * 256 + cta * 128, k);
     }
     __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
                                                          uint32_t t_row, int h) {
-        store_bf16_row256(p.dX + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 512 + h * 256, t_row);
+        store_bf16_row256(p.dX + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + (tl.nb + h) * 256, t_row);
     }
 };
 
@@ -739,12 +769,13 @@ struct PairDwPolicy {
         int S, H, F, D, F_d, S_loc;
         int j_tiles, n_blocks, j_tiles_per_shard;
         int n_group;   // hidden blocks per group: their columns of X / dY stay in L2 while the [S,F] operand streams
+        int wide_tiles;
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
     };
     struct Tile {
-        int which, jt, nb, k;
+        int which, jt, nb, k, halves;
     };
     __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
     __device__ static __forceinline__ int inner(const Params& p) { return p.S_loc / kBK; }
@@ -811,18 +842,27 @@ struct PairDwPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_cols(p, tl, cta, row, t_row, tl.nb * 256);
     }
+    // mixed-width kernel: rows of the tile grid are (family, intermediate tile)
+    __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
+        Tile o;
+        int row;
+        mixed_tile(t, p.wide_tiles, p.n_blocks, 3 * p.j_tiles, false, row, o.nb, o.halves);
+        o.which = row / p.j_tiles;
+        o.jt = row - o.which * p.j_tiles;
+        o.k = o.jt / p.j_tiles_per_shard;
+        return o;
+    }
     __device__ static __forceinline__ void load_wide(const Params& p, const Tile& tl, int r, int i, uint32_t cta,
                                                      uint32_t sa, uint32_t sb, uint32_t bar) {
         const int s0 = r * p.S_loc + i * kBK;
         const CUtensorMap* ma = tl.which == 0 ? &p.map_a : (tl.which == 1 ? &p.map_dg : &p.map_du);
         const CUtensorMap* mb = tl.which == 0 ? &p.map_dy : &p.map_x;
         pair_load_mnmajor(sa, ma, bar, tl.jt * 256 + cta * 128, s0, 0, 2);
-        pair_load_mnmajor(sb, mb, bar, tl.nb * 512 + cta * 128, s0, 0, 2);
-        pair_load_mnmajor(sb + 16384, mb, bar, tl.nb * 512 + 256 + cta * 128, s0, 0, 2);
+        for (int h = 0; h < tl.halves; ++h) pair_load_mnmajor(sb + h * 16384, mb, bar, (tl.nb + h) * 256 + cta * 128, s0, 0, 2);
     }
     __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
                                                          uint32_t t_row, int h) {
-        store_cols(p, tl, cta, row, t_row, tl.nb * 512 + h * 256);
+        store_cols(p, tl, cta, row, t_row, (tl.nb + h) * 256);
     }
 };
 

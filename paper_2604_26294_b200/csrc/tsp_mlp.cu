@@ -305,18 +305,24 @@ tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, 
 // ---------------------------------------------------------------------------------------------
 // CTA-pair launches (tile = 256 rows per pair).  Chosen when (S/D) % 256 == 0 (and (F/D) % 256 == 0 for dW).
 // ---------------------------------------------------------------------------------------------
-// 256 x 512 tiles move a quarter less data per FLOP but halve the tile count: take them only when the last round of
-// tiles over the CTA pairs stays about as full as with 256 x 256 tiles (wave quantisation costs more than they gain).
-bool use_wide(const tsp_mlp_plan_t* plan, int bit, int H, int narrow_tiles, int k_blocks) {
-    if (H % 512 != 0) return false;
-    if (plan->wide_mask >= 0) return (plan->wide_mask & bit) != 0;
-    if (k_blocks < 200) return false;   // short K loops cannot amortise the epilogue that no longer overlaps
+// Mixed-width tile list for the long-K GEMMs: how many 256 x 512 tiles to put in front of the 256 x 256 ones.
+// Wide tiles move a quarter less data per FLOP and halve DRAM re-reads, but take two time units each and do not
+// overlap their epilogue; they are used for whole rounds of the CTA pairs as long as the total number of time units
+// does not grow, and only when the K loop is long enough to amortise the epilogue.  Returns 0 for "narrow kernel".
+int mixed_wide_tiles(const tsp_mlp_plan_t* plan, int bit, int n_blocks, int narrow_tiles, int k_blocks) {
+    if (n_blocks % 2 != 0) return 0;
     const int pairs = plan->sm_count / 2;
-    auto fill = [pairs](int tiles) {
-        const int rounds = (tiles + pairs - 1) / pairs;
-        return static_cast<double>(tiles) / (static_cast<double>(rounds) * pairs);
-    };
-    return fill(narrow_tiles / 2) >= fill(narrow_tiles) - 0.03;
+    const int all_wide = narrow_tiles / 2;
+    if (plan->wide_mask >= 0) return (plan->wide_mask & bit) ? all_wide : 0;
+    if (k_blocks < 200) return 0;
+    const int rounds_narrow = (narrow_tiles + pairs - 1) / pairs;
+    if (2 * ((all_wide + pairs - 1) / pairs) <= rounds_narrow) return all_wide;
+    for (int k = all_wide / pairs; k >= 1; --k) {
+        const int wide = k * pairs;
+        const int rest = narrow_tiles - 2 * wide;
+        if (2 * k + (rest + pairs - 1) / pairs <= rounds_narrow) return wide;
+    }
+    return 0;
 }
 
 template <class Params>
@@ -412,9 +418,9 @@ tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* W
     p.tiles_per_rank = static_cast<int>(S / D / 256);
     const int group = plan->group > 0 ? plan->group : 8;
     p.group = p.m_tiles < group ? p.m_tiles : group;
-    if (use_wide(plan, 1, H, p.m_tiles * p.n_blocks, F / 64)) {   // 256 x 512 tiles
-        p.n_blocks = H / 512;
-        fill_common(plan, p, p.m_tiles * p.n_blocks);
+    p.wide_tiles = mixed_wide_tiles(plan, 1, p.n_blocks, p.m_tiles * p.n_blocks, F / 64);
+    if (p.wide_tiles > 0) {
+        fill_common(plan, p, p.m_tiles * p.n_blocks - p.wide_tiles);   // wide tiles count once in the list
         return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDownPolicy>, p, stream);
     }
     fill_common(plan, p, p.m_tiles * p.n_blocks);
@@ -437,9 +443,9 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
     p.tiles_per_rank = static_cast<int>(S / D / 256);
     const int group = plan->dx_group > 0 ? plan->dx_group : 8;
     p.group = p.m_tiles < group ? p.m_tiles : group;
-    if (use_wide(plan, 2, H, p.m_tiles * p.n_blocks, 2 * F / 64)) {
-        p.n_blocks = H / 512;
-        fill_common(plan, p, p.m_tiles * p.n_blocks);
+    p.wide_tiles = mixed_wide_tiles(plan, 2, p.n_blocks, p.m_tiles * p.n_blocks, 2 * F / 64);
+    if (p.wide_tiles > 0) {
+        fill_common(plan, p, p.m_tiles * p.n_blocks - p.wide_tiles);
         return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDxPolicy>, p, stream);
     }
     fill_common(plan, p, p.m_tiles * p.n_blocks);
@@ -466,11 +472,9 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     // hidden blocks are taken in groups whose columns of X / dY (S * 512 bytes per block) fit in about 32 MB of L2
     int n_group = plan->dw_group > 0 ? plan->dw_group : static_cast<int>((32ull << 20) / (512ull * static_cast<size_t>(S)));
     if (n_group < 1) n_group = 1;
-    if (use_wide(plan, 4, H, 3 * p.j_tiles * p.n_blocks, static_cast<int>(S / 64))) {
-        p.n_blocks = H / 512;
-        n_group = (n_group + 1) / 2;
-        p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
-        fill_common(plan, p, 3 * p.j_tiles * p.n_blocks);
+    p.wide_tiles = mixed_wide_tiles(plan, 4, p.n_blocks, 3 * p.j_tiles * p.n_blocks, static_cast<int>(S / 64));
+    if (p.wide_tiles > 0) {
+        fill_common(plan, p, 3 * p.j_tiles * p.n_blocks - p.wide_tiles);
         return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDwPolicy>, p, stream);
     }
     p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
