@@ -117,3 +117,46 @@ def test_training_config_backward_sampled():
         assert g.shape == r.shape, name
         assert rel_fro(g, r) <= TOL_ORACLE, (name, rel_fro(g, r))
         assert worst_row_error(g.T if name != "dWd" else g, r.T if name != "dWd" else r) <= TOL_ROW, name
+
+
+def test_repeated_runs_are_bitwise_identical():
+    # A race between the producer, MMA and epilogue roles (or between the two CTAs of a pair) would show up as
+    # run-to-run differences; the schedule is static and no atomics are used, so every run must give the same bits.
+    import torch
+
+    from paper_2604_26294_b200 import binding as b
+
+    wl = inp.WORKLOADS["train"]
+    S, H, F, D = wl.S, wl.H, wl.F, wl.D
+    g = torch.Generator(device="cuda")
+    g.manual_seed(5)
+    X = torch.randn(S, H, device="cuda", generator=g).bfloat16()
+    dY = torch.randn(S, H, device="cuda", generator=g).bfloat16()
+    Wg = (torch.randn(D, H, F // D, device="cuda", generator=g) * H ** -0.5).bfloat16()
+    Wu = (torch.randn(D, H, F // D, device="cuda", generator=g) * H ** -0.5).bfloat16()
+    Wd = (torch.randn(D, F // D, H, device="cuda", generator=g) * F ** -0.5).bfloat16()
+    plan = b.tsp_mlp_plan(H, F, D)
+    try:
+        ws = torch.empty(b.tsp_mlp_workspace_bytes(plan, S, b.TSP_WS_BACKWARD), dtype=torch.uint8, device="cuda")
+        b.tsp_mlp_set_workspace(plan, ws)
+        outs = []
+        for it in range(12):
+            Y = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
+            dX = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
+            dWg = torch.empty(D, H, F // D, dtype=torch.float32, device="cuda")
+            dWu = torch.empty_like(dWg)
+            dWd = torch.empty(D, F // D, H, dtype=torch.float32, device="cuda")
+            b.tsp_mlp_forward(plan, X, Wg, Wu, Wd, Y, S, D)
+            b.tsp_mlp_backward(plan, X, Wg, Wu, Wd, dY, dX, dWg, dWu, dWd, S, D)
+            torch.cuda.synchronize()
+            assert b.tsp_mlp_status(plan) == b.TSP_OK
+            cur = (Y.view(torch.int16), dX.view(torch.int16), dWg.view(torch.int32), dWu.view(torch.int32),
+                   dWd.view(torch.int32))
+            if it == 0:
+                outs = [c.clone() for c in cur]
+            else:
+                for name, a, c in zip(("Y", "dX", "dWg", "dWu", "dWd"), outs, cur):
+                    assert bool((a == c).all()), (it, name)
+            del Y, dX, dWg, dWu, dWd
+    finally:
+        b.tsp_mlp_plan_destroy(plan)
