@@ -36,8 +36,8 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel
 # at the named workload, from the ncu capture summarised under profiles/.  None = not captured.
 NCU_DRAM_BYTES = {
-    ("gate_up", "7b_short"): 0.6358e9 + 0.2264e9,   # profiles/ncu_full_pair_kernels_7b_train.txt (same shapes)
-    ("gate_up", "train"): 0.6358e9 + 0.2264e9,
+    ("gate_up", "7b_short"): 0.6718e9 + 0.2261e9,   # profiles/ncu_full_pair_kernels_7b_train.txt (same shapes)
+    ("gate_up", "train"): 0.6718e9 + 0.2261e9,
 }
 
 
@@ -383,8 +383,8 @@ def run_gpu(args, wl):
     gate_up_flops = 4.0 * S * H * F
     achieved = gate_up_flops / (gate_up_ms * 1e-3) / 1e12
     pairs = (S // D) % 256 == 0 and os.environ.get("TSP_MLP_PAIR", "1") != "0"
-    gate_up_name = "pair_gemm_kernel<PairGateUpPolicy>" if pairs else "gate_up_swiglu_kernel"
-    down_name = "pair_gemm_kernel<PairDownPolicy>" if pairs else "down_accumulate_kernel"
+    gate_up_name = "pair_gemm_kernel<PairGateUpPolicyT<false>>" if pairs else "gate_up_swiglu_kernel"
+    down_name = "pair_{gemm,wide}_kernel<PairDownPolicy>" if pairs else "down_accumulate_kernel"
     roofline = {
         "bound": "tensor", "kernel": gate_up_name, "achieved": achieved, "peak": peaks["burst"],
         "unit": UNIT, "frac": achieved / peaks["burst"], "peak_source": f"of {peaks['source']} (burst bf16 GEMM)",
