@@ -10,7 +10,7 @@
  *
  * Conventions for every entry point
  *   - All matrix arguments are DEVICE pointers unless the name ends in _host.
- *     Row-major, bf16 (2 bytes) unless stated; 16-byte aligned.
+ *     Row-major, bf16 (2 bytes) unless stated; inputs 16-byte aligned, outputs (Y, dX, dW*) 32-byte aligned.
  *       X, Y, dY, dX : [S, H]            rank r = rows [r*S/D, (r+1)*S/D)
  *       Wg, Wu       : [D][H][F/D]       shard k = gate/up columns k*F/D .. (k+1)*F/D
  *       Wd           : [D][F/D][H]       shard k = down rows       k*F/D .. (k+1)*F/D

@@ -350,14 +350,11 @@ __device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t
         uint32_t v[32];
         tmem_ld32(t_row + c * 32, v);
         tmem_ld_wait();
-        uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+        uint32_t pk[16];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            dst[q] = make_uint4(pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])),
-                                pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
-                                pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
-                                pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
-        }
+        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+        st_global_256(out + c * 32, pk[0], pk[1], pk[2], pk[3], pk[4], pk[5], pk[6], pk[7]);
+        st_global_256(out + c * 32 + 16, pk[8], pk[9], pk[10], pk[11], pk[12], pk[13], pk[14], pk[15]);
     }
 }
 
@@ -434,23 +431,22 @@ struct PairGateUpPolicyT {
                     packed[i] = pack_bf16x2(gate_act(g0, p.act) * __uint_as_float(u[2 * i]),
                                             gate_act(g1, p.act) * __uint_as_float(u[2 * i + 1]));
                 }
-                uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                st_global_256(out + c * 32, packed[0], packed[1], packed[2], packed[3], packed[4], packed[5], packed[6],
+                              packed[7]);
+                st_global_256(out + c * 32 + 16, packed[8], packed[9], packed[10], packed[11], packed[12], packed[13],
+                              packed[14], packed[15]);
             }
         } else {
-            const float4* da_row = reinterpret_cast<const float4*>(p.dA + off);
+            const float* da_row = p.dA + off;
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {
-                float4 da4[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) da4[q] = __ldg(da_row + c * 4 + q);   // issued before the tensor-memory loads
+                uint32_t da4[2][8];
+                ld_global_nc_256(da_row + c * 16, da4[0]);       // issued before the tensor-memory loads
+                ld_global_nc_256(da_row + c * 16 + 8, da4[1]);
                 uint32_t g[16], u[16];
                 tmem_ld16(t_row + c * 16, g);
                 tmem_ld16(t_row + 128 + c * 16, u);
                 tmem_ld_wait();
-                const float* da = reinterpret_cast<const float*>(da4);
                 uint32_t pa[8], pg[8], pu[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
@@ -459,7 +455,7 @@ struct PairGateUpPolicyT {
                     for (int e = 0; e < 2; ++e) {
                         const float gg = __uint_as_float(g[2 * i + e]);
                         const float uu = __uint_as_float(u[2 * i + e]);
-                        const float dd = da[2 * i + e];
+                        const float dd = __uint_as_float(da4[(2 * i + e) >> 3][(2 * i + e) & 7]);
                         float sg, ds;
                         gate_act_grad(gg, p.act, sg, ds);                   // sigma(G), sigma'(G)
                         va[e] = sg * uu;                                    // A
@@ -470,15 +466,9 @@ struct PairGateUpPolicyT {
                     pg[i] = pack_bf16x2(vg[0], vg[1]);
                     pu[i] = pack_bf16x2(vu[0], vu[1]);
                 }
-                uint4* oa = reinterpret_cast<uint4*>(p.A + off + c * 16);
-                uint4* og = reinterpret_cast<uint4*>(p.dG + off + c * 16);
-                uint4* ou = reinterpret_cast<uint4*>(p.dU + off + c * 16);
-                oa[0] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
-                oa[1] = make_uint4(pa[4], pa[5], pa[6], pa[7]);
-                og[0] = make_uint4(pg[0], pg[1], pg[2], pg[3]);
-                og[1] = make_uint4(pg[4], pg[5], pg[6], pg[7]);
-                ou[0] = make_uint4(pu[0], pu[1], pu[2], pu[3]);
-                ou[1] = make_uint4(pu[4], pu[5], pu[6], pu[7]);
+                st_global_256(p.A + off + c * 16, pa[0], pa[1], pa[2], pa[3], pa[4], pa[5], pa[6], pa[7]);
+                st_global_256(p.dG + off + c * 16, pg[0], pg[1], pg[2], pg[3], pg[4], pg[5], pg[6], pg[7]);
+                st_global_256(p.dU + off + c * 16, pu[0], pu[1], pu[2], pu[3], pu[4], pu[5], pu[6], pu[7]);
             }
         }
     }
@@ -526,16 +516,16 @@ struct PairDaPolicy {
         pair_load_kmajor(sb, &p.map_wd, bar, kb * kBK, tl.jt * 256 + cta * 128, 0);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        float4* dst = reinterpret_cast<float4*>(p.dA + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F + tl.jt * 256);
+        float* dst = p.dA + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F + tl.jt * 256;
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
             uint32_t v[32];
             tmem_ld32(t_row + c * 32, v);
             tmem_ld_wait();
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-                dst[c * 8 + q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
-                                             __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+            for (int q = 0; q < 4; ++q)
+                st_global_256(dst + c * 32 + q * 8, v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
+                              v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
         }
     }
 };
@@ -827,11 +817,11 @@ struct PairDwPolicy {
             tmem_ld_wait();
             const int h0 = h_base + c * 32;
             if (tl.which == 0) {
-                float4* dst = reinterpret_cast<float4*>(p.dWd + static_cast<size_t>(j) * p.H + h0);
+                float* dst = p.dWd + static_cast<size_t>(j) * p.H + h0;
 #pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
-                                         __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                for (int q = 0; q < 4; ++q)
+                    st_global_256(dst + q * 8, v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4], v[8 * q + 5],
+                                  v[8 * q + 6], v[8 * q + 7]);
             } else {
                 float* base = (tl.which == 1 ? p.dWg : p.dWu) + static_cast<size_t>(tl.k) * p.H * F_d + (j - tl.k * F_d);
 #pragma unroll

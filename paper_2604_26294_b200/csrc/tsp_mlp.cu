@@ -104,6 +104,7 @@ bool encode_sharded(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, ui
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }  // outputs: 256-bit stores
 
 tsp_status_t check_call(const tsp_mlp_plan_t* plan, int64_t S, int D) {
     if (!plan) return TSP_ERR_INVALID_ARG;
@@ -649,7 +650,7 @@ tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg
     tsp_status_t st = check_call(plan, S, D);
     if (st != TSP_OK) return st;
     if (!X || !Wg || !Wu || !Wd || !Y) return TSP_ERR_INVALID_ARG;
-    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(Y)) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned32(Y)) return TSP_ERR_INVALID_ARG;
     if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes(plan, S, TSP_WS_FORWARD))
         return TSP_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -717,7 +718,7 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
     tsp_status_t st = check_call(plan, S, D);
     if (st != TSP_OK) return st;
     if (!X || !Wg || !Wu || !Wd || !Y) return TSP_ERR_INVALID_ARG;
-    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(Y)) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned32(Y)) return TSP_ERR_INVALID_ARG;
     if (compute_stream == copy_stream) return TSP_ERR_INVALID_ARG;
     if ((S / D) % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
     if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_staged(plan, S)) return TSP_ERR_WORKSPACE;
@@ -828,8 +829,8 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
     tsp_status_t st = check_call(plan, S, D);
     if (st != TSP_OK) return st;
     if (!X || !Wg || !Wu || !Wd || !dY || !dX || !dWg || !dWu || !dWd) return TSP_ERR_INVALID_ARG;
-    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(dY) || !aligned16(dX) ||
-        !aligned16(dWg) || !aligned16(dWu) || !aligned16(dWd))
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(dY) || !aligned32(dX) ||
+        !aligned32(dWg) || !aligned32(dWu) || !aligned32(dWd))
         return TSP_ERR_INVALID_ARG;
     if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes(plan, S, TSP_WS_BACKWARD))
         return TSP_ERR_WORKSPACE;
