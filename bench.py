@@ -250,6 +250,9 @@ def run_gpu(args, wl):
     copy_stream = torch.cuda.Stream() if staged else None
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     b.tsp_mlp_set_workspace(plan, ws)
+    stored = train and args.stored_activations
+    if stored:
+        saved = torch.empty(b.tsp_mlp_saved_bytes(plan, S), dtype=torch.uint8, device="cuda")
     if train:
         dY = dev(host.dY)
         dX = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
@@ -258,6 +261,10 @@ def run_gpu(args, wl):
         dWd = torch.empty(D, F // D, H, dtype=torch.float32, device="cuda")
 
     def step():
+        if stored:
+            b.tsp_mlp_forward_save(plan, X, Wg, Wu, Wd, Y, saved, S, D)
+            b.tsp_mlp_backward_saved(plan, X, Wg, Wu, Wd, dY, saved, dX, dWg, dWu, dWd, S, D)
+            return
         if staged:
             b.tsp_mlp_forward_staged(plan, X, Wg, Wu, Wd, Y, S, D, torch.cuda.current_stream(), copy_stream)
         else:
@@ -273,7 +280,7 @@ def run_gpu(args, wl):
     assert b.tsp_mlp_status(plan) == b.TSP_OK, "device-side wait timed out during warm-up"
     # counted after a call has been made: the backward count depends on the shape-dependent path taken
     kernels_per_step = (2 * D if staged else b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD)) + (
-        b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_BACKWARD) if train else 0)
+        (3 if stored else b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_BACKWARD)) if train else 0)
 
     # ---- timed region: K steps, inputs resident in HBM ----
     calls_per_step = 2 if train else 1
@@ -407,7 +414,9 @@ def run_gpu(args, wl):
         "dtype": "bf16", "data": "synthetic",
         "ms_per_step_kernels_median": float(np.median(step_sums)), "ms_per_step_kernels_min": float(np.min(step_sums)),
         "context": context,
-        "config": {"workload": wl.name, "pass": "forward+backward" if train else "forward", "S": S, "H": H, "F": F,
+        "config": {"workload": wl.name,
+                   "pass": ("forward+backward (stored activations)" if stored else
+                            "forward+backward (G, U recomputed)" if train else "forward"), "S": S, "H": H, "F": F,
                    "D": D, "tokens_per_rank": S // D, "shard_width": F // D, "model_flops_per_step": model_flops,
                    "l2": "inputs larger than L2 (X+W = %.0f MB, intermediate %.0f MB)" % (
                        (2 * S * H + 6 * H * F) / 1e6, 2 * S * F / 1e6),
@@ -433,6 +442,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="7b_short", choices=sorted(inp.WORKLOADS))
     ap.add_argument("--backward", action="store_true", help="time forward + backward (as the `train` workload does)")
+    ap.add_argument("--stored-activations", action="store_true",
+                    help="training step through tsp_mlp_forward_save / tsp_mlp_backward_saved (no recomputation)")
     ap.add_argument("--mode", default="direct", choices=["direct", "staged"],
                     help="staged: Algorithm 2 step by step with the shard transfer emulated on a side stream")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])

@@ -111,6 +111,27 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
                               float* dWd, int64_t S, int D, void* cuda_stream);
 
 /*
+ * Stored-activation training path.  The activation-memory analysis (Section 4.2) distinguishes full
+ * recomputation (only the layer input is kept: what tsp_mlp_backward does, recomputing G and U from X)
+ * from keeping the MLP activations.  This pair of calls is the second regime: tsp_mlp_forward_save computes
+ * the same Y as tsp_mlp_forward and additionally keeps, in the caller-owned device buffer `saved`
+ * (tsp_mlp_saved_bytes(plan, S) bytes, 256-byte aligned), A = sigma(G)*U, P = U*sigma'(G) and Q = sigma(G),
+ * each [S,F] in bf16.  tsp_mlp_backward_saved then needs no gate|up GEMM: dA = dY Wd^T stays in tensor memory
+ * and its epilogue writes dG = dA*P and dU = dA*Q (bf16, workspace); dX and the fp32 weight gradients follow
+ * as in tsp_mlp_backward (A is read from `saved`).  Hardware FLOPs equal model FLOPs (18 S H F per training
+ * step instead of 22 S H F); the cost is 3 S F bf16 elements of memory and one more bf16 rounding in dG, dU.
+ * Workspace for tsp_mlp_backward_saved: 2 * S * F * 2 bytes (tsp_mlp_workspace_bytes(.., TSP_WS_BACKWARD) is
+ * enough).  Shapes: (S/D) % 256 == 0 and F % 256 == 0, otherwise TSP_ERR_UNSUPPORTED_SHAPE.  tsp_mlp_forward_save
+ * does not use the plan's workspace.
+ */
+size_t tsp_mlp_saved_bytes(const tsp_mlp_plan_t* plan, int64_t S);
+tsp_status_t tsp_mlp_forward_save(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu,
+                                  const void* Wd, void* Y, void* saved, int64_t S, int D, void* cuda_stream);
+tsp_status_t tsp_mlp_backward_saved(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu,
+                                    const void* Wd, const void* dY, const void* saved, void* dX, float* dWg,
+                                    float* dWu, float* dWd, int64_t S, int D, void* cuda_stream);
+
+/*
  * tsp_mlp_forward_host - the same forward for callers whose tensors live in HOST
  * memory (pinned memory gives asynchronous copies).  Copies X, Wg, Wu, Wd to device
  * staging inside the workspace, runs tsp_mlp_forward, copies Y back; all on

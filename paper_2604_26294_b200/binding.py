@@ -37,6 +37,9 @@ SIGNATURES = {
     "tsp_mlp_workspace_bytes_host": (ctypes.c_size_t, [_P, ctypes.c_int64]),
     "tsp_mlp_set_workspace": (ctypes.c_int, [_P, _P, ctypes.c_size_t]),
     "tsp_mlp_forward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_mlp_saved_bytes": (ctypes.c_size_t, [_P, ctypes.c_int64]),
+    "tsp_mlp_forward_save": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_mlp_backward_saved": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_forward_host": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_backward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_workspace_bytes_staged": (ctypes.c_size_t, [_P, ctypes.c_int64]),
@@ -193,6 +196,23 @@ def tsp_mlp_selftest_wait_expiry(plan, limit_ms: int = 20, stream=None) -> None:
     """Make one bounded device-side wait expire on purpose (sets the plan's status word; harmless)."""
     _check(load_library().tsp_mlp_selftest_wait_expiry(plan, limit_ms, _stream_handle(stream)),
            "tsp_mlp_selftest_wait_expiry", plan)
+
+
+def tsp_mlp_saved_bytes(plan, S: int) -> int:
+    return int(load_library().tsp_mlp_saved_bytes(plan, S))
+
+
+def tsp_mlp_forward_save(plan, X, Wg, Wu, Wd, Y, saved, S: int, D: int, stream=None) -> None:
+    """Forward that also keeps A, U*sigma'(G) and sigma(G) in `saved` for tsp_mlp_backward_saved."""
+    _check(load_library().tsp_mlp_forward_save(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(Y), _ptr(saved), S, D,
+                                               _stream_handle(stream)), "tsp_mlp_forward_save", plan)
+
+
+def tsp_mlp_backward_saved(plan, X, Wg, Wu, Wd, dY, saved, dX, dWg, dWu, dWd, S: int, D: int, stream=None) -> None:
+    """Backward from stored activations (no gate|up recomputation)."""
+    _check(load_library().tsp_mlp_backward_saved(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(dY), _ptr(saved),
+                                                 _ptr(dX), _ptr(dWg), _ptr(dWu), _ptr(dWd), S, D,
+                                                 _stream_handle(stream)), "tsp_mlp_backward_saved", plan)
 
 
 def tsp_mlp_status(plan) -> int:

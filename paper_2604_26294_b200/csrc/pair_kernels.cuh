@@ -359,9 +359,12 @@ __device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t
 }
 
 // ---- gate | up + SwiGLU: tile = 256 tokens x 128 intermediate columns; CTA 0 loads the Wg half of B, CTA 1 the Wu half.
-// kBackward = false: epilogue writes A = silu(G) * U.
-// kBackward = true : epilogue also reads dA (fp32, from the dA GEMM) and writes A, dG = dA*U*silu'(G), dU = dA*silu(G).
-template <bool kBackward>
+// kMode 0 (forward)            : epilogue writes A = sigma(G) * U.
+// kMode 1 (backward, recompute): epilogue also reads dA (fp32, from the dA GEMM) and writes A, dG = dA*U*sigma'(G),
+//                                dU = dA*sigma(G).
+// kMode 2 (forward, storing)   : epilogue writes A and the two factors the backward pass needs, P = U*sigma'(G) and
+//                                Q = sigma(G), in bf16 (into p.dG and p.dU), so that no recomputation is needed later.
+template <int kMode>
 struct PairGateUpPolicyT {
     static constexpr bool kAMn = false, kBMn = true;
     struct Params {
@@ -416,7 +419,7 @@ struct PairGateUpPolicyT {
         // p.F is the row pitch of A: F in direct mode, F/D in staged mode (where the shard offset is dropped)
         const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F +
                            (p.rank_indexed ? 0 : static_cast<size_t>(tl.k) * p.F_d) + tl.jl * 128;
-        if constexpr (!kBackward) {
+        if constexpr (kMode == 0) {
             __nv_bfloat16* out = p.A + off;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
@@ -435,6 +438,35 @@ struct PairGateUpPolicyT {
                               packed[7]);
                 st_global_256(out + c * 32 + 16, packed[8], packed[9], packed[10], packed[11], packed[12], packed[13],
                               packed[14], packed[15]);
+            }
+        } else if constexpr (kMode == 2) {
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+                uint32_t g[16], u[16];
+                tmem_ld16(t_row + c * 16, g);
+                tmem_ld16(t_row + 128 + c * 16, u);
+                tmem_ld_wait();
+                uint32_t pa[8], pp[8], pq[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float va[2], vp[2], vq[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float gg = __uint_as_float(g[2 * i + e]);
+                        const float uu = __uint_as_float(u[2 * i + e]);
+                        float sg, ds;
+                        gate_act_grad(gg, p.act, sg, ds);
+                        va[e] = sg * uu;   // A
+                        vp[e] = uu * ds;   // P = U * sigma'(G)
+                        vq[e] = sg;        // Q = sigma(G)
+                    }
+                    pa[i] = pack_bf16x2(va[0], va[1]);
+                    pp[i] = pack_bf16x2(vp[0], vp[1]);
+                    pq[i] = pack_bf16x2(vq[0], vq[1]);
+                }
+                st_global_256(p.A + off + c * 16, pa[0], pa[1], pa[2], pa[3], pa[4], pa[5], pa[6], pa[7]);
+                st_global_256(p.dG + off + c * 16, pp[0], pp[1], pp[2], pp[3], pp[4], pp[5], pp[6], pp[7]);
+                st_global_256(p.dU + off + c * 16, pq[0], pq[1], pq[2], pq[3], pq[4], pq[5], pq[6], pq[7]);
             }
         } else {
             const float* da_row = p.dA + off;
@@ -473,15 +505,24 @@ struct PairGateUpPolicyT {
         }
     }
 };
-using PairGateUpPolicy = PairGateUpPolicyT<false>;
-using PairGateBwdPolicy = PairGateUpPolicyT<true>;
+using PairGateUpPolicy = PairGateUpPolicyT<0>;
+using PairGateBwdPolicy = PairGateUpPolicyT<1>;
+using PairGateSavePolicy = PairGateUpPolicyT<2>;
 
-// ---- dA = dY Wd^T (fp32 out): tile = 256 tokens x 256 intermediate columns; K = H ---------------------
-struct PairDaPolicy {
+// ---- dA = dY Wd^T: tile = 256 tokens x 256 intermediate columns; K = H ------------------------------------
+// kSaved = false: dA is written in fp32 (the gate|up GEMM of the recomputing backward consumes it).
+// kSaved = true : the forward pass stored P = U*sigma'(G) and Q = sigma(G); the epilogue forms dG = dA*P and
+//                 dU = dA*Q in fp32 and writes them in bf16, so dA never leaves tensor memory.
+template <bool kSaved>
+struct PairDaPolicyT {
     static constexpr bool kAMn = false, kBMn = false;
     struct Params {
         CUtensorMap map_dy, map_wd;  // (H, S, 1) box (64,128); (H, F, 1) box (64,128)
-        float* dA;                   // [S, F] fp32
+        float* dA;                   // [S, F] fp32 (kSaved = false)
+        const __nv_bfloat16* P;      // [S, F] (kSaved = true)
+        const __nv_bfloat16* Q;      // [S, F]
+        __nv_bfloat16* dG;           // [S, F]
+        __nv_bfloat16* dU;           // [S, F]
         int S, H, F, D;
         int m_tiles, j_tiles, band;
         int num_tiles, stages;
@@ -516,19 +557,45 @@ struct PairDaPolicy {
         pair_load_kmajor(sb, &p.map_wd, bar, kb * kBK, tl.jt * 256 + cta * 128, 0);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        float* dst = p.dA + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F + tl.jt * 256;
+        const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F + tl.jt * 256;
+        if constexpr (!kSaved) {
+            float* dst = p.dA + off;
 #pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
-            uint32_t v[32];
-            tmem_ld32(t_row + c * 32, v);
-            tmem_ld_wait();
+            for (int c = 0; c < 8; ++c) {
+                uint32_t v[32];
+                tmem_ld32(t_row + c * 32, v);
+                tmem_ld_wait();
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                st_global_256(dst + c * 32 + q * 8, v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
-                              v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
+                for (int q = 0; q < 4; ++q)
+                    st_global_256(dst + c * 32 + q * 8, v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
+                                  v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
+            }
+        } else {
+#pragma unroll 1
+            for (int c = 0; c < 16; ++c) {
+                uint32_t pr[8], qr[8], v[16];
+                ld_global_nc_256(p.P + off + c * 16, pr);   // 16 bf16 each, issued before the tensor-memory load
+                ld_global_nc_256(p.Q + off + c * 16, qr);
+                tmem_ld16(t_row + c * 16, v);
+                tmem_ld_wait();
+                uint32_t og[8], ou[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    // a bf16 pair widens to fp32 by shifting: low half is element 2i, high half element 2i+1
+                    const float p0 = __uint_as_float(pr[i] << 16), p1 = __uint_as_float(pr[i] & 0xFFFF0000u);
+                    const float q0 = __uint_as_float(qr[i] << 16), q1 = __uint_as_float(qr[i] & 0xFFFF0000u);
+                    const float d0 = __uint_as_float(v[2 * i]), d1 = __uint_as_float(v[2 * i + 1]);
+                    og[i] = pack_bf16x2(d0 * p0, d1 * p1);   // dG = dA * U * sigma'(G)
+                    ou[i] = pack_bf16x2(d0 * q0, d1 * q1);   // dU = dA * sigma(G)
+                }
+                st_global_256(p.dG + off + c * 16, og[0], og[1], og[2], og[3], og[4], og[5], og[6], og[7]);
+                st_global_256(p.dU + off + c * 16, ou[0], ou[1], ou[2], ou[3], ou[4], ou[5], ou[6], ou[7]);
+            }
         }
     }
 };
+using PairDaPolicy = PairDaPolicyT<false>;
+using PairDaSavedPolicy = PairDaPolicyT<true>;
 
 // ---- down projection: tile = 256 tokens x 256 hidden; K = F in ring order --------------------------
 struct PairDownPolicy {

@@ -359,10 +359,10 @@ tsp_status_t launch_pair(tsp_mlp_plan_t* plan, Kernel kernel, const Params& p, c
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
 
-template <bool kBackward>
+template <int kMode>
 tsp_status_t launch_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A,
                               const float* dA, void* dG, void* dU, int64_t S, cudaStream_t stream) {
-    using Policy = tsp::PairGateUpPolicyT<kBackward>;
+    using Policy = tsp::PairGateUpPolicyT<kMode>;
     const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
     typename Policy::Params p;
     std::memset(&p, 0, sizeof(p));
@@ -387,23 +387,34 @@ tsp_status_t launch_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* W
 
 tsp_status_t launch_gate_up_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A, int64_t S,
                                  cudaStream_t stream) {
-    return launch_gate_pair<false>(plan, X, Wg, Wu, A, nullptr, nullptr, nullptr, S, stream);
+    return launch_gate_pair<0>(plan, X, Wg, Wu, A, nullptr, nullptr, nullptr, S, stream);
 }
 
-// dA = dY Wd^T in fp32 (needs F % 256 == 0)
-tsp_status_t launch_da_pair(tsp_mlp_plan_t* plan, const void* dY, const void* Wd, float* dA, int64_t S, cudaStream_t stream) {
+// dA = dY Wd^T (needs F % 256 == 0).  kSaved = false: fp32 dA out; kSaved = true: dG = dA*P, dU = dA*Q out.
+template <bool kSaved>
+tsp_status_t launch_da_pair_t(tsp_mlp_plan_t* plan, const void* dY, const void* Wd, float* dA, const void* P, const void* Q,
+                              void* dG, void* dU, int64_t S, cudaStream_t stream) {
+    using Policy = tsp::PairDaPolicyT<kSaved>;
     const int H = plan->H, F = plan->F, D = plan->D;
-    tsp::PairDaPolicy::Params p;
+    typename Policy::Params p;
     std::memset(&p, 0, sizeof(p));
     if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 128)) return TSP_ERR_CUDA;
     if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 128)) return TSP_ERR_CUDA;
     p.dA = dA;
+    p.P = static_cast<const __nv_bfloat16*>(P);
+    p.Q = static_cast<const __nv_bfloat16*>(Q);
+    p.dG = static_cast<__nv_bfloat16*>(dG);
+    p.dU = static_cast<__nv_bfloat16*>(dU);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.m_tiles = static_cast<int>(S / 256);
     p.j_tiles = F / 256;
     p.band = gate_band(plan, p.m_tiles);
     fill_common(plan, p, p.m_tiles * p.j_tiles);
-    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDaPolicy>, p, stream);
+    return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
+}
+
+tsp_status_t launch_da_pair(tsp_mlp_plan_t* plan, const void* dY, const void* Wd, float* dA, int64_t S, cudaStream_t stream) {
+    return launch_da_pair_t<false>(plan, dY, Wd, dA, nullptr, nullptr, nullptr, nullptr, S, stream);
 }
 
 tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* Wd, void* Y, int64_t S, cudaStream_t stream) {
@@ -777,7 +788,7 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
         const void* cur_u = t == 0 ? Wu : recv(t & 1, 1);
         const void* cur_d = t == 0 ? Wd : recv(t & 1, 2);
         {
-            using Policy = tsp::PairGateUpPolicyT<false>;
+            using Policy = tsp::PairGateUpPolicyT<0>;
             Policy::Params p;
             std::memset(&p, 0, sizeof(p));
             if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
@@ -823,6 +834,73 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
     return TSP_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Stored-activation training path (the "no recomputation" regime of the activation-memory analysis): the forward
+// pass keeps A, P = U*sigma'(G) and Q = sigma(G) in a caller-owned buffer; the backward pass then needs no gate|up GEMM.
+// ---------------------------------------------------------------------------------------------
+size_t tsp_mlp_saved_bytes(const tsp_mlp_plan_t* plan, int64_t S) {
+    if (!plan || S <= 0) return 0;
+    return 3 * align_up(static_cast<size_t>(S) * plan->F * 2, 256);
+}
+
+static tsp_status_t check_saved_shapes(const tsp_mlp_plan_t* plan, int64_t S) {
+    if (!plan->use_pairs || (S / plan->D) % 256 != 0 || plan->F % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_forward_save(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
+                                  void* Y, void* saved, int64_t S, int D, void* cuda_stream) {
+    tsp_status_t st = check_call(plan, S, D);
+    if (st != TSP_OK) return st;
+    if (!X || !Wg || !Wu || !Wd || !Y || !saved) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned32(Y) ||
+        (reinterpret_cast<uintptr_t>(saved) & 255u))
+        return TSP_ERR_INVALID_ARG;
+    if ((st = check_saved_shapes(plan, S)) != TSP_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t one = align_up(static_cast<size_t>(S) * plan->F * 2, 256);
+    uint8_t* base = static_cast<uint8_t*>(saved);
+    Profiler prof(plan, stream);
+    st = launch_gate_pair<2>(plan, X, Wg, Wu, base, nullptr, base + one, base + 2 * one, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    st = launch_down_pair(plan, base, Wd, Y, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    return TSP_OK;
+}
+
+tsp_status_t tsp_mlp_backward_saved(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
+                                    const void* dY, const void* saved, void* dX, float* dWg, float* dWu, float* dWd,
+                                    int64_t S, int D, void* cuda_stream) {
+    tsp_status_t st = check_call(plan, S, D);
+    if (st != TSP_OK) return st;
+    if (!X || !Wg || !Wu || !Wd || !dY || !saved || !dX || !dWg || !dWu || !dWd) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(dY) || !aligned32(dX) ||
+        !aligned32(dWg) || !aligned32(dWu) || !aligned32(dWd) || (reinterpret_cast<uintptr_t>(saved) & 255u))
+        return TSP_ERR_INVALID_ARG;
+    if ((st = check_saved_shapes(plan, S)) != TSP_OK) return st;
+    const size_t one = align_up(static_cast<size_t>(S) * plan->F * 2, 256);
+    if (!plan->workspace || plan->workspace_bytes < 2 * one) return TSP_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint8_t* sv = static_cast<const uint8_t*>(saved);
+    uint8_t* ws = static_cast<uint8_t*>(plan->workspace);
+    void* dG = ws;
+    void* dU = ws + one;
+    Profiler prof(plan, stream);
+    st = launch_da_pair_t<true>(plan, dY, Wd, nullptr, sv + one, sv + 2 * one, dG, dU, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    st = launch_bwd_dx_pair(plan, dG, dU, Wg, Wu, dX, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    st = pairs_for_dw(plan) ? launch_bwd_dw_pair(plan, X, dY, sv, dG, dU, dWg, dWu, dWd, S, stream)
+                            : launch_bwd_dw(plan, X, dY, sv, dG, dU, dWg, dWu, dWd, S, stream);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    return TSP_OK;
+}
+
 tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
                               const void* dY, void* dX, float* dWg, float* dWu, float* dWd, int64_t S, int D,
                               void* cuda_stream) {
@@ -848,7 +926,7 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
         st = launch_da_pair(plan, dY, Wd, dA, S, stream);
         if (st != TSP_OK) return st;
         prof.mark();
-        st = launch_gate_pair<true>(plan, X, Wg, Wu, A, dA, dG, dU, S, stream);
+        st = launch_gate_pair<1>(plan, X, Wg, Wu, A, dA, dG, dU, S, stream);
     } else {
         st = launch_bwd_gate(plan, X, Wg, Wu, Wd, dY, A, dG, dU, S, stream);
     }
