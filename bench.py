@@ -390,7 +390,7 @@ def run_gpu(args, wl):
     gate_up_flops = 4.0 * S * H * F
     achieved = gate_up_flops / (gate_up_ms * 1e-3) / 1e12
     pairs = (S // D) % 256 == 0 and os.environ.get("TSP_MLP_PAIR", "1") != "0"
-    gate_up_name = "pair_gemm_kernel<PairGateUpPolicyT<false>>" if pairs else "gate_up_swiglu_kernel"
+    gate_up_name = ("pair_gemm_kernel<PairGateUpPolicyT<%d>>" % (2 if stored else 0)) if pairs else "gate_up_swiglu_kernel"
     down_name = "pair_{gemm,wide}_kernel<PairDownPolicy>" if pairs else "down_accumulate_kernel"
     roofline = {
         "bound": "tensor", "kernel": gate_up_name, "achieved": achieved, "peak": peaks["burst"],

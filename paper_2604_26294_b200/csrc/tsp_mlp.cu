@@ -60,6 +60,9 @@ struct tsp_mlp_plan {
     int wide_mask;              // 256 x 512 tiles for: bit 0 down, bit 1 dX, bit 2 dW (env TSP_MLP_WIDE)
     int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
+    cudaStream_t host_copy_stream;           // tsp_mlp_forward_host: uploads Wd while the gate|up kernel runs
+    cudaEvent_t host_events[3];
+    bool host_ready;
 };
 
 namespace {
@@ -594,6 +597,7 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->group = env_int("TSP_MLP_GROUP", 0);
     plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
     plan->last_backward_kernels = 3;
+    plan->host_ready = false;
     plan->phase_mask = env_int("TSP_MLP_PHASES", 3);
     plan->act = TSP_ACT_SILU;
     plan->wide_mask = env_int("TSP_MLP_WIDE", -1);   // -1: decide per launch from the tile counts
@@ -622,6 +626,10 @@ tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan) {
     if (!plan) return TSP_ERR_INVALID_ARG;
     tsp_mlp_profile_end(plan);
     for (auto& ev : plan->staged_events) cudaEventDestroy(ev);
+    if (plan->host_ready) {
+        for (auto& ev : plan->host_events) cudaEventDestroy(ev);
+        cudaStreamDestroy(plan->host_copy_stream);
+    }
     if (plan->status_dev) cudaFree(plan->status_dev);
     delete plan;
     return TSP_OK;
@@ -656,8 +664,17 @@ tsp_status_t tsp_mlp_set_activation(tsp_mlp_plan_t* plan, int activation) {
     return TSP_OK;
 }
 
+static tsp_status_t forward_impl(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
+                                 void* Y, int64_t S, int D, void* cuda_stream, cudaEvent_t wait_before_down);
+
 tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
                              void* Y, int64_t S, int D, void* cuda_stream) {
+    return forward_impl(plan, X, Wg, Wu, Wd, Y, S, D, cuda_stream, nullptr);
+}
+
+// `wait_before_down`: if set, the down-projection kernel additionally waits for this event (Wd still arriving).
+static tsp_status_t forward_impl(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, const void* Wd,
+                                 void* Y, int64_t S, int D, void* cuda_stream, cudaEvent_t wait_before_down) {
     tsp_status_t st = check_call(plan, S, D);
     if (st != TSP_OK) return st;
     if (!X || !Wg || !Wu || !Wd || !Y) return TSP_ERR_INVALID_ARG;
@@ -673,6 +690,10 @@ tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg
         if (st != TSP_OK) return st;
     }
     prof.mark();
+    if (wait_before_down) {
+        cudaError_t e = cudaStreamWaitEvent(stream, wait_before_down, 0);
+        if (e != cudaSuccess) return cuda_fail(plan, e);
+    }
     if (plan->phase_mask & 2) {
         st = pairs ? launch_down_pair(plan, plan->workspace, Wd, Y, S, stream)
                    : launch_down(plan, plan->workspace, Wd, Y, S, stream);
@@ -699,12 +720,24 @@ tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, cons
     uint8_t* dWu = dWg + w;
     uint8_t* dWd = dWu + w;
     cudaError_t e;
+    if (!plan->host_ready) {   // created on first use: a side stream and three events (no device memory)
+        if ((e = cudaStreamCreateWithFlags(&plan->host_copy_stream, cudaStreamNonBlocking)) != cudaSuccess)
+            return cuda_fail(plan, e);
+        for (auto& ev : plan->host_events)
+            if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(plan, e);
+        plan->host_ready = true;
+    }
+    cudaStream_t side = plan->host_copy_stream;
+    // X, Wg, Wu first: the gate|up kernel needs them; Wd follows on the side stream and arrives while gate|up runs.
     if ((e = cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
     if ((e = cudaMemcpyAsync(dWg, Wg_host, wb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
     if ((e = cudaMemcpyAsync(dWu, Wu_host, wb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
-    if ((e = cudaMemcpyAsync(dWd, Wd_host, wb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaEventRecord(plan->host_events[0], stream)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaStreamWaitEvent(side, plan->host_events[0], 0)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaMemcpyAsync(dWd, Wd_host, wb, cudaMemcpyHostToDevice, side)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaEventRecord(plan->host_events[1], side)) != cudaSuccess) return cuda_fail(plan, e);
     // The forward proper uses only the first `a` bytes of the workspace.
-    st = tsp_mlp_forward(plan, dX, dWg, dWu, dWd, dY, S, D, cuda_stream);
+    st = forward_impl(plan, dX, dWg, dWu, dWd, dY, S, D, cuda_stream, plan->host_events[1]);
     if (st != TSP_OK) return st;
     if ((e = cudaMemcpyAsync(Y_host, dY, xb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(plan, e);
     return TSP_OK;
