@@ -136,8 +136,10 @@ __device__ __forceinline__ void pair_teardown(SharedCtl* ctl, const WaitCtx& w) 
 
 // ------------------------------------------------------------------------------------------------
 // Generic pair kernel: tile = 256 rows (128 per CTA) x 256 columns, one K loop, two accumulator buffers.
-// Policy: Params{num_tiles, stages, status, timeout_ns}, Tile decode(p, tile), k_blocks(p),
-//         load(p, tile, kb, cta, sa, sb, bar), kAMn, kBMn, epilogue(p, tile, cta, row, t_row).
+// Policy: Params{num_tiles, stages, status, timeout_ns}; Tile decode(p, tile); the K loop is outer(p) x inner(p)
+//         k-blocks with sel = select(p, tile, o) chosen once per outer step (the shard or rank met at that ring step);
+//         load(p, tile, sel, i, cta, sa, sb, bar) issues this CTA's TMA loads of one k-block; kAMn / kBMn give the
+//         operand majors; epilogue(p, tile, cta, row, t_row) drains one accumulator row.
 // ------------------------------------------------------------------------------------------------
 template <class Policy>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
