@@ -64,6 +64,8 @@ WORKLOADS = {
     "train": Workload("train", S=8192, H=4096, F=14336, D=8),
     # the paper's own 7B-class MLP: expansion factor 4, intermediate width 4 * 4096 (reference-model table)
     "7b_paper": Workload("7b_paper", S=8192, H=4096, F=16384, D=8),
+    # a larger model shape (hidden 8192, intermediate 28672) to exercise other H / F than the 7B ones
+    "70b_short": Workload("70b_short", S=4096, H=8192, F=28672, D=8),
 }
 
 

@@ -56,6 +56,14 @@ def test_paper_7b_shape_forward_sampled_rows():
     _check_forward_rows(prob, Y, inp.sample_rows(wl.S, wl.D), _weights64(prob.host))
 
 
+def test_larger_model_shape_forward_sampled_rows():
+    # hidden 8192, intermediate 28672: other band / group sizes and twice the K of the 7B shapes
+    wl = inp.WORKLOADS["70b_short"]
+    prob = DeviceProblem(wl.S, wl.H, wl.F, wl.D, seed=0)
+    Y = prob.forward()
+    _check_forward_rows(prob, Y, inp.sample_rows(wl.S, wl.D), _weights64(prob.host))
+
+
 def test_7b_long_forward_sampled_rows():
     wl = inp.WORKLOADS["7b_long"]
     prob = DeviceProblem(wl.S, wl.H, wl.F, wl.D, seed=0)
