@@ -226,6 +226,13 @@ def run_gpu(args, wl):
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    # the library normally arrives built; if it is missing or older than its sources, rank 0 compiles it (nvcc, ~1 min)
+    from paper_2604_26294_b200 import build as _build
+
+    if local_rank == 0:
+        _build.build_library()
+    if world > 1:
+        dist.barrier()
 
     def barrier():
         if world > 1:
