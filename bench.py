@@ -36,8 +36,8 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel
 # at the named workload, from the ncu capture summarised under profiles/.  None = not captured.
 NCU_DRAM_BYTES = {
-    ("gate_up", "7b_short"): 0.6718e9 + 0.2261e9,   # profiles/ncu_full_pair_kernels_7b_train.txt (same shapes)
-    ("gate_up", "train"): 0.6718e9 + 0.2261e9,
+    ("gate_up", "7b_short"): 0.6946e9 + 0.2263e9,   # profiles/ncu_full_pair_kernels_7b_train.txt (same shapes)
+    ("gate_up", "train"): 0.6946e9 + 0.2263e9,
 }
 
 
