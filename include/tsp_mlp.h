@@ -22,8 +22,11 @@
  *     the default stream).  Argument and launch errors are returned at once; a device
  *     wait that ran out of time is reported by tsp_mlp_status after a synchronize.
  *   - No exceptions, no abort, no CPU fallback.  Unsupported shapes are refused before
- *     any launch.  Supported: H % 256 == 0, (F/D) % 128 == 0, (S/D) % 128 == 0, F % D == 0,
- *     S % D == 0, 1 <= D <= 64.
+ *     any launch.  Supported: H % 256 == 0, (F/D) % 128 == 0, F % D == 0, S % D == 0 (any number
+ *     of tokens per rank >= 1), 1 <= D <= 64, S <= 2^24.  The model dimensions must fit the tile
+ *     sizes; the token count need not: the last token tile of a rank is loaded whole and only its
+ *     valid rows are stored.  When S/D is not a multiple of 64 the weight gradients contract the
+ *     tokens in ascending order instead of rank order (a k-block would otherwise straddle two ranks).
  *   - A plan must not be used from two host threads at once, nor on two streams at
  *     once (the workspace and status word are shared).
  *   - Results are deterministic: no atomics, fixed accumulation order.
@@ -43,7 +46,7 @@ typedef struct tsp_mlp_plan tsp_mlp_plan_t; /* opaque; created by tsp_mlp_plan, 
 typedef enum {
     TSP_OK = 0,
     TSP_ERR_INVALID_ARG = -1,        /* null pointer, misaligned pointer, D differs from the plan, S <= 0 */
-    TSP_ERR_UNSUPPORTED_SHAPE = -2,  /* divisibility rules above not met */
+    TSP_ERR_UNSUPPORTED_SHAPE = -2,  /* divisibility rules above not met (or a path-specific rule, see each call) */
     TSP_ERR_UNSUPPORTED_DEVICE = -3, /* current device is not compute capability 10.x */
     TSP_ERR_CUDA = -4,               /* a CUDA runtime / driver call failed (see tsp_mlp_last_cuda_error) */
     TSP_ERR_WORKSPACE = -5,          /* workspace missing or smaller than tsp_mlp_workspace_bytes */
@@ -121,7 +124,9 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
  * as in tsp_mlp_backward (A is read from `saved`).  Hardware FLOPs equal model FLOPs (18 S H F per training
  * step instead of 22 S H F); the cost is 3 S F bf16 elements of memory and one more bf16 rounding in dG, dU.
  * Workspace for tsp_mlp_backward_saved: 2 * S * F * 2 bytes (tsp_mlp_workspace_bytes(.., TSP_WS_BACKWARD) is
- * enough).  Shapes: (S/D) % 256 == 0 and F % 256 == 0, otherwise TSP_ERR_UNSUPPORTED_SHAPE.  tsp_mlp_forward_save
+ * enough).  Shapes: F % 256 == 0 and a token count per rank that the CTA-pair kernels take (S/D a multiple of
+ * 256, or large enough that padding the last 256-row tile costs little), otherwise TSP_ERR_UNSUPPORTED_SHAPE.
+ * tsp_mlp_forward_save
  * does not use the plan's workspace.
  */
 size_t tsp_mlp_saved_bytes(const tsp_mlp_plan_t* plan, int64_t S);
@@ -153,7 +158,9 @@ tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, cons
  * scratch, then the down projection of that shard added into an fp32 [S, H] accumulator; the last step
  * rounds the accumulator to bf16 Y.  Events order "received" before "compute t+1" and "computed t-1"
  * before the buffers are overwritten.  Same result as tsp_mlp_forward up to fp32 summation order
- * (per-shard partial sums are formed first).  Needs (S/D) % 256 == 0, two distinct streams, and a
+ * (per-shard partial sums are formed first).  Needs a token count per rank that the CTA-pair kernels
+ * take (S/D a multiple of 256, or large enough that padding the last 256-row tile costs little: the same
+ * rule tsp_mlp_forward applies internally), two distinct streams, and a
  * workspace of tsp_mlp_workspace_bytes_staged(plan, S) bytes (scratch, accumulator, 2 x 3 receive buffers
  * of the size of one weight matrix).  2*D kernels and at most 6*(D-1) copies per call.
  */
@@ -234,7 +241,7 @@ tsp_status_t tsp_mlp_profile_read(tsp_mlp_plan_t* plan, int call_index, int* n_k
 tsp_status_t tsp_mlp_profile_end(tsp_mlp_plan_t* plan);
 
 /* Number of kernels one forward call launches (pass=TSP_WS_FORWARD: 2), or that the most recent
- * tsp_mlp_backward on this plan launched (pass=TSP_WS_BACKWARD: 4 when (S/D) % 256 == 0 and F % 256 == 0,
+ * tsp_mlp_backward on this plan launched (pass=TSP_WS_BACKWARD: 4 on the CTA-pair path with F % 256 == 0,
  * else 3; 3 before the first backward call). */
 int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass);
 

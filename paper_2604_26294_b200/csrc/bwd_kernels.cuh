@@ -36,7 +36,7 @@ struct BwdGateParams {
     __nv_bfloat16* A;     // [S, F]
     __nv_bfloat16* dG;    // [S, F]
     __nv_bfloat16* dU;    // [S, F]
-    int S, H, F, D;
+    int S, H, F, D, S_loc;
     int m_blocks, blocks_per_rank, jl_blocks, band, num_tiles, stages;
     int act;              // gate activation
     int* status;
@@ -44,7 +44,7 @@ struct BwdGateParams {
 };
 
 struct BwdGateTile {
-    int mb, r, k, jl;
+    int mb, r, k, jl, row0, valid;
 };
 
 __device__ __forceinline__ BwdGateTile bwd_gate_tile(const BwdGateParams& p, int tile) {
@@ -58,7 +58,7 @@ __device__ __forceinline__ BwdGateTile bwd_gate_tile(const BwdGateParams& p, int
     BwdGateTile o;
     o.jl = rem / band_sz;
     o.mb = band_start + rem % band_sz;
-    o.r = o.mb / p.blocks_per_rank;
+    token_tile(o.mb, p.blocks_per_rank, p.S_loc, 128, o.r, o.row0, o.valid);
     o.k = (o.r - t + p.D) % p.D;
     return o;
 }
@@ -96,12 +96,12 @@ __global__ void __launch_bounds__(kNumThreads, 1) bwd_gate_kernel(const __grid_c
                     ctl->issued[ps.stage] = 1u + ps.phase;
                     if (kb < k_blocks) {  // dA = dY Wd_k^T
                         mbar_arrive_expect_tx(bar, kBytesDA);
-                        load_kmajor(sa, &p.map_dy, bar, kb * kBK, tl.mb * 128, 0);
+                        load_kmajor(sa, &p.map_dy, bar, kb * kBK, tl.row0, 0);
                         load_kmajor(sb, &p.map_wd, bar, kb * kBK, tl.k * F_d + tl.jl * 128, 0);
                     } else {              // G | U = X [Wg_k | Wu_k]
                         const int h0 = (kb - k_blocks) * kBK;
                         mbar_arrive_expect_tx(bar, kBytesGU);
-                        load_kmajor(sa, &p.map_x, bar, h0, tl.mb * 128, 0);
+                        load_kmajor(sa, &p.map_x, bar, h0, tl.row0, 0);
                         load_mnmajor(sb, &p.map_wg, bar, tl.jl * 128, h0, tl.k, 2);
                         load_mnmajor(sb + 2 * 8192, &p.map_wu, bar, tl.jl * 128, h0, tl.k, 2);
                     }
@@ -154,7 +154,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) bwd_gate_kernel(const __grid_c
             if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[slot]), (it >> 1) & 1, w, kErrWaitTmemFull))) break;
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            const size_t off = static_cast<size_t>(tl.mb * 128 + row) * p.F + static_cast<size_t>(tl.k) * F_d + tl.jl * 128;
+            const bool live = row < tl.valid;
+            const size_t off = static_cast<size_t>(tl.row0 + row) * p.F + static_cast<size_t>(tl.k) * F_d + tl.jl * 128;
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {
                 uint32_t g[16], u[16], da[16];
@@ -184,12 +185,14 @@ __global__ void __launch_bounds__(kNumThreads, 1) bwd_gate_kernel(const __grid_c
                 uint4* oa = reinterpret_cast<uint4*>(p.A + off + c * 16);
                 uint4* og = reinterpret_cast<uint4*>(p.dG + off + c * 16);
                 uint4* ou = reinterpret_cast<uint4*>(p.dU + off + c * 16);
-                oa[0] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
-                oa[1] = make_uint4(pa[4], pa[5], pa[6], pa[7]);
-                og[0] = make_uint4(pg[0], pg[1], pg[2], pg[3]);
-                og[1] = make_uint4(pg[4], pg[5], pg[6], pg[7]);
-                ou[0] = make_uint4(pu[0], pu[1], pu[2], pu[3]);
-                ou[1] = make_uint4(pu[4], pu[5], pu[6], pu[7]);
+                if (live) {
+                    oa[0] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
+                    oa[1] = make_uint4(pa[4], pa[5], pa[6], pa[7]);
+                    og[0] = make_uint4(pg[0], pg[1], pg[2], pg[3]);
+                    og[1] = make_uint4(pg[4], pg[5], pg[6], pg[7]);
+                    ou[0] = make_uint4(pu[0], pu[1], pu[2], pu[3]);
+                    ou[1] = make_uint4(pu[4], pu[5], pu[6], pu[7]);
+                }
             }
             tc_fence_before_sync();
             mbar_arrive(smem_u32(&ctl->tmem_empty[2]));
@@ -291,13 +294,13 @@ struct BwdDxPolicy {
         CUtensorMap map_wg;  // Wg (F/D, H, D)   box (64, 256)   K-major B operand (rows = hidden index)
         CUtensorMap map_wu;  // Wu likewise
         __nv_bfloat16* dX;   // [S, H]
-        int S, H, F, D;
+        int S, H, F, D, S_loc;
         int m_blocks, n_blocks, blocks_per_rank, group, num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
     };
     struct Tile {
-        int mb, nb, r;
+        int mb, nb, r, row0, valid;
     };
     __device__ static __forceinline__ int k_blocks(const Params& p) { return 2 * (p.F / kBK); }
     __device__ static __forceinline__ void prefetch(const Params& p) {
@@ -315,7 +318,7 @@ struct BwdDxPolicy {
         Tile o;
         o.nb = rem / g_sz;
         o.mb = g_start + rem % g_sz;
-        o.r = o.mb / p.blocks_per_rank;
+        token_tile(o.mb, p.blocks_per_rank, p.S_loc, 128, o.r, o.row0, o.valid);
         return o;
     }
     // k-block order: ring step t -> shard k = (r - t) mod D -> 64-wide slice of the shard -> (dG Wg^T, dU Wu^T)
@@ -328,11 +331,12 @@ struct BwdDxPolicy {
         const int k = (tl.r - t + p.D) % p.D;
         const int j0 = (rem >> 1) * kBK;
         const bool up = rem & 1;
-        load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * F_d + j0, tl.mb * 128, 0);
+        load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * F_d + j0, tl.row0, 0);
         load_kmajor(sb, up ? &p.map_wu : &p.map_wg, bar, j0, tl.nb * 256, k);
     }
     __device__ static __forceinline__ void store(const Params& p, const Tile& tl, int row, int c, const uint32_t (&v)[32]) {
-        __nv_bfloat16* out = p.dX + static_cast<size_t>(tl.mb * 128 + row) * p.H + tl.nb * 256 + c * 32;
+        if (row >= tl.valid) return;
+        __nv_bfloat16* out = p.dX + static_cast<size_t>(tl.row0 + row) * p.H + tl.nb * 256 + c * 32;
         uint4* dst = reinterpret_cast<uint4*>(out);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -360,6 +364,7 @@ struct BwdDwPolicy {
         float* dWg;          // [D][H][F/D]
         float* dWu;          // [D][H][F/D]
         int S, H, F, D;
+        int k_linear;        // 0, or ceil(S / 64) when the tokens are contracted in ascending order (ragged ranks)
         int j_blocks, n_blocks, num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -367,7 +372,7 @@ struct BwdDwPolicy {
     struct Tile {
         int which, jb, nb, k;
     };
-    __device__ static __forceinline__ int k_blocks(const Params& p) { return p.S / kBK; }
+    __device__ static __forceinline__ int k_blocks(const Params& p) { return p.k_linear ? p.k_linear : p.S / kBK; }
     __device__ static __forceinline__ void prefetch(const Params& p) {
         tma_prefetch_desc(&p.map_a);
         tma_prefetch_desc(&p.map_dg);
@@ -388,11 +393,16 @@ struct BwdDwPolicy {
     // token order: shard k meets the ranks in the order r = (k + t) mod D
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int kb, uint32_t sa, uint32_t sb,
                                                 uint32_t bar) {
-        const int S_loc = p.S / p.D;
-        const int per_rank = S_loc / kBK;
-        const int t = kb / per_rank;
-        const int r = (tl.k + t) % p.D;
-        const int s0 = r * S_loc + (kb - t * per_rank) * kBK;
+        int s0;
+        if (p.k_linear) {   // ragged ranks: ascending token order, the tail k-block is zero-filled by the TMA unit
+            s0 = kb * kBK;
+        } else {
+            const int S_loc = p.S / p.D;
+            const int per_rank = S_loc / kBK;
+            const int t = kb / per_rank;
+            const int r = (tl.k + t) % p.D;
+            s0 = r * S_loc + (kb - t * per_rank) * kBK;
+        }
         const CUtensorMap* ma = tl.which == 0 ? &p.map_a : (tl.which == 1 ? &p.map_dg : &p.map_du);
         const CUtensorMap* mb = tl.which == 0 ? &p.map_dy : &p.map_x;
         load_mnmajor(sa, ma, bar, tl.jb * 128, s0, 0, 2);

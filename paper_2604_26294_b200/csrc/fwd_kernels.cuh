@@ -21,9 +21,9 @@ struct GateUpParams {
     CUtensorMap map_wg;  // Wg as (F/D, H, D),  box (64, 64, 1)    MN-major B operand
     CUtensorMap map_wu;  // Wu likewise
     __nv_bfloat16* A;    // [S, F] bf16 intermediate
-    int S, H, F, D;
-    int m_blocks;        // S / 128
-    int blocks_per_rank; // (S/D) / 128
+    int S, H, F, D, S_loc;
+    int m_blocks;        // D * blocks_per_rank
+    int blocks_per_rank; // ceil((S/D) / 128): the last block of a rank may be partial
     int jl_blocks;       // (F/D) / 128
     int band;            // token blocks per band (their X rows stay L2-resident while the shards stream)
     int shared_order;    // 0: ranks of a band follow the ring (different shards at a time); 1: same column block for all
@@ -35,7 +35,7 @@ struct GateUpParams {
 };
 
 struct GateUpTile {
-    int mb, r, k, jl;
+    int mb, r, k, jl, row0, valid;
 };
 
 // Tile order: band of token blocks -> ring step t -> column block jl of the shard -> token block.
@@ -51,7 +51,7 @@ __device__ __forceinline__ GateUpTile gate_up_tile(const GateUpParams& p, int ti
     GateUpTile o;
     o.jl = rem / band_sz;
     o.mb = band_start + rem % band_sz;
-    o.r = o.mb / p.blocks_per_rank;
+    token_tile(o.mb, p.blocks_per_rank, p.S_loc, kBM, o.r, o.row0, o.valid);
     o.k = p.shared_order ? t : (o.r - t + p.D) % p.D;
     return o;
 }
@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) gate_up_swiglu_kernel(const __
                     const uint32_t sa = smem_base + ps.stage * kStageBytes, sb = sa + kABytes;
                     ctl->issued[ps.stage] = 1u + ps.phase;
                     mbar_arrive_expect_tx(bar, kStageBytes);
-                    load_kmajor(sa, &p.map_x, bar, kb * kBK, tl.mb * kBM, 0);
+                    load_kmajor(sa, &p.map_x, bar, kb * kBK, tl.row0, 0);
                     load_mnmajor(sb, &p.map_wg, bar, tl.jl * 128, kb * kBK, tl.k, 2);
                     load_mnmajor(sb + 2 * 8192, &p.map_wu, bar, tl.jl * 128, kb * kBK, tl.k, 2);
                     ps.advance(p.stages);
@@ -126,7 +126,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) gate_up_swiglu_kernel(const __
             if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[buf]), acc_phase, w, kErrWaitTmemFull))) break;
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
-            __nv_bfloat16* out = p.A + static_cast<size_t>(tl.mb * kBM + row) * p.F +
+            const bool live = row < tl.valid;   // rows past the rank's end are not stored
+            __nv_bfloat16* out = p.A + static_cast<size_t>(tl.row0 + row) * p.F +
                                  static_cast<size_t>(tl.k) * (p.F / p.D) + tl.jl * 128;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
@@ -143,9 +144,11 @@ __global__ void __launch_bounds__(kNumThreads, 1) gate_up_swiglu_kernel(const __
                     packed[i] = pack_bf16x2(a0, a1);
                 }
                 uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+                if (live) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                    for (int q = 0; q < 4; ++q)
+                        dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                }
             }
             tc_fence_before_sync();
             mbar_arrive(smem_u32(&ctl->tmem_empty[buf]));
@@ -162,8 +165,8 @@ struct DownParams {
     CUtensorMap map_a;   // A  as (F, S, 1), box (64, 128, 1)   K-major A operand
     CUtensorMap map_wd;  // Wd as (H, F, 1), box (64, 64, 1)    MN-major B operand ([D][F/D][H] is [F][H])
     __nv_bfloat16* Y;    // [S, H]
-    int S, H, F, D;
-    int m_blocks, n_blocks;  // S/128, H/256
+    int S, H, F, D, S_loc;
+    int m_blocks, n_blocks;  // D * blocks_per_rank, H/256
     int blocks_per_rank;
     int group;               // token blocks per tile group (share Wd column blocks in L2)
     int num_tiles;
@@ -173,7 +176,7 @@ struct DownParams {
 };
 
 struct DownTile {
-    int mb, nb, r;
+    int mb, nb, r, row0, valid;
 };
 
 __device__ __forceinline__ DownTile down_tile(const DownParams& p, int tile) {
@@ -185,7 +188,7 @@ __device__ __forceinline__ DownTile down_tile(const DownParams& p, int tile) {
     DownTile o;
     o.nb = rem / g_sz;
     o.mb = g_start + rem % g_sz;
-    o.r = o.mb / p.blocks_per_rank;
+    token_tile(o.mb, p.blocks_per_rank, p.S_loc, kBM, o.r, o.row0, o.valid);
     return o;
 }
 
@@ -220,7 +223,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) down_accumulate_kernel(const _
                         const int f0 = k * F_d + kb * kBK;
                         ctl->issued[ps.stage] = 1u + ps.phase;
                         mbar_arrive_expect_tx(bar, kStageBytes);
-                        load_kmajor(sa, &p.map_a, bar, f0, tl.mb * kBM, 0);
+                        load_kmajor(sa, &p.map_a, bar, f0, tl.row0, 0);
                         load_mnmajor(sb, &p.map_wd, bar, tl.nb * 256, f0, 0, 4);
                         ps.advance(p.stages);
                     }
@@ -263,20 +266,23 @@ __global__ void __launch_bounds__(kNumThreads, 1) down_accumulate_kernel(const _
             if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[buf]), acc_phase, w, kErrWaitTmemFull))) break;
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
-            __nv_bfloat16* out = p.Y + static_cast<size_t>(tl.mb * kBM + row) * p.H + tl.nb * 256;
+            const bool live = row < tl.valid;
+            __nv_bfloat16* out = p.Y + static_cast<size_t>(tl.row0 + row) * p.H + tl.nb * 256;
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {
                 uint32_t v[32];
                 tmem_ld32(t_row + c * 32, v);
                 tmem_ld_wait();
                 uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+                if (live) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    dst[q] = make_uint4(
-                        pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])),
-                        pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
-                        pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
-                        pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
+                    for (int q = 0; q < 4; ++q) {
+                        dst[q] = make_uint4(
+                            pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])),
+                            pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
+                            pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
+                            pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
+                    }
                 }
             }
             tc_fence_before_sync();

@@ -171,6 +171,15 @@ __global__ void wait_expiry_selftest_kernel(int* status, unsigned long long limi
     __syncthreads();
 }
 
+// Token tile `mt` when every rank owns S_loc consecutive rows cut into tiles of TM rows; the last tile of a rank may be
+// partial (its remaining rows belong to the next rank, or lie beyond the tensor, and are loaded but never stored).
+__device__ __forceinline__ void token_tile(int mt, int tiles_per_rank, int S_loc, int TM, int& r, int& row0, int& valid) {
+    r = mt / tiles_per_rank;
+    const int lt = mt - r * tiles_per_rank;
+    row0 = r * S_loc + lt * TM;
+    valid = min(TM, S_loc - lt * TM);
+}
+
 // ---- epilogue helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);

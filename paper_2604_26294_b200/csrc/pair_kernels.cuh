@@ -346,7 +346,7 @@ pair_wide_kernel(const __grid_constant__ typename Policy::Params p) {
 }
 
 // ---- store helpers ---------------------------------------------------------------------------------
-__device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t_row) {
+__device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t_row, bool live) {
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
         uint32_t v[32];
@@ -355,8 +355,10 @@ __device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-        st_global_256(out + c * 32, pk[0], pk[1], pk[2], pk[3], pk[4], pk[5], pk[6], pk[7]);
-        st_global_256(out + c * 32 + 16, pk[8], pk[9], pk[10], pk[11], pk[12], pk[13], pk[14], pk[15]);
+        if (live) {
+            st_global_256(out + c * 32, pk[0], pk[1], pk[2], pk[3], pk[4], pk[5], pk[6], pk[7]);
+            st_global_256(out + c * 32 + 16, pk[8], pk[9], pk[10], pk[11], pk[12], pk[13], pk[14], pk[15]);
+        }
     }
 }
 
@@ -375,7 +377,7 @@ struct PairGateUpPolicyT {
         const float* dA;      // [S, F] fp32 (backward only)
         __nv_bfloat16* dG;    // [S, F] (backward only)
         __nv_bfloat16* dU;    // [S, F] (backward only)
-        int S, H, F, D, F_d;
+        int S, H, F, D, F_d, S_loc;
         int m_tiles, tiles_per_rank, jl_blocks, band, shared_order;
         int act;              // gate activation
         int rank_indexed;     // staged mode: one ring step per launch; the weight tensors hold, at index r, the
@@ -385,7 +387,7 @@ struct PairGateUpPolicyT {
         unsigned long long timeout_ns;
     };
     struct Tile {
-        int mt, k, jl;
+        int mt, k, jl, row0, valid;
     };
     __device__ static __forceinline__ int outer(const Params&) { return 1; }
     __device__ static __forceinline__ int inner(const Params& p) { return p.H / kBK; }
@@ -408,18 +410,20 @@ struct PairGateUpPolicyT {
         Tile o;
         o.jl = rem / band_sz;
         o.mt = band_start + rem % band_sz;
-        const int r = o.mt / p.tiles_per_rank;
+        int r;
+        token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, r, o.row0, o.valid);
         o.k = p.rank_indexed ? r : (p.shared_order ? t : (r - t + p.D) % p.D);
         return o;
     }
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int k, int kb, uint32_t cta,
                                                 uint32_t sa, uint32_t sb, uint32_t bar) {
-        pair_load_kmajor(sa, &p.map_x, bar, kb * kBK, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sa, &p.map_x, bar, kb * kBK, tl.row0 + cta * 128, 0);
         pair_load_mnmajor(sb, cta == 0 ? &p.map_wg : &p.map_wu, bar, tl.jl * 128, kb * kBK, k, 2);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         // p.F is the row pitch of A: F in direct mode, F/D in staged mode (where the shard offset is dropped)
-        const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F +
+        const bool live = static_cast<int>(cta) * 128 + row < tl.valid;   // rows past the rank's end are not stored
+        const size_t off = static_cast<size_t>(tl.row0 + cta * 128 + row) * p.F +
                            (p.rank_indexed ? 0 : static_cast<size_t>(tl.k) * p.F_d) + tl.jl * 128;
         if constexpr (kMode == 0) {
             __nv_bfloat16* out = p.A + off;
@@ -436,10 +440,12 @@ struct PairGateUpPolicyT {
                     packed[i] = pack_bf16x2(gate_act(g0, p.act) * __uint_as_float(u[2 * i]),
                                             gate_act(g1, p.act) * __uint_as_float(u[2 * i + 1]));
                 }
-                st_global_256(out + c * 32, packed[0], packed[1], packed[2], packed[3], packed[4], packed[5], packed[6],
-                              packed[7]);
-                st_global_256(out + c * 32 + 16, packed[8], packed[9], packed[10], packed[11], packed[12], packed[13],
-                              packed[14], packed[15]);
+                if (live) {
+                    st_global_256(out + c * 32, packed[0], packed[1], packed[2], packed[3], packed[4], packed[5], packed[6],
+                                  packed[7]);
+                    st_global_256(out + c * 32 + 16, packed[8], packed[9], packed[10], packed[11], packed[12], packed[13],
+                                  packed[14], packed[15]);
+                }
             }
         } else if constexpr (kMode == 2) {
 #pragma unroll 1
@@ -466,17 +472,21 @@ struct PairGateUpPolicyT {
                     pp[i] = pack_bf16x2(vp[0], vp[1]);
                     pq[i] = pack_bf16x2(vq[0], vq[1]);
                 }
-                st_global_256(p.A + off + c * 16, pa[0], pa[1], pa[2], pa[3], pa[4], pa[5], pa[6], pa[7]);
-                st_global_256(p.dG + off + c * 16, pp[0], pp[1], pp[2], pp[3], pp[4], pp[5], pp[6], pp[7]);
-                st_global_256(p.dU + off + c * 16, pq[0], pq[1], pq[2], pq[3], pq[4], pq[5], pq[6], pq[7]);
+                if (live) {
+                    st_global_256(p.A + off + c * 16, pa[0], pa[1], pa[2], pa[3], pa[4], pa[5], pa[6], pa[7]);
+                    st_global_256(p.dG + off + c * 16, pp[0], pp[1], pp[2], pp[3], pp[4], pp[5], pp[6], pp[7]);
+                    st_global_256(p.dU + off + c * 16, pq[0], pq[1], pq[2], pq[3], pq[4], pq[5], pq[6], pq[7]);
+                }
             }
         } else {
             const float* da_row = p.dA + off;
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {
-                uint32_t da4[2][8];
-                ld_global_nc_256(da_row + c * 16, da4[0]);       // issued before the tensor-memory loads
-                ld_global_nc_256(da_row + c * 16 + 8, da4[1]);
+                uint32_t da4[2][8] = {};
+                if (live) {
+                    ld_global_nc_256(da_row + c * 16, da4[0]);       // issued before the tensor-memory loads
+                    ld_global_nc_256(da_row + c * 16 + 8, da4[1]);
+                }
                 uint32_t g[16], u[16];
                 tmem_ld16(t_row + c * 16, g);
                 tmem_ld16(t_row + 128 + c * 16, u);
@@ -500,9 +510,11 @@ struct PairGateUpPolicyT {
                     pg[i] = pack_bf16x2(vg[0], vg[1]);
                     pu[i] = pack_bf16x2(vu[0], vu[1]);
                 }
-                st_global_256(p.A + off + c * 16, pa[0], pa[1], pa[2], pa[3], pa[4], pa[5], pa[6], pa[7]);
-                st_global_256(p.dG + off + c * 16, pg[0], pg[1], pg[2], pg[3], pg[4], pg[5], pg[6], pg[7]);
-                st_global_256(p.dU + off + c * 16, pu[0], pu[1], pu[2], pu[3], pu[4], pu[5], pu[6], pu[7]);
+                if (live) {
+                    st_global_256(p.A + off + c * 16, pa[0], pa[1], pa[2], pa[3], pa[4], pa[5], pa[6], pa[7]);
+                    st_global_256(p.dG + off + c * 16, pg[0], pg[1], pg[2], pg[3], pg[4], pg[5], pg[6], pg[7]);
+                    st_global_256(p.dU + off + c * 16, pu[0], pu[1], pu[2], pu[3], pu[4], pu[5], pu[6], pu[7]);
+                }
             }
         }
     }
@@ -525,14 +537,14 @@ struct PairDaPolicyT {
         const __nv_bfloat16* Q;      // [S, F]
         __nv_bfloat16* dG;           // [S, F]
         __nv_bfloat16* dU;           // [S, F]
-        int S, H, F, D;
-        int m_tiles, j_tiles, band;
+        int S, H, F, D, S_loc;
+        int m_tiles, tiles_per_rank, j_tiles, band;
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
     };
     struct Tile {
-        int mt, jt;
+        int mt, jt, row0, valid;
     };
     __device__ static __forceinline__ int outer(const Params&) { return 1; }
     __device__ static __forceinline__ int inner(const Params& p) { return p.H / kBK; }
@@ -551,15 +563,18 @@ struct PairDaPolicyT {
         Tile o;
         o.jt = rem / band_sz;
         o.mt = band_start + rem % band_sz;
+        int r;
+        token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, r, o.row0, o.valid);
         return o;
     }
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int, int kb, uint32_t cta, uint32_t sa,
                                                 uint32_t sb, uint32_t bar) {
-        pair_load_kmajor(sa, &p.map_dy, bar, kb * kBK, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sa, &p.map_dy, bar, kb * kBK, tl.row0 + cta * 128, 0);
         pair_load_kmajor(sb, &p.map_wd, bar, kb * kBK, tl.jt * 256 + cta * 128, 0);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.F + tl.jt * 256;
+        const bool live = static_cast<int>(cta) * 128 + row < tl.valid;
+        const size_t off = static_cast<size_t>(tl.row0 + cta * 128 + row) * p.F + tl.jt * 256;
         if constexpr (!kSaved) {
             float* dst = p.dA + off;
 #pragma unroll 1
@@ -567,17 +582,21 @@ struct PairDaPolicyT {
                 uint32_t v[32];
                 tmem_ld32(t_row + c * 32, v);
                 tmem_ld_wait();
+                if (live) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    st_global_256(dst + c * 32 + q * 8, v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
-                                  v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
+                    for (int q = 0; q < 4; ++q)
+                        st_global_256(dst + c * 32 + q * 8, v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
+                                      v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
+                }
             }
         } else {
 #pragma unroll 1
             for (int c = 0; c < 16; ++c) {
-                uint32_t pr[8], qr[8], v[16];
-                ld_global_nc_256(p.P + off + c * 16, pr);   // 16 bf16 each, issued before the tensor-memory load
-                ld_global_nc_256(p.Q + off + c * 16, qr);
+                uint32_t pr[8] = {}, qr[8] = {}, v[16];
+                if (live) {
+                    ld_global_nc_256(p.P + off + c * 16, pr);   // 16 bf16 each, issued before the tensor-memory load
+                    ld_global_nc_256(p.Q + off + c * 16, qr);
+                }
                 tmem_ld16(t_row + c * 16, v);
                 tmem_ld_wait();
                 uint32_t og[8], ou[8];
@@ -590,8 +609,10 @@ struct PairDaPolicyT {
                     og[i] = pack_bf16x2(d0 * p0, d1 * p1);   // dG = dA * U * sigma'(G)
                     ou[i] = pack_bf16x2(d0 * q0, d1 * q1);   // dU = dA * sigma(G)
                 }
-                st_global_256(p.dG + off + c * 16, og[0], og[1], og[2], og[3], og[4], og[5], og[6], og[7]);
-                st_global_256(p.dU + off + c * 16, ou[0], ou[1], ou[2], ou[3], ou[4], ou[5], ou[6], ou[7]);
+                if (live) {
+                    st_global_256(p.dG + off + c * 16, og[0], og[1], og[2], og[3], og[4], og[5], og[6], og[7]);
+                    st_global_256(p.dU + off + c * 16, ou[0], ou[1], ou[2], ou[3], ou[4], ou[5], ou[6], ou[7]);
+                }
             }
         }
     }
@@ -605,7 +626,7 @@ struct PairDownPolicy {
     struct Params {
         CUtensorMap map_a, map_wd;  // boxes (64,128), (64,64)
         __nv_bfloat16* Y;
-        int S, H, F, D, F_d;
+        int S, H, F, D, F_d, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;   // mixed-width kernel: number of 256 x 512 tiles at the head of the tile list
         int num_tiles, stages;
@@ -613,7 +634,7 @@ struct PairDownPolicy {
         unsigned long long timeout_ns;
     };
     struct Tile {
-        int mt, nb, r, halves;
+        int mt, nb, r, halves, row0, valid;
     };
     __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
     __device__ static __forceinline__ int inner(const Params& p) { return p.F_d / kBK; }
@@ -637,35 +658,37 @@ struct PairDownPolicy {
         // token tiles are taken from the last to the first: the producer kernel wrote the last rows most recently,
         // so they are the ones still in L2
         o.mt = p.m_tiles - 1 - (g_start + rem % g_sz);
-        o.r = o.mt / p.tiles_per_rank;
+        token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
                                                 uint32_t sa, uint32_t sb, uint32_t bar) {
         const int f0 = k * p.F_d + i * kBK;
-        pair_load_kmajor(sa, &p.map_a, bar, f0, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sa, &p.map_a, bar, f0, tl.row0 + cta * 128, 0);
         pair_load_mnmajor(sb, &p.map_wd, bar, tl.nb * 256 + cta * 128, f0, 0, 2);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
+        store_bf16_row256(p.Y + static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + tl.nb * 256, t_row,
+                          static_cast<int>(cta) * 128 + row < tl.valid);
     }
     // mixed-width kernel: tl.nb is the first 256-column block, tl.halves the number of column blocks
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
         mixed_tile(t, p.wide_tiles, p.n_blocks, p.m_tiles, true, o.mt, o.nb, o.halves);
-        o.r = o.mt / p.tiles_per_rank;
+        token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }
     __device__ static __forceinline__ void load_wide(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
                                                      uint32_t sa, uint32_t sb, uint32_t bar) {
         const int f0 = k * p.F_d + i * kBK;
-        pair_load_kmajor(sa, &p.map_a, bar, f0, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sa, &p.map_a, bar, f0, tl.row0 + cta * 128, 0);
         for (int h = 0; h < tl.halves; ++h)
             pair_load_mnmajor(sb + h * 16384, &p.map_wd, bar, (tl.nb + h) * 256 + cta * 128, f0, 0, 2);
     }
     __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
                                                          uint32_t t_row, int h) {
-        store_bf16_row256(p.Y + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + (tl.nb + h) * 256, t_row);
+        store_bf16_row256(p.Y + static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + (tl.nb + h) * 256, t_row,
+                          static_cast<int>(cta) * 128 + row < tl.valid);
     }
 };
 
@@ -678,7 +701,7 @@ struct PairDownStagedPolicy {
         CUtensorMap map_a, map_wd;  // A_step (F/D, S, 1) box (64,128); Wd buffers (H, F/D, D) box (64,64)
         float* Yacc;                // [S, H] fp32
         __nv_bfloat16* Y;           // [S, H]
-        int S, H, F_d, D, mode;
+        int S, H, F_d, D, mode, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int num_tiles, stages;
         int* status;
@@ -703,21 +726,22 @@ struct PairDownStagedPolicy {
         // token tiles are taken from the last to the first: the producer kernel wrote the last rows most recently,
         // so they are the ones still in L2
         o.mt = p.m_tiles - 1 - (g_start + rem % g_sz);
-        o.r = o.mt / p.tiles_per_rank;
+        token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int r, int i, uint32_t cta, uint32_t sa,
                                                 uint32_t sb, uint32_t bar) {
-        pair_load_kmajor(sa, &p.map_a, bar, i * kBK, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sa, &p.map_a, bar, i * kBK, tl.row0 + cta * 128, 0);
         pair_load_mnmajor(sb, &p.map_wd, bar, tl.nb * 256 + cta * 128, i * kBK, r, 2);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        const size_t off = static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256;
+        const bool live = static_cast<int>(cta) * 128 + row < tl.valid;
+        const size_t off = static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + tl.nb * 256;
         float4* acc = reinterpret_cast<float4*>(p.Yacc + off);
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
-            float4 prev[8];
-            if (p.mode == 1 || p.mode == 2) {
+            float4 prev[8] = {};
+            if (live && (p.mode == 1 || p.mode == 2)) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q) prev[q] = acc[c * 8 + q];
             }
@@ -733,6 +757,7 @@ struct PairDownStagedPolicy {
                     f[4 * q] += prev[q].x; f[4 * q + 1] += prev[q].y; f[4 * q + 2] += prev[q].z; f[4 * q + 3] += prev[q].w;
                 }
             }
+            if (!live) continue;
             if (p.mode <= 1) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q) acc[c * 8 + q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
@@ -753,7 +778,7 @@ struct PairDxPolicy {
     struct Params {
         CUtensorMap map_dg, map_du, map_wg, map_wu;  // boxes (64,128) all
         __nv_bfloat16* dX;
-        int S, H, F, D, F_d;
+        int S, H, F, D, F_d, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;
         int num_tiles, stages;
@@ -784,23 +809,24 @@ struct PairDxPolicy {
         // token tiles are taken from the last to the first: the producer kernel wrote the last rows most recently,
         // so they are the ones still in L2
         o.mt = p.m_tiles - 1 - (g_start + rem % g_sz);
-        o.r = o.mt / p.tiles_per_rank;
+        token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
                                                 uint32_t sa, uint32_t sb, uint32_t bar) {
         const int j0 = (i >> 1) * kBK;
         const bool up = i & 1;
-        pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.row0 + cta * 128, 0);
         pair_load_kmajor(sb, up ? &p.map_wu : &p.map_wg, bar, j0, tl.nb * 256 + cta * 128, k);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        store_bf16_row256(p.dX + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + tl.nb * 256, t_row);
+        store_bf16_row256(p.dX + static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + tl.nb * 256, t_row,
+                          static_cast<int>(cta) * 128 + row < tl.valid);
     }
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
         mixed_tile(t, p.wide_tiles, p.n_blocks, p.m_tiles, true, o.mt, o.nb, o.halves);
-        o.r = o.mt / p.tiles_per_rank;
+        token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }
     __device__ static __forceinline__ void load_wide(const Params& p, const Tile& tl, int k, int i, uint32_t cta,
@@ -808,12 +834,13 @@ struct PairDxPolicy {
         const int j0 = (i >> 1) * kBK;
         const bool up = i & 1;
         const CUtensorMap* mw = up ? &p.map_wu : &p.map_wg;
-        pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.mt * 256 + cta * 128, 0);
+        pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.row0 + cta * 128, 0);
         for (int h = 0; h < tl.halves; ++h) pair_load_kmajor(sb + h * 16384, mw, bar, j0, (tl.nb + h) * 256 + cta * 128, k);
     }
     __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
                                                          uint32_t t_row, int h) {
-        store_bf16_row256(p.dX + static_cast<size_t>(tl.mt * 256 + cta * 128 + row) * p.H + (tl.nb + h) * 256, t_row);
+        store_bf16_row256(p.dX + static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + (tl.nb + h) * 256, t_row,
+                          static_cast<int>(cta) * 128 + row < tl.valid);
     }
 };
 
@@ -828,6 +855,7 @@ struct PairDwPolicy {
         int S, H, F, D, F_d, S_loc;
         int j_tiles, n_blocks, j_tiles_per_shard;
         int n_group;   // hidden blocks per group: their columns of X / dY stay in L2 while the [S,F] operand streams
+        int k_linear;  // 0, or ceil(S / 64) when the token contraction runs in ascending order (ragged ranks)
         int wide_tiles;
         int num_tiles, stages;
         int* status;
@@ -836,10 +864,13 @@ struct PairDwPolicy {
     struct Tile {
         int which, jt, nb, k, halves;
     };
-    __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
-    __device__ static __forceinline__ int inner(const Params& p) { return p.S_loc / kBK; }
-    // shard k meets the ranks in the order r = (k + t) mod D
+    // Tokens are contracted rank by rank in the order shard k meets the ranks, r = (k + t) mod D.  When the tokens per
+    // rank are not a multiple of the k-block (64) a k-block would straddle two ranks, so the tokens are then taken in
+    // plain ascending order, the tail k-block being zero-filled by the TMA unit (p.k_linear = number of k-blocks).
+    __device__ static __forceinline__ int outer(const Params& p) { return p.k_linear ? 1 : p.D; }
+    __device__ static __forceinline__ int inner(const Params& p) { return p.k_linear ? p.k_linear : p.S_loc / kBK; }
     __device__ static __forceinline__ int select(const Params& p, const Tile& tl, int t) {
+        if (p.k_linear) return 0;
         const int r = tl.k + t;
         return r >= p.D ? r - p.D : r;
     }

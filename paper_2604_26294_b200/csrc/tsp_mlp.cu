@@ -112,7 +112,7 @@ bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) ==
 tsp_status_t check_call(const tsp_mlp_plan_t* plan, int64_t S, int D) {
     if (!plan) return TSP_ERR_INVALID_ARG;
     if (D != plan->D || S <= 0) return TSP_ERR_INVALID_ARG;
-    if (S % D != 0 || (S / D) % 128 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (S % D != 0) return TSP_ERR_UNSUPPORTED_SHAPE;   // equal token shards; any number of tokens per rank
     if (S > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
     return TSP_OK;
 }
@@ -167,8 +167,9 @@ tsp_status_t launch_gate_up(tsp_mlp_plan_t* plan, const void* X, const void* Wg,
     if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
     p.A = static_cast<__nv_bfloat16*>(A);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
-    p.m_blocks = static_cast<int>(S / 128);
-    p.blocks_per_rank = static_cast<int>(S / D / 128);
+    p.S_loc = static_cast<int>(S / D);
+    p.blocks_per_rank = (p.S_loc + 127) / 128;
+    p.m_blocks = D * p.blocks_per_rank;
     p.jl_blocks = F_d / 128;
     p.band = 2 * gate_band(plan, (p.m_blocks + 1) / 2);   // same band, counted in 128-token blocks
     if (p.band > p.m_blocks) p.band = p.m_blocks;
@@ -196,9 +197,10 @@ tsp_status_t launch_down(tsp_mlp_plan_t* plan, const void* A, const void* Wd, vo
     if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 64)) return TSP_ERR_CUDA;
     p.Y = static_cast<__nv_bfloat16*>(Y);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
-    p.m_blocks = static_cast<int>(S / 128);
+    p.S_loc = static_cast<int>(S / D);
+    p.blocks_per_rank = (p.S_loc + 127) / 128;
+    p.m_blocks = D * p.blocks_per_rank;
     p.n_blocks = H / 256;
-    p.blocks_per_rank = static_cast<int>(S / D / 128);
     p.group = p.m_blocks < 16 ? p.m_blocks : 16;
     p.num_tiles = p.m_blocks * p.n_blocks;
     p.stages = pick_stages(plan, 48 * 1024, 4);
@@ -228,8 +230,9 @@ tsp_status_t launch_bwd_gate(tsp_mlp_plan_t* plan, const void* X, const void* Wg
     p.dG = static_cast<__nv_bfloat16*>(dG);
     p.dU = static_cast<__nv_bfloat16*>(dU);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
-    p.m_blocks = static_cast<int>(S / 128);
-    p.blocks_per_rank = static_cast<int>(S / D / 128);
+    p.S_loc = static_cast<int>(S / D);
+    p.blocks_per_rank = (p.S_loc + 127) / 128;
+    p.m_blocks = D * p.blocks_per_rank;
     p.jl_blocks = F_d / 128;
     p.band = 2 * gate_band(plan, (p.m_blocks + 1) / 2);
     if (p.band > p.m_blocks) p.band = p.m_blocks;
@@ -259,9 +262,10 @@ tsp_status_t launch_bwd_dx(tsp_mlp_plan_t* plan, const void* dG, const void* dU,
     if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 256)) return TSP_ERR_CUDA;
     p.dX = static_cast<__nv_bfloat16*>(dX);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
-    p.m_blocks = static_cast<int>(S / 128);
+    p.S_loc = static_cast<int>(S / D);
+    p.blocks_per_rank = (p.S_loc + 127) / 128;
+    p.m_blocks = D * p.blocks_per_rank;
     p.n_blocks = H / 256;
-    p.blocks_per_rank = static_cast<int>(S / D / 128);
     p.group = p.m_blocks < 16 ? p.m_blocks : 16;
     p.num_tiles = p.m_blocks * p.n_blocks;
     p.stages = pick_stages(plan, 48 * 1024, 4);
@@ -289,6 +293,7 @@ tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, 
     if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 64)) return TSP_ERR_CUDA;
     p.dWd = dWd; p.dWg = dWg; p.dWu = dWu;
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.k_linear = ((S / D) % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
     p.j_blocks = F / 128;
     p.n_blocks = H / 256;
     p.num_tiles = 3 * p.j_blocks * p.n_blocks;
@@ -378,8 +383,9 @@ tsp_status_t launch_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* W
     p.dU = static_cast<__nv_bfloat16*>(dU);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.F_d = F_d;
-    p.m_tiles = static_cast<int>(S / 256);
-    p.tiles_per_rank = static_cast<int>(S / D / 256);
+    p.S_loc = static_cast<int>(S / D);
+    p.tiles_per_rank = (p.S_loc + 255) / 256;
+    p.m_tiles = D * p.tiles_per_rank;
     p.jl_blocks = F_d / 128;
     p.band = gate_band(plan, p.m_tiles);
     p.shared_order = plan->shared_order;
@@ -409,7 +415,9 @@ tsp_status_t launch_da_pair_t(tsp_mlp_plan_t* plan, const void* dY, const void* 
     p.dG = static_cast<__nv_bfloat16*>(dG);
     p.dU = static_cast<__nv_bfloat16*>(dU);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
-    p.m_tiles = static_cast<int>(S / 256);
+    p.S_loc = static_cast<int>(S / D);
+    p.tiles_per_rank = (p.S_loc + 255) / 256;
+    p.m_tiles = D * p.tiles_per_rank;
     p.j_tiles = F / 256;
     p.band = gate_band(plan, p.m_tiles);
     fill_common(plan, p, p.m_tiles * p.j_tiles);
@@ -428,9 +436,10 @@ tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* W
     if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 64)) return TSP_ERR_CUDA;
     p.Y = static_cast<__nv_bfloat16*>(Y);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D; p.F_d = F / D;
-    p.m_tiles = static_cast<int>(S / 256);
+    p.S_loc = static_cast<int>(S / D);
+    p.tiles_per_rank = (p.S_loc + 255) / 256;
+    p.m_tiles = D * p.tiles_per_rank;
     p.n_blocks = H / 256;
-    p.tiles_per_rank = static_cast<int>(S / D / 256);
     const int group = plan->group > 0 ? plan->group : 8;
     p.group = p.m_tiles < group ? p.m_tiles : group;
     p.wide_tiles = mixed_wide_tiles(plan, 1, p.n_blocks, p.m_tiles * p.n_blocks, F / 64);
@@ -453,9 +462,10 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
     if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 128)) return TSP_ERR_CUDA;
     p.dX = static_cast<__nv_bfloat16*>(dX);
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D; p.F_d = F_d;
-    p.m_tiles = static_cast<int>(S / 256);
+    p.S_loc = static_cast<int>(S / D);
+    p.tiles_per_rank = (p.S_loc + 255) / 256;
+    p.m_tiles = D * p.tiles_per_rank;
     p.n_blocks = H / 256;
-    p.tiles_per_rank = static_cast<int>(S / D / 256);
     const int group = plan->dx_group > 0 ? plan->dx_group : 8;
     p.group = p.m_tiles < group ? p.m_tiles : group;
     p.wide_tiles = mixed_wide_tiles(plan, 2, p.n_blocks, p.m_tiles * p.n_blocks, 2 * F / 64);
@@ -481,6 +491,7 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.F_d = F / D;
     p.S_loc = static_cast<int>(S / D);
+    p.k_linear = (p.S_loc % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
     p.j_tiles = F / 256;
     p.j_tiles_per_shard = p.F_d / 256;
     p.n_blocks = H / 256;
@@ -497,7 +508,14 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDwPolicy>, p, stream);
 }
 
-bool pairs_for_tokens(const tsp_mlp_plan_t* plan, int64_t S) { return plan->use_pairs && (S / plan->D) % 256 == 0; }
+// CTA pairs work on 256-row token tiles, single CTAs on 128-row tiles; a rank's last tile is padded.  Pairs are the
+// faster kernels, so they are taken unless their padding costs clearly more rows than the single-CTA tiling.
+bool pairs_for_tokens(const tsp_mlp_plan_t* plan, int64_t S) {
+    if (!plan->use_pairs) return false;
+    const int64_t s_loc = S / plan->D;
+    const int64_t padded_pair = (s_loc + 255) / 256 * 256, padded_single = (s_loc + 127) / 128 * 128;
+    return padded_pair * 100 <= padded_single * 106;
+}
 bool pairs_for_dw(const tsp_mlp_plan_t* plan) { return plan->use_pairs && (plan->F / plan->D) % 256 == 0; }
 
 // ---------------------------------------------------------------------------------------------
@@ -764,7 +782,7 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
     if (!X || !Wg || !Wu || !Wd || !Y) return TSP_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned32(Y)) return TSP_ERR_INVALID_ARG;
     if (compute_stream == copy_stream) return TSP_ERR_INVALID_ARG;
-    if ((S / D) % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!pairs_for_tokens(plan, S)) return TSP_ERR_UNSUPPORTED_SHAPE;
     if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_staged(plan, S)) return TSP_ERR_WORKSPACE;
     cudaStream_t cs = static_cast<cudaStream_t>(compute_stream), xs = static_cast<cudaStream_t>(copy_stream);
     const int H = plan->H, F = plan->F, F_d = F / D;
@@ -829,8 +847,9 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
             if (!encode_sharded(plan, &p.map_wu, cur_u, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
             p.A = static_cast<__nv_bfloat16*>(A_step);
             p.S = static_cast<int>(S); p.H = H; p.F = F_d; p.D = D; p.F_d = F_d;
-            p.m_tiles = static_cast<int>(S / 256);
-            p.tiles_per_rank = static_cast<int>(S / D / 256);
+            p.S_loc = static_cast<int>(S / D);
+            p.tiles_per_rank = (p.S_loc + 255) / 256;
+            p.m_tiles = D * p.tiles_per_rank;
             p.jl_blocks = F_d / 128;
             p.band = gate_band(plan, p.m_tiles);
             p.rank_indexed = 1;
@@ -848,9 +867,10 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
             p.Y = static_cast<__nv_bfloat16*>(Y);
             p.S = static_cast<int>(S); p.H = H; p.F_d = F_d; p.D = D;
             p.mode = D == 1 ? 3 : (t == 0 ? 0 : (t == D - 1 ? 2 : 1));
-            p.m_tiles = static_cast<int>(S / 256);
+            p.S_loc = static_cast<int>(S / D);
+            p.tiles_per_rank = (p.S_loc + 255) / 256;
+            p.m_tiles = D * p.tiles_per_rank;
             p.n_blocks = H / 256;
-            p.tiles_per_rank = static_cast<int>(S / D / 256);
             const int group = plan->group > 0 ? plan->group : 8;
             p.group = p.m_tiles < group ? p.m_tiles : group;
             fill_common(plan, p, p.m_tiles * p.n_blocks);
@@ -877,7 +897,7 @@ size_t tsp_mlp_saved_bytes(const tsp_mlp_plan_t* plan, int64_t S) {
 }
 
 static tsp_status_t check_saved_shapes(const tsp_mlp_plan_t* plan, int64_t S) {
-    if (!plan->use_pairs || (S / plan->D) % 256 != 0 || plan->F % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!pairs_for_tokens(plan, S) || plan->F % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
     return TSP_OK;
 }
 
@@ -981,7 +1001,7 @@ tsp_status_t tsp_mlp_forward_static(int H, int F, int D, const void* X, const vo
                                     const void* Wd, void* Y, int64_t S, int* timed_out_host, void* cuda_stream) {
     if (H <= 0 || F <= 0 || D <= 0 || D > 64 || S <= 0) return TSP_ERR_INVALID_ARG;
     if (F % D != 0 || (F / D) % 128 != 0 || H % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
-    if (S % D != 0 || (S / D) % 128 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (S % D != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
     if (!X || !Wg || !Wu || !Wd || !Y) return TSP_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd) || !aligned16(Y)) return TSP_ERR_INVALID_ARG;
     // the intermediate must fit the fixed scratch: S * F bf16 elements

@@ -48,9 +48,9 @@ def test_forward_refuses_bad_calls_without_launching(plan):
     # misaligned workspace pointer
     assert lib.tsp_mlp_set_workspace(plan, ws.data_ptr() + 16, 1024) == b.TSP_ERR_INVALID_ARG
     b.tsp_mlp_set_workspace(plan, ws)
-    # D differs from the plan's; S not a multiple of 128 per rank; null and misaligned pointers
+    # D differs from the plan's; S not divisible into D equal token shards; null and misaligned pointers
     assert lib.tsp_mlp_forward(plan, *args, 256, 4, stream) == b.TSP_ERR_INVALID_ARG
-    assert lib.tsp_mlp_forward(plan, *args, 200, 2, stream) == b.TSP_ERR_UNSUPPORTED_SHAPE
+    assert lib.tsp_mlp_forward(plan, *args, 255, 2, stream) == b.TSP_ERR_UNSUPPORTED_SHAPE
     assert lib.tsp_mlp_forward(plan, *args, 0, 2, stream) == b.TSP_ERR_INVALID_ARG
     assert lib.tsp_mlp_forward(plan, None, *args[1:], 256, 2, stream) == b.TSP_ERR_INVALID_ARG
     assert lib.tsp_mlp_forward(plan, args[0] + 2, *args[1:], 256, 2, stream) == b.TSP_ERR_INVALID_ARG

@@ -54,6 +54,17 @@ def test_multi_tile_shapes_full_compare(S, H, F, D):
     _check_full(S, H, F, D, seed=1)
 
 
+@pytest.mark.parametrize("S,H,F,D", [
+    (80, 256, 256, 2),       # 40 tokens per rank
+    (600, 256, 768, 2),      # 300 tokens per rank: single-CTA path; dW contracts the tokens in ascending order
+    (2000, 256, 1024, 2),    # 1000 tokens per rank: CTA pairs, split backward, pair dW with a zero-filled tail k-block
+    (1536, 256, 768, 3),     # 512 per rank (control: multiple of every tile size)
+    (1304, 256, 512, 4),     # 326 tokens per rank
+])
+def test_ragged_token_counts_full_compare(S, H, F, D):
+    _check_full(S, H, F, D, seed=7)
+
+
 def test_wide_tiles_forced(monkeypatch):
     # 256 x 512 tiles for the down projection, dX and dW (normally chosen from the tile counts; forced here)
     monkeypatch.setenv("TSP_MLP_WIDE", "7")

@@ -47,6 +47,19 @@ def test_multi_tile_shapes_full_compare(S, H, F, D):
     _check_full(S, H, F, D, seed=1)
 
 
+@pytest.mark.parametrize("S,H,F,D", [
+    (80, 256, 256, 2),       # 40 tokens per rank: one partial 128-row tile per rank
+    (200, 256, 256, 1),      # 128 + 72 rows
+    (600, 256, 768, 2),      # 300 tokens per rank: single-CTA tiling, 44-row tail
+    (2000, 256, 1024, 2),    # 1000 tokens per rank: CTA pairs, 232-row tail tile
+    (3000, 512, 768, 3),     # three ranks of 1000 tokens
+    (1304, 256, 512, 4),     # 326 tokens per rank (not a multiple of 64 either)
+])
+def test_ragged_token_counts_full_compare(S, H, F, D):
+    # any number of tokens per rank: the last tile of a rank is loaded whole but only its valid rows are stored
+    _check_full(S, H, F, D, seed=7)
+
+
 def test_more_tiles_than_sms():
     # 20480 rows -> 160 token blocks > 148 SMs: persistent CTAs take a second tile (both TMEM buffers, phase flip)
     _check_full(20480, 256, 512, 4, seed=2)

@@ -50,7 +50,8 @@ def _as64(outs):
             inp.unshard_columns(tensor_to_f64(dWu)), inp.unshard_rows(tensor_to_f64(dWd)))
 
 
-@pytest.mark.parametrize("S,H,F,D", [(512, 256, 512, 2), (1536, 768, 1280, 2), (2048, 512, 2048, 4), (2304, 256, 1536, 3)])
+@pytest.mark.parametrize("S,H,F,D", [(512, 256, 512, 2), (1536, 768, 1280, 2), (2048, 512, 2048, 4), (2304, 256, 1536, 3),
+                                     (1500, 256, 768, 3)])   # the last one: 500 tokens per rank (ragged last tile)
 def test_stored_path_matches_oracle_and_recomputing_path(S, H, F, D):
     prob = DeviceProblem(S, H, F, D, seed=41, with_dy=True)
     got = _as64(_run_saved(prob))

@@ -41,7 +41,8 @@ def _staged(prob):
     return Y, ws
 
 
-@pytest.mark.parametrize("S,H,F,D", [(256, 256, 256, 1), (512, 256, 512, 2), (1024, 512, 1536, 4), (2048, 256, 1024, 8)])
+@pytest.mark.parametrize("S,H,F,D", [(256, 256, 256, 1), (512, 256, 512, 2), (1024, 512, 1536, 4), (2048, 256, 1024, 8),
+                                     (2000, 256, 512, 2)])   # the last one: 1000 tokens per rank (ragged last tile)
 def test_staged_forward_matches_oracle_and_direct(S, H, F, D):
     prob = DeviceProblem(S, H, F, D, seed=21)
     Y, ws = _staged(prob)
@@ -78,7 +79,7 @@ def test_receive_buffers_hold_the_ring_rotated_shards():
 def test_staged_refuses_one_stream_and_odd_shapes():
     import torch
 
-    prob = DeviceProblem(256, 256, 768, 2, seed=0)    # 128 tokens per rank: below the 256-row pair tile
+    prob = DeviceProblem(256, 256, 768, 2, seed=0)    # 128 tokens per rank: the single-CTA kernels' territory
     plan = b.tsp_mlp_plan(256, 768, 2)
     try:
         ws = torch.empty(b.tsp_mlp_workspace_bytes_staged(plan, 256), dtype=torch.uint8, device="cuda")

@@ -72,7 +72,7 @@ def test_static_forward_refuses_what_does_not_fit():
         b.tsp_mlp_forward_static(H, F, D, x, x, x, x, x, S)
     assert err.value.code == b.TSP_ERR_STATIC_LIMIT
     assert "fixed scratch" in str(err.value)
-    # shape rules still come first
+    # shape rules still come first (101 tokens cannot be split into 2 equal shards)
     with pytest.raises(b.TspError) as err:
-        b.tsp_mlp_forward_static(H, F, D, x, x, x, x, x, 100)
+        b.tsp_mlp_forward_static(H, F, D, x, x, x, x, x, 101)
     assert err.value.code == b.TSP_ERR_UNSUPPORTED_SHAPE
