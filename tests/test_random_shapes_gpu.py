@@ -1,7 +1,7 @@
 """Seeded sweep over legal shapes: every path the shape allows (forward, recomputing backward, stored-activation
 backward, staged forward) against the fp64 oracle.  The shapes are drawn once from a fixed seed so the test is
 deterministic; they mix odd shard counts, tile counts that do not divide the band / group sizes, one and several
-k-blocks per shard, and both kernel families (128 or 256 tokens per rank decide single CTA vs CTA pairs)."""
+k-blocks per shard, ragged token counts per rank, and both kernel families (single CTA vs CTA pairs)."""
 import numpy as np
 import pytest
 
@@ -19,9 +19,9 @@ TOL = 1e-2
 def _shapes():
     rng = np.random.default_rng(20260426)
     out = []
-    while len(out) < 14:
+    while len(out) < 18:
         D = int(rng.choice([1, 2, 3, 4, 5, 6, 8]))
-        s_loc = int(rng.choice([128, 256, 384, 512, 768]))
+        s_loc = int(rng.choice([72, 128, 200, 256, 384, 500, 512, 768, 1000]))
         H = int(rng.choice([256, 512, 768, 1024]))
         f_d = int(rng.choice([128, 256, 384, 512, 640]))
         S, F = D * s_loc, D * f_d
@@ -60,7 +60,8 @@ def test_every_available_path_matches_the_oracle(S, H, F, D):
                         inp.unshard_rows(tensor_to_f64(dWd))), gref):
         check(n, g, r)
 
-    pair_tokens = (S // D) % 256 == 0
+    s_loc = S // D
+    pair_tokens = ((s_loc + 255) // 256 * 256) * 100 <= ((s_loc + 127) // 128 * 128) * 106   # the library's own rule
     plan = b.tsp_mlp_plan(H, F, D)
     try:
         if pair_tokens:
