@@ -218,7 +218,10 @@ __global__ void __launch_bounds__(kNumThreads, 1) tile_gemm_kernel(const __grid_
     cta_setup(ctl, p.stages, 2, kEpilogueThreads);
     const uint32_t tmem_base = ctl->tmem_base;
     WaitCtx w{&ctl->abort, p.status, p.timeout_ns};
-    const int k_blocks = Policy::k_blocks(p);
+    // The K loop is outer() x inner() k-blocks; the shard (or rank) of an outer step is chosen once, so the producer's
+    // per-k-block path has no integer division.
+    const int n_outer = Policy::outer(p), n_inner = Policy::inner(p);
+    const int k_blocks = n_outer * n_inner;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -227,14 +230,17 @@ __global__ void __launch_bounds__(kNumThreads, 1) tile_gemm_kernel(const __grid_
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
                 const typename Policy::Tile tl = Policy::decode(p, tile);
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!(ok = wait_bar(smem_u32(&ctl->empty[ps.stage]), ps.phase ^ 1u, w, kErrWaitEmpty))) break;
-                    const uint32_t bar = smem_u32(&ctl->full[ps.stage]);
-                    const uint32_t sa = smem_base + ps.stage * kStageBytes, sb = sa + kABytes;
-                    ctl->issued[ps.stage] = 1u + ps.phase;
-                    mbar_arrive_expect_tx(bar, kStageBytes);
-                    Policy::load(p, tl, kb, sa, sb, bar);
-                    ps.advance(p.stages);
+                for (int o = 0; o < n_outer && ok; ++o) {
+                    const int sel = Policy::select(p, tl, o);
+                    for (int i = 0; i < n_inner; ++i) {
+                        if (!(ok = wait_bar(smem_u32(&ctl->empty[ps.stage]), ps.phase ^ 1u, w, kErrWaitEmpty))) break;
+                        const uint32_t bar = smem_u32(&ctl->full[ps.stage]);
+                        const uint32_t sa = smem_base + ps.stage * kStageBytes, sb = sa + kABytes;
+                        ctl->issued[ps.stage] = 1u + ps.phase;
+                        mbar_arrive_expect_tx(bar, kStageBytes);
+                        Policy::load(p, tl, sel, i, sa, sb, bar);
+                        ps.advance(p.stages);
+                    }
                 }
             }
         }
@@ -294,7 +300,7 @@ struct BwdDxPolicy {
         CUtensorMap map_wg;  // Wg (F/D, H, D)   box (64, 256)   K-major B operand (rows = hidden index)
         CUtensorMap map_wu;  // Wu likewise
         __nv_bfloat16* dX;   // [S, H]
-        int S, H, F, D, S_loc;
+        int S, H, F, D, S_loc, F_d;
         int m_blocks, n_blocks, blocks_per_rank, group, num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -302,7 +308,13 @@ struct BwdDxPolicy {
     struct Tile {
         int mb, nb, r, row0, valid;
     };
-    __device__ static __forceinline__ int k_blocks(const Params& p) { return 2 * (p.F / kBK); }
+    __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
+    __device__ static __forceinline__ int inner(const Params& p) { return 2 * (p.F_d / kBK); }
+    // shard held at ring step t: k = (r - t) mod D
+    __device__ static __forceinline__ int select(const Params& p, const Tile& tl, int t) {
+        const int k = tl.r - t;
+        return k < 0 ? k + p.D : k;
+    }
     __device__ static __forceinline__ void prefetch(const Params& p) {
         tma_prefetch_desc(&p.map_dg);
         tma_prefetch_desc(&p.map_du);
@@ -322,16 +334,11 @@ struct BwdDxPolicy {
         return o;
     }
     // k-block order: ring step t -> shard k = (r - t) mod D -> 64-wide slice of the shard -> (dG Wg^T, dU Wu^T)
-    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int kb, uint32_t sa, uint32_t sb,
+    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int k, int i, uint32_t sa, uint32_t sb,
                                                 uint32_t bar) {
-        const int F_d = p.F / p.D;
-        const int per_shard = 2 * (F_d / kBK);
-        const int t = kb / per_shard;
-        const int rem = kb - t * per_shard;
-        const int k = (tl.r - t + p.D) % p.D;
-        const int j0 = (rem >> 1) * kBK;
-        const bool up = rem & 1;
-        load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * F_d + j0, tl.row0, 0);
+        const int j0 = (i >> 1) * kBK;
+        const bool up = i & 1;
+        load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.row0, 0);
         load_kmajor(sb, up ? &p.map_wu : &p.map_wg, bar, j0, tl.nb * 256, k);
     }
     __device__ static __forceinline__ void store(const Params& p, const Tile& tl, int row, int c, const uint32_t (&v)[32]) {
@@ -363,7 +370,7 @@ struct BwdDwPolicy {
         float* dWd;          // [D][F/D][H] = [F][H]
         float* dWg;          // [D][H][F/D]
         float* dWu;          // [D][H][F/D]
-        int S, H, F, D;
+        int S, H, F, D, S_loc;
         int k_linear;        // 0, or ceil(S / 64) when the tokens are contracted in ascending order (ragged ranks)
         int j_blocks, n_blocks, num_tiles, stages;
         int* status;
@@ -372,7 +379,14 @@ struct BwdDwPolicy {
     struct Tile {
         int which, jb, nb, k;
     };
-    __device__ static __forceinline__ int k_blocks(const Params& p) { return p.k_linear ? p.k_linear : p.S / kBK; }
+    // rank order r = (k + t) mod D; ascending token order when a 64-token k-block would straddle two ranks
+    __device__ static __forceinline__ int outer(const Params& p) { return p.k_linear ? 1 : p.D; }
+    __device__ static __forceinline__ int inner(const Params& p) { return p.k_linear ? p.k_linear : p.S_loc / kBK; }
+    __device__ static __forceinline__ int select(const Params& p, const Tile& tl, int t) {
+        if (p.k_linear) return 0;
+        const int r = tl.k + t;
+        return r >= p.D ? r - p.D : r;
+    }
     __device__ static __forceinline__ void prefetch(const Params& p) {
         tma_prefetch_desc(&p.map_a);
         tma_prefetch_desc(&p.map_dg);
@@ -390,19 +404,9 @@ struct BwdDwPolicy {
         o.k = o.jb / ((p.F / p.D) / 128);
         return o;
     }
-    // token order: shard k meets the ranks in the order r = (k + t) mod D
-    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int kb, uint32_t sa, uint32_t sb,
+    __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int r, int i, uint32_t sa, uint32_t sb,
                                                 uint32_t bar) {
-        int s0;
-        if (p.k_linear) {   // ragged ranks: ascending token order, the tail k-block is zero-filled by the TMA unit
-            s0 = kb * kBK;
-        } else {
-            const int S_loc = p.S / p.D;
-            const int per_rank = S_loc / kBK;
-            const int t = kb / per_rank;
-            const int r = (tl.k + t) % p.D;
-            s0 = r * S_loc + (kb - t * per_rank) * kBK;
-        }
+        const int s0 = r * p.S_loc + i * kBK;
         const CUtensorMap* ma = tl.which == 0 ? &p.map_a : (tl.which == 1 ? &p.map_dg : &p.map_du);
         const CUtensorMap* mb = tl.which == 0 ? &p.map_dy : &p.map_x;
         load_mnmajor(sa, ma, bar, tl.jb * 128, s0, 0, 2);

@@ -261,7 +261,7 @@ tsp_status_t launch_bwd_dx(tsp_mlp_plan_t* plan, const void* dG, const void* dU,
     if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 256)) return TSP_ERR_CUDA;
     if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 256)) return TSP_ERR_CUDA;
     p.dX = static_cast<__nv_bfloat16*>(dX);
-    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D; p.F_d = F_d;
     p.S_loc = static_cast<int>(S / D);
     p.blocks_per_rank = (p.S_loc + 127) / 128;
     p.m_blocks = D * p.blocks_per_rank;
@@ -293,7 +293,8 @@ tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, 
     if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 64)) return TSP_ERR_CUDA;
     p.dWd = dWd; p.dWg = dWg; p.dWu = dWu;
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
-    p.k_linear = ((S / D) % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
+    p.S_loc = static_cast<int>(S / D);
+    p.k_linear = (p.S_loc % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
     p.j_blocks = F / 128;
     p.n_blocks = H / 256;
     p.num_tiles = 3 * p.j_blocks * p.n_blocks;
