@@ -496,8 +496,9 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     p.j_tiles = F / 256;
     p.j_tiles_per_shard = p.F_d / 256;
     p.n_blocks = H / 256;
-    // hidden blocks are taken in groups whose columns of X / dY (S * 512 bytes per block) fit in about 32 MB of L2
-    int n_group = plan->dw_group > 0 ? plan->dw_group : static_cast<int>((32ull << 20) / (512ull * static_cast<size_t>(S)));
+    // hidden blocks are taken in groups whose columns of X / dY (S * 512 bytes per block) take about 64 MB (measured:
+    // DRAM reads of the dW kernel at S = 8192 are 8.9 / 7.2 / 4.4 / 4.1 GB for groups of 2 / 4 / 8 / 16 blocks)
+    int n_group = plan->dw_group > 0 ? plan->dw_group : static_cast<int>((64ull << 20) / (512ull * static_cast<size_t>(S)));
     if (n_group < 1) n_group = 1;
     p.wide_tiles = mixed_wide_tiles(plan, 4, p.n_blocks, 3 * p.j_tiles * p.n_blocks, static_cast<int>(S / 64));
     if (p.wide_tiles > 0) {
