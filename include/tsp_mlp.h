@@ -170,6 +170,53 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
                                     void* copy_stream);
 
 /*
+ * tsp_mlp_ring_step - ONE step of Algorithm 2 on ONE rank's data: what rank p runs between the
+ * AsyncRingSendRecv and the Wait of ring step t, when every rank has a GPU of its own and the weight shards
+ * really travel (the caller moves them: NCCL send / receive or peer copies on a communication stream).
+ *   t = 0:        Yacc  = (act(X_p Wg_k) * (X_p Wu_k)) Wd_k         (the "Y <- 0" of the algorithm is folded in)
+ *   0 < t < D-1:  Yacc += ...
+ *   t = D-1:      Y_p   = bf16(Yacc + ...)                          (D = 1: Y_p = bf16(...) directly)
+ * X_p, Y_p: [S_loc, H] bf16 (this rank's tokens only); Wg_k, Wu_k: [H, F/D] bf16 and Wd_k: [F/D, H] bf16, the
+ * shard the rank holds at this step (k = (p - t) mod D when the caller follows the ring; the kernels do not
+ * care which).  The fp32 accumulator Yacc [S_loc, H] and the bf16 scratch A [S_loc, F/D] live in the plan's
+ * workspace (tsp_mlp_workspace_bytes_ring(plan, S_loc, TSP_WS_FORWARD) bytes) and carry the state from step to
+ * step, so the D calls of one forward pass must use the same plan, workspace and S_loc, in the order t = 0..D-1 on
+ * one stream (or otherwise ordered).  Two kernels per call (gate|up with the activation epilogue; down projection
+ * of the shard added to the accumulator).  Any S_loc >= 1.  The result equals tsp_mlp_forward_staged's
+ * rows of rank p bit for bit (same kernels, same summation order).
+ * Errors: INVALID_ARG (null / misaligned pointer, t outside [0, D), D not the plan's), UNSUPPORTED_SHAPE
+ * (S_loc < 1 or > 2^24), WORKSPACE.
+ */
+size_t tsp_mlp_workspace_bytes_ring(const tsp_mlp_plan_t* plan, int64_t S_loc, int pass);
+tsp_status_t tsp_mlp_ring_step(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
+                               const void* Wd_k, void* Y_p, int64_t S_loc, int t, int D, void* cuda_stream);
+
+/*
+ * Backward pass of one ring step on one rank's data (the backward mirrors the forward weight movement, and the
+ * partial weight gradients the ranks produce for a shard are summed to its owner: Sections 4.3.4 and 4.7).  Split
+ * in two calls so that the caller can let a travelling dW accumulator arrive while the first call computes:
+ *
+ * tsp_mlp_ring_step_backward_dx: with the shard (Wg_k, Wu_k, Wd_k) held at step t and this rank's X_p, dY_p
+ *   [S_loc, H] bf16: recomputes G, U; dA = dY_p Wd_k^T (fp32); A, dG, dU (bf16, left in the workspace for the dW
+ *   call); dXacc (+)= dG Wg_k^T + dU Wu_k^T, with the fp32 partial sum carried in the workspace from t = 0 to
+ *   t = D-1, where dX_p [S_loc, H] is stored in bf16 (D = 1: stored directly).  Three kernels.
+ * tsp_mlp_ring_step_backward_dw: from the A, dG, dU the preceding _dx call left: this rank's contribution to the
+ *   shard's weight gradients, dWd_k (+)= A^T dY_p [F/D, H], dWg_k (+)= X_p^T dG, dWu_k (+)= X_p^T dU [H, F/D], fp32.
+ *   accumulate = 0 overwrites (the owner's own contribution, or a partial to be reduced by the caller),
+ *   accumulate = 1 adds to what the buffers hold (an accumulator that travels with the shard: the sum then runs
+ *   over the ranks in the order the shard meets them, r = (k + t) mod D).  One kernel.
+ * Both need (F/D) % 256 == 0 and the workspace of tsp_mlp_workspace_bytes_ring(plan, S_loc, TSP_WS_BACKWARD);
+ * calls of one backward pass go t = 0..D-1, _dx before _dw within a step, ordered on the GPU.
+ * Errors as for tsp_mlp_ring_step; UNSUPPORTED_SHAPE also when (F/D) % 256 != 0.
+ */
+tsp_status_t tsp_mlp_ring_step_backward_dx(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
+                                           const void* Wd_k, const void* dY_p, void* dX_p, int64_t S_loc, int t, int D,
+                                           void* cuda_stream);
+tsp_status_t tsp_mlp_ring_step_backward_dw(tsp_mlp_plan_t* plan, const void* X_p, const void* dY_p, float* dWg_k,
+                                           float* dWu_k, float* dWd_k, int64_t S_loc, int accumulate, int D,
+                                           void* cuda_stream);
+
+/*
  * tsp_mlp_forward_static - the forward pass for callers that cannot obtain device memory at call time.
  * (The paper has no counterpart of this entry point; it exists for integration reasons only.)
  *

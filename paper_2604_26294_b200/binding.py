@@ -44,6 +44,12 @@ SIGNATURES = {
     "tsp_mlp_backward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_mlp_workspace_bytes_staged": (ctypes.c_size_t, [_P, ctypes.c_int64]),
     "tsp_mlp_forward_staged": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P, _P]),
+    "tsp_mlp_workspace_bytes_ring": (ctypes.c_size_t, [_P, ctypes.c_int64, ctypes.c_int]),
+    "tsp_mlp_ring_step_backward_dx": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                                     _P]),
+    "tsp_mlp_ring_step_backward_dw": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                                     _P]),
+    "tsp_mlp_ring_step": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_forward_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, _P,
                                               ctypes.c_int64, ctypes.POINTER(ctypes.c_int), _P]),
     "tsp_mlp_selftest_wait_expiry": (ctypes.c_int, [_P, ctypes.c_int, _P]),
@@ -178,6 +184,31 @@ def tsp_mlp_forward_staged(plan, X, Wg, Wu, Wd, Y, S: int, D: int, compute_strea
     _check(load_library().tsp_mlp_forward_staged(plan, _ptr(X), _ptr(Wg), _ptr(Wu), _ptr(Wd), _ptr(Y), S, D,
                                                  _stream_handle(compute_stream), _stream_handle(copy_stream)),
            "tsp_mlp_forward_staged", plan)
+
+
+def tsp_mlp_workspace_bytes_ring(plan, S_loc: int, backward: int = TSP_WS_FORWARD) -> int:
+    return int(load_library().tsp_mlp_workspace_bytes_ring(plan, S_loc, backward))
+
+
+def tsp_mlp_ring_step(plan, X_p, Wg_k, Wu_k, Wd_k, Y_p, S_loc: int, t: int, D: int, stream=None) -> None:
+    """One ring step of Algorithm 2 on one rank's tokens and the one shard it holds at step t."""
+    _check(load_library().tsp_mlp_ring_step(plan, _ptr(X_p), _ptr(Wg_k), _ptr(Wu_k), _ptr(Wd_k), _ptr(Y_p), S_loc, t, D,
+                                            _stream_handle(stream)), "tsp_mlp_ring_step", plan)
+
+
+def tsp_mlp_ring_step_backward_dx(plan, X_p, Wg_k, Wu_k, Wd_k, dY_p, dX_p, S_loc: int, t: int, D: int, stream=None) -> None:
+    """Backward of one ring step, first part: A, dG, dU into the workspace and the carried dX sum."""
+    _check(load_library().tsp_mlp_ring_step_backward_dx(plan, _ptr(X_p), _ptr(Wg_k), _ptr(Wu_k), _ptr(Wd_k), _ptr(dY_p),
+                                                        _ptr(dX_p), S_loc, t, D, _stream_handle(stream)),
+           "tsp_mlp_ring_step_backward_dx", plan)
+
+
+def tsp_mlp_ring_step_backward_dw(plan, X_p, dY_p, dWg_k, dWu_k, dWd_k, S_loc: int, accumulate: int, D: int,
+                                  stream=None) -> None:
+    """Backward of one ring step, second part: this rank's contribution to the held shard's weight gradients."""
+    _check(load_library().tsp_mlp_ring_step_backward_dw(plan, _ptr(X_p), _ptr(dY_p), _ptr(dWg_k), _ptr(dWu_k),
+                                                        _ptr(dWd_k), S_loc, accumulate, D, _stream_handle(stream)),
+           "tsp_mlp_ring_step_backward_dw", plan)
 
 
 def tsp_mlp_forward_static(H: int, F: int, D: int, X, Wg, Wu, Wd, Y, S: int, timed_out=None, stream=None) -> None:

@@ -362,6 +362,45 @@ __device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t
     }
 }
 
+// One accumulator row of 256 columns whose sum is carried from launch to launch in an fp32 buffer (one ring step per
+// launch): add_prev reads the carried value and adds it, to_fp32 writes the new partial sum back, otherwise the row is
+// rounded once to bf16 into `out`.  Rows that are not live only drain tensor memory.
+__device__ __forceinline__ void carry_row256(float* acc_row, __nv_bfloat16* out, uint32_t t_row, bool live, bool add_prev,
+                                             bool to_fp32) {
+    float4* acc = reinterpret_cast<float4*>(acc_row);
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+        float4 prev[8] = {};
+        if (live && add_prev) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) prev[q] = acc[c * 8 + q];
+        }
+        uint32_t v[32];
+        tmem_ld32(t_row + c * 32, v);
+        tmem_ld_wait();
+        float f[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
+        if (add_prev) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                f[4 * q] += prev[q].x; f[4 * q + 1] += prev[q].y; f[4 * q + 2] += prev[q].z; f[4 * q + 3] += prev[q].w;
+            }
+        }
+        if (!live) continue;
+        if (to_fp32) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[c * 8 + q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+        } else {
+            uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                dst[q] = make_uint4(pack_bf16x2(f[8 * q], f[8 * q + 1]), pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
+                                    pack_bf16x2(f[8 * q + 4], f[8 * q + 5]), pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+        }
+    }
+}
+
 // ---- gate | up + SwiGLU: tile = 256 tokens x 128 intermediate columns; CTA 0 loads the Wg half of B, CTA 1 the Wu half.
 // kMode 0 (forward)            : epilogue writes A = sigma(G) * U.
 // kMode 1 (backward, recompute): epilogue also reads dA (fp32, from the dA GEMM) and writes A, dG = dA*U*sigma'(G),
@@ -737,38 +776,7 @@ struct PairDownStagedPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         const bool live = static_cast<int>(cta) * 128 + row < tl.valid;
         const size_t off = static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + tl.nb * 256;
-        float4* acc = reinterpret_cast<float4*>(p.Yacc + off);
-#pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
-            float4 prev[8] = {};
-            if (live && (p.mode == 1 || p.mode == 2)) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q) prev[q] = acc[c * 8 + q];
-            }
-            uint32_t v[32];
-            tmem_ld32(t_row + c * 32, v);
-            tmem_ld_wait();
-            float f[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
-            if (p.mode == 1 || p.mode == 2) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    f[4 * q] += prev[q].x; f[4 * q + 1] += prev[q].y; f[4 * q + 2] += prev[q].z; f[4 * q + 3] += prev[q].w;
-                }
-            }
-            if (!live) continue;
-            if (p.mode <= 1) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc[c * 8 + q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
-            } else {
-                uint4* dst = reinterpret_cast<uint4*>(p.Y + off + c * 32);
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    dst[q] = make_uint4(pack_bf16x2(f[8 * q], f[8 * q + 1]), pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
-                                        pack_bf16x2(f[8 * q + 4], f[8 * q + 5]), pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
-            }
-        }
+        carry_row256(p.Yacc + off, p.Y + off, t_row, live, p.mode == 1 || p.mode == 2, p.mode <= 1);
     }
 };
 
@@ -778,6 +786,8 @@ struct PairDxPolicy {
     struct Params {
         CUtensorMap map_dg, map_du, map_wg, map_wu;  // boxes (64,128) all
         __nv_bfloat16* dX;
+        float* dXacc;  // [S, H] fp32 partial sums carried between launches (one ring step per launch), or null
+        int carry;     // 0: the launch covers all shards, dX stored directly; 1 first, 2 middle, 3 last step of a carried sum
         int S, H, F, D, F_d, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;
@@ -819,9 +829,15 @@ struct PairDxPolicy {
         pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.row0 + cta * 128, 0);
         pair_load_kmajor(sb, up ? &p.map_wu : &p.map_wg, bar, j0, tl.nb * 256 + cta * 128, k);
     }
+    __device__ static __forceinline__ void store_block(const Params& p, const Tile& tl, uint32_t cta, int row,
+                                                       uint32_t t_row, int nb) {
+        const size_t off = static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + nb * 256;
+        const bool live = static_cast<int>(cta) * 128 + row < tl.valid;
+        if (p.carry == 0) store_bf16_row256(p.dX + off, t_row, live);
+        else carry_row256(p.dXacc + off, p.dX + off, t_row, live, p.carry >= 2, p.carry <= 2);
+    }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
-        store_bf16_row256(p.dX + static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + tl.nb * 256, t_row,
-                          static_cast<int>(cta) * 128 + row < tl.valid);
+        store_block(p, tl, cta, row, t_row, tl.nb);
     }
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
@@ -839,8 +855,7 @@ struct PairDxPolicy {
     }
     __device__ static __forceinline__ void epilogue_half(const Params& p, const Tile& tl, uint32_t cta, int row,
                                                          uint32_t t_row, int h) {
-        store_bf16_row256(p.dX + static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + (tl.nb + h) * 256, t_row,
-                          static_cast<int>(cta) * 128 + row < tl.valid);
+        store_block(p, tl, cta, row, t_row, tl.nb + h);
     }
 };
 
@@ -856,6 +871,7 @@ struct PairDwPolicy {
         int j_tiles, n_blocks, j_tiles_per_shard;
         int n_group;   // hidden blocks per group: their columns of X / dY stay in L2 while the [S,F] operand streams
         int k_linear;  // 0, or ceil(S / 64) when the token contraction runs in ascending order (ragged ranks)
+        int accumulate;  // 0: dW overwritten; 1: the tile's sum is added to what dW holds (partial sums of other ranks)
         int wide_tiles;
         int num_tiles, stages;
         int* status;
@@ -918,6 +934,16 @@ struct PairDwPolicy {
             const int h0 = h_base + c * 32;
             if (tl.which == 0) {
                 float* dst = p.dWd + static_cast<size_t>(j) * p.H + h0;
+                if (p.accumulate) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 prev = *reinterpret_cast<const float4*>(dst + q * 4);
+                        v[4 * q] = __float_as_uint(__uint_as_float(v[4 * q]) + prev.x);
+                        v[4 * q + 1] = __float_as_uint(__uint_as_float(v[4 * q + 1]) + prev.y);
+                        v[4 * q + 2] = __float_as_uint(__uint_as_float(v[4 * q + 2]) + prev.z);
+                        v[4 * q + 3] = __float_as_uint(__uint_as_float(v[4 * q + 3]) + prev.w);
+                    }
+                }
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     st_global_256(dst + q * 8, v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4], v[8 * q + 5],
@@ -925,7 +951,10 @@ struct PairDwPolicy {
             } else {
                 float* base = (tl.which == 1 ? p.dWg : p.dWu) + static_cast<size_t>(tl.k) * p.H * F_d + (j - tl.k * F_d);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) base[static_cast<size_t>(h0 + i) * F_d] = __uint_as_float(v[i]);
+                for (int i = 0; i < 32; ++i) {
+                    float* dst = base + static_cast<size_t>(h0 + i) * F_d;
+                    *dst = p.accumulate ? __uint_as_float(v[i]) + *dst : __uint_as_float(v[i]);
+                }
             }
         }
     }

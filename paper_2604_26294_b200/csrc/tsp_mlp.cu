@@ -453,7 +453,7 @@ tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* W
 }
 
 tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void* dU, const void* Wg, const void* Wu,
-                                void* dX, int64_t S, cudaStream_t stream) {
+                                void* dX, int64_t S, cudaStream_t stream, float* dXacc = nullptr, int carry = 0) {
     const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
     tsp::PairDxPolicy::Params p;
     std::memset(&p, 0, sizeof(p));
@@ -462,6 +462,8 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
     if (!encode_sharded(plan, &p.map_wg, Wg, D, H, F_d, 64, 128)) return TSP_ERR_CUDA;
     if (!encode_sharded(plan, &p.map_wu, Wu, D, H, F_d, 64, 128)) return TSP_ERR_CUDA;
     p.dX = static_cast<__nv_bfloat16*>(dX);
+    p.dXacc = dXacc;
+    p.carry = carry;
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D; p.F_d = F_d;
     p.S_loc = static_cast<int>(S / D);
     p.tiles_per_rank = (p.S_loc + 255) / 256;
@@ -479,7 +481,8 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
 }
 
 tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
-                                const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream) {
+                                const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream,
+                                int accumulate = 0) {
     const int H = plan->H, F = plan->F, D = plan->D;
     tsp::PairDwPolicy::Params p;
     std::memset(&p, 0, sizeof(p));
@@ -489,6 +492,7 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 64)) return TSP_ERR_CUDA;
     if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 64)) return TSP_ERR_CUDA;
     p.dWd = dWd; p.dWg = dWg; p.dWu = dWu;
+    p.accumulate = accumulate;
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.F_d = F / D;
     p.S_loc = static_cast<int>(S / D);
@@ -519,6 +523,71 @@ bool pairs_for_tokens(const tsp_mlp_plan_t* plan, int64_t S) {
     return padded_pair * 100 <= padded_single * 106;
 }
 bool pairs_for_dw(const tsp_mlp_plan_t* plan) { return plan->use_pairs && (plan->F / plan->D) % 256 == 0; }
+
+// While alive, the plan describes ONE rank's problem: a single shard of width F/D applied to that rank's tokens
+// (the launch helpers read H, F, D from the plan).  Used by the per-rank ring-step entry points.
+struct OneShardView {
+    tsp_mlp_plan_t* plan;
+    int F, D;
+    explicit OneShardView(tsp_mlp_plan_t* p) : plan(p), F(p->F), D(p->D) {
+        plan->F = F / D;
+        plan->D = 1;
+    }
+    ~OneShardView() {
+        plan->F = F;
+        plan->D = D;
+    }
+};
+
+// One ring step for `n_ranks` ranks at once (S tokens in all): gate|up GEMM of every rank's tokens against the shard
+// in that rank's buffer slot into the [S, F/D] scratch, then the down projection of that shard added to the fp32
+// accumulator.  mode: 0 first step, 1 middle, 2 last (rounds to bf16 Y), 3 only step.
+tsp_status_t launch_forward_step(tsp_mlp_plan_t* plan, const void* X, const void* cur_g, const void* cur_u,
+                                 const void* cur_d, void* A_step, float* Yacc, void* Y, int64_t S, int n_ranks, int mode,
+                                 cudaStream_t cs) {
+    const int H = plan->H, F_d = plan->F / plan->D, D = n_ranks;
+    tsp_status_t st;
+    {
+        using Policy = tsp::PairGateUpPolicyT<0>;
+        Policy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_sharded(plan, &p.map_wg, cur_g, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_sharded(plan, &p.map_wu, cur_u, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+        p.A = static_cast<__nv_bfloat16*>(A_step);
+        p.S = static_cast<int>(S); p.H = H; p.F = F_d; p.D = D; p.F_d = F_d;
+        p.S_loc = static_cast<int>(S / D);
+        p.tiles_per_rank = (p.S_loc + 255) / 256;
+        p.m_tiles = D * p.tiles_per_rank;
+        p.jl_blocks = F_d / 128;
+        p.band = gate_band(plan, p.m_tiles);
+        p.rank_indexed = 1;
+        p.act = plan->act;
+        fill_common(plan, p, p.m_tiles * p.jl_blocks);
+        st = launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, cs);
+        if (st != TSP_OK) return st;
+    }
+    {
+        tsp::PairDownStagedPolicy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(plan, &p.map_a, A_step, S, F_d, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_sharded(plan, &p.map_wd, cur_d, D, F_d, H, 64, 64)) return TSP_ERR_CUDA;
+        p.Yacc = Yacc;
+        p.Y = static_cast<__nv_bfloat16*>(Y);
+        p.S = static_cast<int>(S); p.H = H; p.F_d = F_d; p.D = D;
+        p.mode = mode;
+        p.S_loc = static_cast<int>(S / D);
+        p.tiles_per_rank = (p.S_loc + 255) / 256;
+        p.m_tiles = D * p.tiles_per_rank;
+        p.n_blocks = H / 256;
+        const int group = plan->group > 0 ? plan->group : 8;
+        p.group = p.m_tiles < group ? p.m_tiles : group;
+        fill_common(plan, p, p.m_tiles * p.n_blocks);
+        st = launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownStagedPolicy>, p, cs);
+        if (st != TSP_OK) return st;
+    }
+    return TSP_OK;
+}
 
 // ---------------------------------------------------------------------------------------------
 // Fixed scratch for tsp_mlp_forward_static: part of the library image, so every GPU that loads the
@@ -840,45 +909,9 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
         const void* cur_g = t == 0 ? Wg : recv(t & 1, 0);
         const void* cur_u = t == 0 ? Wu : recv(t & 1, 1);
         const void* cur_d = t == 0 ? Wd : recv(t & 1, 2);
-        {
-            using Policy = tsp::PairGateUpPolicyT<0>;
-            Policy::Params p;
-            std::memset(&p, 0, sizeof(p));
-            if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
-            if (!encode_sharded(plan, &p.map_wg, cur_g, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
-            if (!encode_sharded(plan, &p.map_wu, cur_u, D, H, F_d, 64, 64)) return TSP_ERR_CUDA;
-            p.A = static_cast<__nv_bfloat16*>(A_step);
-            p.S = static_cast<int>(S); p.H = H; p.F = F_d; p.D = D; p.F_d = F_d;
-            p.S_loc = static_cast<int>(S / D);
-            p.tiles_per_rank = (p.S_loc + 255) / 256;
-            p.m_tiles = D * p.tiles_per_rank;
-            p.jl_blocks = F_d / 128;
-            p.band = gate_band(plan, p.m_tiles);
-            p.rank_indexed = 1;
-            p.act = plan->act;
-            fill_common(plan, p, p.m_tiles * p.jl_blocks);
-            st = launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, cs);
-            if (st != TSP_OK) return st;
-        }
-        {
-            tsp::PairDownStagedPolicy::Params p;
-            std::memset(&p, 0, sizeof(p));
-            if (!encode_matrix(plan, &p.map_a, A_step, S, F_d, 64, 128)) return TSP_ERR_CUDA;
-            if (!encode_sharded(plan, &p.map_wd, cur_d, D, F_d, H, 64, 64)) return TSP_ERR_CUDA;
-            p.Yacc = Yacc;
-            p.Y = static_cast<__nv_bfloat16*>(Y);
-            p.S = static_cast<int>(S); p.H = H; p.F_d = F_d; p.D = D;
-            p.mode = D == 1 ? 3 : (t == 0 ? 0 : (t == D - 1 ? 2 : 1));
-            p.S_loc = static_cast<int>(S / D);
-            p.tiles_per_rank = (p.S_loc + 255) / 256;
-            p.m_tiles = D * p.tiles_per_rank;
-            p.n_blocks = H / 256;
-            const int group = plan->group > 0 ? plan->group : 8;
-            p.group = p.m_tiles < group ? p.m_tiles : group;
-            fill_common(plan, p, p.m_tiles * p.n_blocks);
-            st = launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownStagedPolicy>, p, cs);
-            if (st != TSP_OK) return st;
-        }
+        st = launch_forward_step(plan, X, cur_g, cur_u, cur_d, A_step, Yacc, Y, S, D,
+                                 D == 1 ? 3 : (t == 0 ? 0 : (t == D - 1 ? 2 : 1)), cs);
+        if (st != TSP_OK) return st;
         if ((e = cudaEventRecord(ev_done(t), cs)) != cudaSuccess) return cuda_fail(plan, e);
     }
     prof.mark();
@@ -887,6 +920,91 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
     if ((e = cudaEventRecord(ev_end, xs)) != cudaSuccess) return cuda_fail(plan, e);
     if ((e = cudaStreamWaitEvent(cs, ev_end, 0)) != cudaSuccess) return cuda_fail(plan, e);
     return TSP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// One ring step on one rank's data (every rank on a GPU of its own; the caller moves the shards).
+// ---------------------------------------------------------------------------------------------
+size_t tsp_mlp_workspace_bytes_ring(const tsp_mlp_plan_t* plan, int64_t S_loc, int pass) {
+    if (!plan || S_loc <= 0) return 0;
+    const size_t one = align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2, 256);
+    const size_t acc = align_up(static_cast<size_t>(S_loc) * plan->H * 4, 256);
+    if (pass == TSP_WS_FORWARD) return one + acc;                       // A | Yacc
+    if (pass == TSP_WS_BACKWARD) return 3 * one + 2 * one + acc;        // A, dG, dU | dA (fp32) | dXacc
+    return 0;
+}
+
+tsp_status_t tsp_mlp_ring_step(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
+                               const void* Wd_k, void* Y_p, int64_t S_loc, int t, int D, void* cuda_stream) {
+    if (!plan || D != plan->D || t < 0 || t >= D) return TSP_ERR_INVALID_ARG;
+    if (S_loc < 1 || S_loc > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X_p || !Wg_k || !Wu_k || !Wd_k || !Y_p) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X_p) || !aligned16(Wg_k) || !aligned16(Wu_k) || !aligned16(Wd_k) || !aligned32(Y_p))
+        return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_ring(plan, S_loc, TSP_WS_FORWARD))
+        return TSP_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* base = static_cast<uint8_t*>(plan->workspace);
+    void* A_step = base;
+    float* Yacc = reinterpret_cast<float*>(base + align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2, 256));
+    Profiler prof(plan, cs);
+    tsp_status_t st = launch_forward_step(plan, X_p, Wg_k, Wu_k, Wd_k, A_step, Yacc, Y_p, S_loc, 1,
+                                          D == 1 ? 3 : (t == 0 ? 0 : (t == D - 1 ? 2 : 1)), cs);
+    prof.mark();
+    return st;
+}
+
+tsp_status_t tsp_mlp_ring_step_backward_dx(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
+                                           const void* Wd_k, const void* dY_p, void* dX_p, int64_t S_loc, int t, int D,
+                                           void* cuda_stream) {
+    if (!plan || D != plan->D || t < 0 || t >= D) return TSP_ERR_INVALID_ARG;
+    if (S_loc < 1 || S_loc > (1ll << 24) || (plan->F / plan->D) % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X_p || !Wg_k || !Wu_k || !Wd_k || !dY_p || !dX_p) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X_p) || !aligned16(Wg_k) || !aligned16(Wu_k) || !aligned16(Wd_k) || !aligned16(dY_p) || !aligned32(dX_p))
+        return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_ring(plan, S_loc, TSP_WS_BACKWARD))
+        return TSP_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    const size_t one = align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2, 256);
+    uint8_t* base = static_cast<uint8_t*>(plan->workspace);
+    void* A = base;
+    void* dG = base + one;
+    void* dU = base + 2 * one;
+    float* dA = reinterpret_cast<float*>(base + 3 * one);
+    float* dXacc = reinterpret_cast<float*>(base + 5 * one);
+    Profiler prof(plan, cs);
+    OneShardView view(plan);
+    tsp_status_t st = launch_da_pair(plan, dY_p, Wd_k, dA, S_loc, cs);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    st = launch_gate_pair<1>(plan, X_p, Wg_k, Wu_k, A, dA, dG, dU, S_loc, cs);
+    if (st != TSP_OK) return st;
+    prof.mark();
+    const int carry = D == 1 ? 0 : (t == 0 ? 1 : (t == D - 1 ? 3 : 2));
+    st = launch_bwd_dx_pair(plan, dG, dU, Wg_k, Wu_k, dX_p, S_loc, cs, dXacc, carry);
+    prof.mark();
+    return st;
+}
+
+tsp_status_t tsp_mlp_ring_step_backward_dw(tsp_mlp_plan_t* plan, const void* X_p, const void* dY_p, float* dWg_k,
+                                           float* dWu_k, float* dWd_k, int64_t S_loc, int accumulate, int D,
+                                           void* cuda_stream) {
+    if (!plan || D != plan->D || (accumulate != 0 && accumulate != 1)) return TSP_ERR_INVALID_ARG;
+    if (S_loc < 1 || S_loc > (1ll << 24) || (plan->F / plan->D) % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X_p || !dY_p || !dWg_k || !dWu_k || !dWd_k) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X_p) || !aligned16(dY_p) || !aligned32(dWg_k) || !aligned32(dWu_k) || !aligned32(dWd_k))
+        return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_ring(plan, S_loc, TSP_WS_BACKWARD))
+        return TSP_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    const size_t one = align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2, 256);
+    uint8_t* base = static_cast<uint8_t*>(plan->workspace);
+    Profiler prof(plan, cs);
+    OneShardView view(plan);
+    tsp_status_t st = launch_bwd_dw_pair(plan, X_p, dY_p, base, base + one, base + 2 * one, dWg_k, dWu_k, dWd_k, S_loc, cs,
+                                         accumulate);
+    prof.mark();
+    return st;
 }
 
 // ---------------------------------------------------------------------------------------------

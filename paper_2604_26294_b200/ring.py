@@ -1,0 +1,165 @@
+"""Algorithm 2 across real ranks: one process per GPU, each owning one token shard and one weight shard.
+
+The single-GPU entry points keep all D shards resident, so nothing moves.  Here the shards really travel:
+at every ring step a rank posts "send my current shard to p+1, receive the next one from p-1"
+(AsyncRingSendRecv), computes the step with the shard it holds (`tsp_mlp_ring_step*`), waits, and swaps
+buffers.  `torch.distributed` does the transport (NCCL over NVLink on GPUs; gloo on CPU, which is how the
+schedule is tested without GPUs); every FLOP of a step runs in the library's kernels.
+
+Backward pass: the weights travel as in the forward pass (Section 4.3.4: the backward mirrors the forward
+weight movement) and the partial weight gradients are summed to the owner (Section 4.7) by an fp32
+accumulator that travels WITH its shard: the rank holding shard k at step t adds its contribution and passes
+the accumulator on, so after the last hop the owner holds the sum over the ranks in the order the shard met
+them, r = (k + t) mod D.  This is a ring reduce-scatter whose transfers overlap the next step's GEMMs.
+
+The two schedule functions are transport- and device-agnostic (compute is a callback); `TspRingMlp` binds them
+to the CUDA library.
+"""
+from __future__ import annotations
+
+from typing import Callable, Sequence
+
+import torch
+import torch.distributed as dist
+
+
+def ring_neighbours(rank: int, D: int) -> tuple[int, int]:
+    """(destination, source) of a rank's ring transfers: send to p+1, receive from p-1 (Algorithm 2)."""
+    return (rank + 1) % D, (rank - 1) % D
+
+
+def shard_at_step(rank: int, t: int, D: int) -> int:
+    """Index of the weight shard rank `rank` holds at ring step t."""
+    return (rank - t) % D
+
+
+def _exchange(send: torch.Tensor, recv: torch.Tensor, rank: int, D: int, group=None):
+    dst, src = ring_neighbours(rank, D)
+    if group is not None:
+        dst, src = dist.get_global_rank(group, dst), dist.get_global_rank(group, src)
+    ops = [dist.P2POp(dist.isend, send, dst, group), dist.P2POp(dist.irecv, recv, src, group)]
+    return dist.batch_isend_irecv(ops)
+
+
+def _wait(reqs) -> None:
+    for r in reqs:
+        r.wait()
+
+
+def ring_forward(compute: Callable[[int, int, torch.Tensor], None], own_shard: torch.Tensor,
+                 recv_bufs: Sequence[torch.Tensor], rank: int, D: int, group=None) -> None:
+    """The loop of Algorithm 2 on one rank.
+
+    compute(t, k, shard) runs ring step t with the packed shard k = (rank - t) mod D it is handed;
+    own_shard is this rank's packed shard (never written); recv_bufs are two buffers of the same shape
+    that alternate as receive target.  The transfer for step t+1 is posted before step t computes.
+    """
+    cur = own_shard
+    for t in range(D):
+        reqs = []
+        if t < D - 1:
+            nxt = recv_bufs[t & 1]
+            reqs = _exchange(cur, nxt, rank, D, group)
+        compute(t, shard_at_step(rank, t, D), cur)
+        _wait(reqs)                      # Wait(): the next shard has arrived, the current one has left
+        if t < D - 1:
+            cur = nxt
+
+
+def ring_backward(compute_dx: Callable[[int, int, torch.Tensor], None],
+                  compute_dw: Callable[[int, int, torch.Tensor, bool], None], own_shard: torch.Tensor,
+                  recv_bufs: Sequence[torch.Tensor], dw_bufs: Sequence[torch.Tensor], rank: int, D: int,
+                  group=None) -> torch.Tensor:
+    """Backward ring on one rank; returns the buffer holding the summed gradient of this rank's OWN shard.
+
+    compute_dx(t, k, shard): everything of step t that does not touch the weight-gradient accumulator.
+    compute_dw(t, k, acc, accumulate): add (or, at t = 0, write) this rank's contribution for shard k into acc.
+    dw_bufs: two fp32 buffers shaped like a packed shard; they alternate as "accumulator of the shard I hold"
+    and "accumulator arriving for the next step".
+    """
+    cur = own_shard
+    acc_reqs = []
+    for t in range(D):
+        reqs = []
+        if t < D - 1:
+            nxt = recv_bufs[t & 1]
+            reqs = _exchange(cur, nxt, rank, D, group)
+        k = shard_at_step(rank, t, D)
+        compute_dx(t, k, cur)
+        _wait(acc_reqs)                  # the accumulator of shard k has arrived from p-1 (nothing to wait for at t = 0)
+        acc = dw_bufs[t & 1]
+        compute_dw(t, k, acc, t > 0)
+        if D > 1:                        # pass it on; the hop after the last step delivers it to the owner
+            acc_reqs = _exchange(acc, dw_bufs[(t + 1) & 1], rank, D, group)
+        _wait(reqs)
+        if t < D - 1:
+            cur = nxt
+    _wait(acc_reqs)
+    return dw_bufs[D & 1] if D > 1 else dw_bufs[0]
+
+
+def pack_shard(Wg_k: torch.Tensor, Wu_k: torch.Tensor, Wd_k: torch.Tensor) -> torch.Tensor:
+    """One contiguous message per ring step: [Wg_k | Wu_k | Wd_k] flattened."""
+    return torch.cat([Wg_k.reshape(-1), Wu_k.reshape(-1), Wd_k.reshape(-1)])
+
+
+def unpack_shard(buf: torch.Tensor, H: int, F_d: int):
+    """Views (Wg_k [H, F_d], Wu_k [H, F_d], Wd_k [F_d, H]) into a packed shard (or packed gradient) buffer."""
+    n = H * F_d
+    return buf[:n].view(H, F_d), buf[n:2 * n].view(H, F_d), buf[2 * n:3 * n].view(F_d, H)
+
+
+class TspRingMlp:
+    """One rank of the TSP gated ring MLP on its own GPU: the schedule above driving the library's step kernels."""
+
+    def __init__(self, H: int, F: int, D: int, rank: int, S_loc: int, group=None, training: bool = False,
+                 activation: int | None = None):
+        from . import binding as b   # fails loudly without the CUDA library or a GPU
+
+        self.b, self.H, self.F, self.D, self.rank, self.S_loc, self.group = b, H, F, D, rank, S_loc, group
+        self.F_d = F // D
+        dev = torch.device("cuda", torch.cuda.current_device())
+        self.plan = b.tsp_mlp_plan(H, F, D)
+        if activation is not None:
+            b.tsp_mlp_set_activation(self.plan, activation)
+        nbytes = b.tsp_mlp_workspace_bytes_ring(self.plan, S_loc, b.TSP_WS_BACKWARD if training else b.TSP_WS_FORWARD)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        b.tsp_mlp_set_workspace(self.plan, self.workspace)
+        n = 3 * H * self.F_d
+        self.recv_bufs = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(2)] if D > 1 else []
+        self.dw_bufs = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(2 if D > 1 else 1)] if training else []
+
+    def close(self) -> None:
+        if self.plan is not None:
+            self.b.tsp_mlp_plan_destroy(self.plan)
+            self.plan = None
+
+    def forward(self, X_p: torch.Tensor, shard: torch.Tensor, Y_p: torch.Tensor | None = None) -> torch.Tensor:
+        """Y_p = rows of this rank of the gated MLP over all D shards; `shard` is this rank's packed own shard."""
+        if Y_p is None:
+            Y_p = torch.empty_like(X_p)
+
+        def compute(t, k, buf):
+            Wg, Wu, Wd = unpack_shard(buf, self.H, self.F_d)
+            self.b.tsp_mlp_ring_step(self.plan, X_p, Wg, Wu, Wd, Y_p, self.S_loc, t, self.D)
+
+        ring_forward(compute, shard, self.recv_bufs, self.rank, self.D, self.group)
+        return Y_p
+
+    def backward(self, X_p: torch.Tensor, shard: torch.Tensor, dY_p: torch.Tensor, dX_p: torch.Tensor | None = None):
+        """Returns (dX_p, (dWg, dWu, dWd)) with the weight gradients of this rank's own shard, fp32, summed over ranks."""
+        if not self.dw_bufs:
+            raise RuntimeError("TspRingMlp was created with training=False")
+        if dX_p is None:
+            dX_p = torch.empty_like(X_p)
+
+        def compute_dx(t, k, buf):
+            Wg, Wu, Wd = unpack_shard(buf, self.H, self.F_d)
+            self.b.tsp_mlp_ring_step_backward_dx(self.plan, X_p, Wg, Wu, Wd, dY_p, dX_p, self.S_loc, t, self.D)
+
+        def compute_dw(t, k, acc, accumulate):
+            dWg, dWu, dWd = unpack_shard(acc, self.H, self.F_d)
+            self.b.tsp_mlp_ring_step_backward_dw(self.plan, X_p, dY_p, dWg, dWu, dWd, self.S_loc, int(accumulate), self.D)
+
+        out = ring_backward(compute_dx, compute_dw, shard, self.recv_bufs, self.dw_bufs, self.rank, self.D, self.group)
+        return dX_p, unpack_shard(out, self.H, self.F_d)

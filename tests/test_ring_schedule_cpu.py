@@ -1,0 +1,28 @@
+"""The multi-rank ring schedules (forward and backward with travelling gradient accumulators) over gloo on CPU."""
+import json
+import os
+
+import pytest
+
+from paper_2604_26294_b200 import ring
+from tests.test_multi_rank_cpu import ROOT, _torchrun
+
+
+def test_neighbours_and_shard_index():
+    assert ring.ring_neighbours(0, 4) == (1, 3) and ring.ring_neighbours(3, 4) == (0, 2)
+    for D in (1, 2, 3, 8):
+        for r in range(D):
+            met = [ring.shard_at_step(r, t, D) for t in range(D)]
+            assert met[0] == r and sorted(met) == list(range(D))        # own shard first, every shard once
+            assert all(ring.shard_at_step((r + 1) % D, t + 1, D) == met[t] for t in range(D - 1))  # it moves to p+1
+
+
+@pytest.mark.parametrize("world", [2, 3, 4])   # 3 and 4: p+1 and p-1 are different ranks, a reversed ring would show
+def test_ring_schedules_reach_the_unsharded_result(tmp_path, world):
+    res = _torchrun([os.path.join(ROOT, "tests", "ring_worker.py"), str(tmp_path)], nproc=world)
+    assert res.returncode == 0, res.stderr[-3000:]
+    for r in range(world):
+        o = json.load(open(tmp_path / f"rank{r}.json"))
+        assert o["visited"] == [(r - t) % world for t in range(world)]
+        for key in ("err_Y", "err_dX", "err_dWg", "err_dWu", "err_dWd"):
+            assert o[key] <= 1e-12, (r, key, o[key])
