@@ -450,6 +450,95 @@ def run_gpu(args, wl):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# Ring arm (opt-in, --mode ring): the D = N ranks are the N GPUs, every rank holds its own token shard and ONE
+# weight shard, and the shards travel over NCCL send / receive (paper_2604_26294_b200/ring.py).  The work of the
+# workload is divided over the ranks (strong scaling); at N = 1 it is the D = 1 problem through the step kernels.
+# ------------------------------------------------------------------------------------------------
+def run_ring(args, wl):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2604_26294_b200 import binding as b
+    from paper_2604_26294_b200 import build as _build
+    from paper_2604_26294_b200 import ring
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if local_rank == 0:
+        _build.build_library()
+    if world > 1:
+        dist.barrier()
+    train = wl.name == "train" or args.backward
+    S, H, F, D = wl.S, wl.H, wl.F, world
+    if S % D or F % D or (F // D) % (256 if train else 128):
+        raise SystemExit(f"workload {wl.name} does not divide over {D} ranks")
+    S_loc, F_d = S // D, F // D
+    host = inp.make_inputs(S, H, F, seed=0, with_dy=train)      # the same problem on every rank; each keeps its shards
+
+    def dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    X_p = dev(host.X[rank * S_loc:(rank + 1) * S_loc])
+    cols = slice(rank * F_d, (rank + 1) * F_d)
+    shard = ring.pack_shard(dev(host.Wg[:, cols]), dev(host.Wu[:, cols]), dev(host.Wd[cols, :]))
+    Y_p = torch.empty_like(X_p)
+    mlp = ring.TspRingMlp(H, F, D, rank, S_loc, training=train)
+    if train:
+        dY_p = dev(host.dY[rank * S_loc:(rank + 1) * S_loc])
+        dX_p = torch.empty_like(X_p)
+
+    def step():
+        mlp.forward(X_p, shard, Y_p)
+        if train:
+            mlp.backward(X_p, shard, dY_p, dX_p)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    assert b.tsp_mlp_status(mlp.plan) == b.TSP_OK, "device-side wait timed out during warm-up"
+    sampler = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    sampler.stop()
+    assert b.tsp_mlp_status(mlp.plan) == b.TSP_OK, "device-side wait timed out"
+    ms_per_step = max_over_ranks(e0.elapsed_time(e1), world, "cuda") / args.steps
+    model_flops = wl.forward_flops() + (wl.backward_flops() if train else 0.0)   # of the whole job, all ranks together
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": model_flops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "pass": "forward+backward (G, U recomputed)" if train else "forward",
+                       "mode": "ring (one rank per GPU, shards travel over NCCL send/receive)", "S": S, "H": H, "F": F,
+                       "D": D, "tokens_per_rank": S_loc, "shard_width": F_d,
+                       "ring_bytes_sent_per_rank_per_step": (D - 1) * 6 * H * F_d + (D * 12 * H * F_d if train and D > 1 else 0)},
+            "clocks": sampler.summary(), "gpu_launches": int(args.steps * D * (6 if train else 2)),
+            "e2e": None, "roofline": None, "cpu_baseline": None,
+        }
+        print(json.dumps(line), flush=True)
+    mlp.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -459,8 +548,9 @@ def main():
     ap.add_argument("--backward", action="store_true", help="time forward + backward (as the `train` workload does)")
     ap.add_argument("--stored-activations", action="store_true",
                     help="training step through tsp_mlp_forward_save / tsp_mlp_backward_saved (no recomputation)")
-    ap.add_argument("--mode", default="direct", choices=["direct", "staged"],
-                    help="staged: Algorithm 2 step by step with the shard transfer emulated on a side stream")
+    ap.add_argument("--mode", default="direct", choices=["direct", "staged", "ring"],
+                    help="staged: Algorithm 2 step by step with the shard transfer emulated on a side stream; "
+                         "ring: D = N ranks on N GPUs, the shards travel between the GPUs")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the torch-eager context measurement")
@@ -469,6 +559,8 @@ def main():
     wl = inp.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.mode == "ring":
+        run_ring(args, wl)
     else:
         run_gpu(args, wl)
 

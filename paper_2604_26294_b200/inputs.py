@@ -170,3 +170,62 @@ def sample_columns(F: int, D: int, count: int, seed: int = 2) -> np.ndarray:
     for k in range(D):
         cols.extend(k * F_d + rng.choice(F_d, size=min(per, F_d), replace=False))
     return np.sort(np.asarray(cols, dtype=np.int64))
+
+
+# ----------------------------------------------------------------------------------------
+# Projection GEMMs of TSP attention (Algorithm 1): seeded inputs only, no arithmetic of the method.
+# ----------------------------------------------------------------------------------------
+@dataclass(frozen=True)
+class AttnWorkload:
+    """S tokens, hidden H, query width Hq = n_heads * head_dim, key/value width Hkv = Hq / g, D shards."""
+
+    name: str
+    S: int
+    H: int
+    Hq: int
+    Hkv: int
+    D: int
+
+    def qkv_flops(self) -> float:
+        return 2.0 * self.S * self.H * (self.Hq + 2 * self.Hkv)
+
+    def out_flops(self) -> float:
+        return 2.0 * self.S * self.Hq * self.H
+
+
+ATTN_WORKLOADS = {
+    "attn_tiny": AttnWorkload("attn_tiny", S=256, H=256, Hq=512, Hkv=256, D=2),
+    # 7B-class layer of the reference-model table: h = 4096, 32 heads of 128; MHA and a GQA variant (g = 4)
+    "attn_7b_mha": AttnWorkload("attn_7b_mha", S=8192, H=4096, Hq=4096, Hkv=4096, D=8),
+    "attn_7b_gqa4": AttnWorkload("attn_7b_gqa4", S=8192, H=4096, Hq=4096, Hkv=1024, D=8),
+    "attn_7b_long": AttnWorkload("attn_7b_long", S=65536, H=4096, Hq=4096, Hkv=4096, D=8),
+}
+
+
+@dataclass
+class AttnInputs:
+    """bf16 bit patterns (uint16), unsharded layouts (rows of the weights = output features)."""
+
+    X: np.ndarray   # [S, H]
+    Wq: np.ndarray  # [Hq, H]
+    Wk: np.ndarray  # [Hkv, H]
+    Wv: np.ndarray  # [Hkv, H]
+    A: np.ndarray   # [S, Hq]   stand-in for the attention output fed to the output projection
+    Wo: np.ndarray  # [H, Hq]
+
+
+def make_attn_inputs(S: int, H: int, Hq: int, Hkv: int, seed: int = 0) -> AttnInputs:
+    """Draw order X, Wq, Wk, Wv, A, Wo; X, A ~ N(0,1); Wq, Wk, Wv ~ N(0, var 1/H); Wo ~ N(0, var 1/Hq)."""
+    rng = np.random.Generator(np.random.Philox(seed))
+    X = _draw_bf16(rng, (S, H), 1.0)
+    Wq = _draw_bf16(rng, (Hq, H), H ** -0.5)
+    Wk = _draw_bf16(rng, (Hkv, H), H ** -0.5)
+    Wv = _draw_bf16(rng, (Hkv, H), H ** -0.5)
+    A = _draw_bf16(rng, (S, Hq), 1.0)
+    Wo = _draw_bf16(rng, (H, Hq), Hq ** -0.5)
+    return AttnInputs(X, Wq, Wk, Wv, A, Wo)
+
+
+def shard_out_columns(Wo: np.ndarray, D: int) -> np.ndarray:
+    """[H, Hq] -> [D, H, Hq/D]: shard r of the output projection holds the columns of shard r's heads."""
+    return shard_columns(Wo, D)
