@@ -52,6 +52,14 @@ SIGNATURES = {
     "tsp_mlp_ring_step": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_forward_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, _P,
                                               ctypes.c_int64, ctypes.POINTER(ctypes.c_int), _P]),
+    "tsp_attn_plan": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(_P)]),
+    "tsp_attn_plan_destroy": (ctypes.c_int, [_P]),
+    "tsp_attn_qkv_forward": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_attn_out_forward": (ctypes.c_int, [_P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_attn_status": (ctypes.c_int, [_P]),
+    "tsp_attn_profile_begin": (ctypes.c_int, [_P, ctypes.c_int]),
+    "tsp_attn_profile_read": (ctypes.c_int, [_P, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]),
+    "tsp_attn_profile_end": (ctypes.c_int, [_P]),
     "tsp_mlp_selftest_wait_expiry": (ctypes.c_int, [_P, ctypes.c_int, _P]),
     "tsp_mlp_status": (ctypes.c_int, [_P]),
     "tsp_mlp_error_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -278,3 +286,43 @@ def tsp_mlp_profile_end(plan) -> None:
 
 def tsp_mlp_kernels_per_call(plan, backward: int = TSP_WS_FORWARD) -> int:
     return int(load_library().tsp_mlp_kernels_per_call(plan, backward))
+
+
+# --------------------------------------------------------------------------- include/tsp_attn.h, same names
+def tsp_attn_plan(H: int, Hq: int, Hkv: int, D: int):
+    """Plan for the projection GEMMs of TSP attention: hidden H, query width Hq, key/value width Hkv, D shards."""
+    out = ctypes.c_void_p()
+    _check(load_library().tsp_attn_plan(H, Hq, Hkv, D, ctypes.byref(out)), "tsp_attn_plan")
+    return out
+
+
+def tsp_attn_plan_destroy(plan) -> None:
+    _check(load_library().tsp_attn_plan_destroy(plan), "tsp_attn_plan_destroy")
+
+
+def tsp_attn_qkv_forward(plan, X, Wq, Wk, Wv, Q, K, V, S: int, D: int, stream=None) -> None:
+    _check(load_library().tsp_attn_qkv_forward(plan, _ptr(X), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(Q), _ptr(K), _ptr(V),
+                                               S, D, _stream_handle(stream)), "tsp_attn_qkv_forward")
+
+
+def tsp_attn_out_forward(plan, A, Wo, Y, S: int, D: int, stream=None) -> None:
+    _check(load_library().tsp_attn_out_forward(plan, _ptr(A), _ptr(Wo), _ptr(Y), S, D, _stream_handle(stream)),
+           "tsp_attn_out_forward")
+
+
+def tsp_attn_status(plan) -> int:
+    return int(load_library().tsp_attn_status(plan))
+
+
+def tsp_attn_profile_begin(plan, max_calls: int) -> None:
+    _check(load_library().tsp_attn_profile_begin(plan, max_calls), "tsp_attn_profile_begin")
+
+
+def tsp_attn_profile_read(plan, call_index: int) -> float:
+    ms = ctypes.c_float()
+    _check(load_library().tsp_attn_profile_read(plan, call_index, ctypes.byref(ms)), "tsp_attn_profile_read")
+    return float(ms.value)
+
+
+def tsp_attn_profile_end(plan) -> None:
+    _check(load_library().tsp_attn_profile_end(plan), "tsp_attn_profile_end")

@@ -1,0 +1,118 @@
+// C-ABI of the attention projection GEMMs (include/tsp_attn.h).  Included once, at the end of tsp_mlp.cu, because
+// it reuses that file's host helpers (tensor-map encoding, pair launch, status word, profiling events).
+#pragma once
+#include "../../include/tsp_attn.h"
+#include "attn_kernels.cuh"
+
+struct tsp_attn_plan {
+    tsp_mlp_plan_t* base;  // device properties, tensor-map encoder, status word, profiling events
+    int H, Hq, Hkv, D;
+};
+
+extern "C" {
+
+tsp_status_t tsp_attn_plan(int H, int Hq, int Hkv, int D, tsp_attn_plan_t** out) {
+    if (!out) return TSP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (H <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || D > 64) return TSP_ERR_INVALID_ARG;
+    if (H % 256 != 0 || Hq % 256 != 0 || Hkv % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (Hq % D != 0 || Hkv % D != 0 || (Hq / D) % 64 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (H > (1 << 20) || Hq > (1 << 20) || Hkv > (1 << 20)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    tsp_mlp_plan_t* base = nullptr;
+    tsp_status_t st = tsp_mlp_plan(H, 128, 1, &base);  // only the shared machinery of the plan is used
+    if (st != TSP_OK) return st;
+    tsp_attn_plan_t* plan = new (std::nothrow) tsp_attn_plan_t();
+    if (!plan) {
+        tsp_mlp_plan_destroy(base);
+        return TSP_ERR_INVALID_ARG;
+    }
+    plan->base = base;
+    plan->H = H; plan->Hq = Hq; plan->Hkv = Hkv; plan->D = D;
+    *out = plan;
+    return TSP_OK;
+}
+
+tsp_status_t tsp_attn_plan_destroy(tsp_attn_plan_t* plan) {
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    tsp_mlp_plan_destroy(plan->base);
+    delete plan;
+    return TSP_OK;
+}
+
+tsp_status_t tsp_attn_qkv_forward(tsp_attn_plan_t* plan, const void* X, const void* Wq, const void* Wk, const void* Wv,
+                                  void* Q, void* K, void* V, int64_t S, int D, void* cuda_stream) {
+    if (!plan || D != plan->D || S < 1) return TSP_ERR_INVALID_ARG;
+    if (S > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X || !Wq || !Wk || !Wv || !Q || !K || !V) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned32(Q) || !aligned32(K) || !aligned32(V))
+        return TSP_ERR_INVALID_ARG;
+    tsp_mlp_plan_t* base = plan->base;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int H = plan->H, Hq = plan->Hq, Hkv = plan->Hkv;
+    tsp::PairQkvPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(base, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(base, &p.map_wq, Wq, Hq, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(base, &p.map_wk, Wk, Hkv, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_matrix(base, &p.map_wv, Wv, Hkv, H, 64, 128)) return TSP_ERR_CUDA;
+    p.Q = static_cast<__nv_bfloat16*>(Q);
+    p.K = static_cast<__nv_bfloat16*>(K);
+    p.V = static_cast<__nv_bfloat16*>(V);
+    p.S = static_cast<int>(S); p.H = H; p.Hq = Hq; p.Hkv = Hkv;
+    p.m_tiles = static_cast<int>((S + 255) / 256);
+    p.q_blocks = Hq / 256;
+    p.kv_blocks = Hkv / 256;
+    p.n_blocks = p.q_blocks + 2 * p.kv_blocks;
+    p.band = gate_band(base, p.m_tiles);   // the band's rows of X take about 32 MB of L2
+    fill_common(base, p, p.m_tiles * p.n_blocks);
+    Profiler prof(base, stream);
+    tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairQkvPolicy>, p, stream);
+    prof.mark();
+    return st;
+}
+
+tsp_status_t tsp_attn_out_forward(tsp_attn_plan_t* plan, const void* A, const void* Wo, void* Y, int64_t S, int D,
+                                  void* cuda_stream) {
+    if (!plan || D != plan->D || S < 1) return TSP_ERR_INVALID_ARG;
+    if (S > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!A || !Wo || !Y) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(Wo) || !aligned32(Y)) return TSP_ERR_INVALID_ARG;
+    tsp_mlp_plan_t* base = plan->base;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int H = plan->H, Hq = plan->Hq, Hq_d = plan->Hq / plan->D;
+    tsp::PairOutPolicy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(base, &p.map_a, A, S, Hq, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(base, &p.map_wo, Wo, D, H, Hq_d, 64, 128)) return TSP_ERR_CUDA;
+    p.Y = static_cast<__nv_bfloat16*>(Y);
+    p.S = static_cast<int>(S); p.H = H; p.Hq = Hq; p.D = D; p.Hq_d = Hq_d;
+    p.m_tiles = static_cast<int>((S + 255) / 256);
+    p.n_blocks = H / 256;
+    const int group = base->group > 0 ? base->group : 8;
+    p.group = p.m_tiles < group ? p.m_tiles : group;
+    fill_common(base, p, p.m_tiles * p.n_blocks);
+    Profiler prof(base, stream);
+    tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairOutPolicy>, p, stream);
+    prof.mark();
+    return st;
+}
+
+tsp_status_t tsp_attn_status(tsp_attn_plan_t* plan) { return plan ? tsp_mlp_status(plan->base) : TSP_ERR_INVALID_ARG; }
+
+tsp_status_t tsp_attn_profile_begin(tsp_attn_plan_t* plan, int max_calls) {
+    return plan ? tsp_mlp_profile_begin(plan->base, max_calls) : TSP_ERR_INVALID_ARG;
+}
+tsp_status_t tsp_attn_profile_read(tsp_attn_plan_t* plan, int call_index, float* ms_out) {
+    if (!plan || !ms_out) return TSP_ERR_INVALID_ARG;
+    int n = 0;
+    float ms[kMaxKernelsPerCall] = {};
+    tsp_status_t st = tsp_mlp_profile_read(plan->base, call_index, &n, ms);
+    if (st != TSP_OK) return st;
+    *ms_out = n >= 1 ? ms[0] : 0.0f;
+    return TSP_OK;
+}
+tsp_status_t tsp_attn_profile_end(tsp_attn_plan_t* plan) {
+    return plan ? tsp_mlp_profile_end(plan->base) : TSP_ERR_INVALID_ARG;
+}
+
+}  // extern "C"

@@ -1248,3 +1248,6 @@ int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass) {
 }
 
 }  // extern "C"
+
+// Projection GEMMs of TSP attention (Algorithm 1): same library, own header and entry points.
+#include "tsp_attn_host.cuh"

@@ -19,16 +19,20 @@ def lib():
 
 
 def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "tsp_mlp.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(tsp_mlp_\w+)\s*\(", text)))
+    names = set()
+    for header in ("tsp_mlp.h", "tsp_attn.h"):
+        text = open(os.path.join(ROOT, "include", header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(tsp_(?:mlp|attn)_\w+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol(lib):
     names = _declared_functions()
     assert "tsp_mlp_plan" in names and "tsp_mlp_forward" in names and "tsp_mlp_backward" in names
+    assert "tsp_attn_qkv_forward" in names and "tsp_attn_out_forward" in names and "tsp_mlp_ring_step" in names
     for n in names:
-        assert hasattr(lib, n), f"{n} declared in include/tsp_mlp.h but not exported"
+        assert hasattr(lib, n), f"{n} declared in include/ but not exported"
         assert n in b.SIGNATURES, f"{n} has no binding signature"
         assert callable(getattr(b, n)), f"binding lacks {n}"
 
