@@ -539,12 +539,103 @@ def run_ring(args, wl):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# Attention-projection arm (workloads attn_*): the two dense steps of Algorithm 1, one kernel each.
+# ------------------------------------------------------------------------------------------------
+def run_attn(args, wl):
+    import torch
+
+    from oracle import tsp_attn_proj_oracle as attn_orc  # cpu_baseline leg only
+    from paper_2604_26294_b200 import binding as b
+    from paper_2604_26294_b200 import build as _build
+
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("the attention-projection arm runs on one GPU")
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(0)
+    _build.build_library()
+    S, H, Hq, Hkv, D = wl.S, wl.H, wl.Hq, wl.Hkv, wl.D
+    host = inp.make_attn_inputs(S, H, Hq, Hkv, seed=0)
+
+    def dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    X, Wq, Wk, Wv, A = dev(host.X), dev(host.Wq), dev(host.Wk), dev(host.Wv), dev(host.A)
+    Wo = dev(inp.shard_out_columns(host.Wo, D))
+    Q = torch.empty(S, Hq, dtype=torch.bfloat16, device="cuda")
+    K = torch.empty(S, Hkv, dtype=torch.bfloat16, device="cuda")
+    V = torch.empty(S, Hkv, dtype=torch.bfloat16, device="cuda")
+    Y = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
+    plan = b.tsp_attn_plan(H, Hq, Hkv, D)
+
+    def step():
+        b.tsp_attn_qkv_forward(plan, X, Wq, Wk, Wv, Q, K, V, S, D)
+        b.tsp_attn_out_forward(plan, A, Wo, Y, S, D)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    assert b.tsp_attn_status(plan) == b.TSP_OK
+    n_prof = min(4096, 2 * args.steps)
+    b.tsp_attn_profile_begin(plan, n_prof)
+    sampler = ClockSampler(0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.stop()
+    assert b.tsp_attn_status(plan) == b.TSP_OK, "device-side wait timed out"
+    ms_per_step = e0.elapsed_time(e1) / args.steps
+    qkv_ms = float(np.mean([b.tsp_attn_profile_read(plan, i) for i in range(0, n_prof, 2)]))
+    out_ms = float(np.mean([b.tsp_attn_profile_read(plan, i) for i in range(1, n_prof, 2)]))
+    b.tsp_attn_profile_end(plan)
+    flops = wl.qkv_flops() + wl.out_flops()
+    peaks = measured_peaks()
+    achieved = wl.qkv_flops() / (qkv_ms * 1e-3) / 1e12
+    # oracle timed on a bounded sample of rows (row-separable), host cores
+    cpu = None
+    if not args.no_cpu_baseline:
+        f = [inp.bf16_bits_to_f64(a) for a in (host.X, host.Wq, host.Wk, host.Wv, host.A, host.Wo)]
+        rows = np.arange(0, S, max(1, S // 256))[:256]
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < 10.0:
+            attn_orc.qkv_rows(f[0], f[1], f[2], f[3], rows)
+            attn_orc.output_rows(f[4], f[5], rows)
+            reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        cpu = {"value": flops * len(rows) / S / dt / 1e12, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
+               "kind": "oracle", "sample": f"{len(rows)} of {S} token rows, fp64, {reps} repetitions"}
+    line = {
+        "metric": "TSP attention projection GEMMs (Q/K/V + output projection) TFLOP/s on 1 B200",
+        "value": flops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "S": S, "H": H, "Hq": Hq, "Hkv": Hkv, "D": D, "model_flops_per_step": flops,
+                   "l2": "inputs larger than L2 (X + weights + A = %.0f MB)" % (
+                       (2 * S * H + 2 * H * (Hq + 2 * Hkv) + 2 * S * Hq + 2 * H * Hq) / 1e6)},
+        "clocks": sampler.summary(), "gpu_launches": int(2 * args.steps), "e2e": None,
+        "roofline": {"bound": "tensor", "kernel": "pair_gemm_kernel<PairQkvPolicy>", "achieved": achieved,
+                     "peak": peaks["burst"], "unit": UNIT, "frac": achieved / peaks["burst"],
+                     "peak_source": f"of {peaks['source']} (burst bf16 GEMM)", "traffic": None,
+                     "kernels_ms": {"pair_gemm_kernel<PairQkvPolicy>": qkv_ms, "pair_gemm_kernel<PairOutPolicy>": out_ms},
+                     "out_projection_tflops": wl.out_flops() / (out_ms * 1e-3) / 1e12},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    b.tsp_attn_plan_destroy(plan)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="7b_short", choices=sorted(inp.WORKLOADS))
+    ap.add_argument("--workload", default="7b_short", choices=sorted(inp.WORKLOADS) + sorted(inp.ATTN_WORKLOADS))
     ap.add_argument("--backward", action="store_true", help="time forward + backward (as the `train` workload does)")
     ap.add_argument("--stored-activations", action="store_true",
                     help="training step through tsp_mlp_forward_save / tsp_mlp_backward_saved (no recomputation)")
@@ -556,6 +647,10 @@ def main():
     ap.add_argument("--no-context", action="store_true", help="skip the torch-eager context measurement")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()
+    if args.workload in inp.ATTN_WORKLOADS:
+        if args.impl == "reference":
+            raise SystemExit("the reference arm covers the gated-MLP workloads")
+        return run_attn(args, inp.ATTN_WORKLOADS[args.workload])
     wl = inp.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)
