@@ -21,6 +21,14 @@ projection matrices and the loop reaches exactly the unsharded result:
 
     Q = X Wq^T [S, Hq]   K = X Wk^T [S, Hkv]   V = X Wv^T [S, Hkv]       Y = A Wo^T [S, H],   Wo = [Wo^(0) | .. | Wo^(D-1)]
 
+Backward (the paper only says that the backward pass mirrors the forward weight movement and that the partial
+weight gradients the ranks produce for a shard are summed to its owner, Sections 4.3.4 and 4.7): the derivatives of
+the two definitions for upstream gradients dQ, dK, dV and dY,
+
+    dX = dQ Wq + dK Wk + dV Wv      dWq = dQ^T X   dWk = dK^T X   dWv = dV^T X      dA = dY Wo      dWo = dY^T A
+
+with the sums over tokens running over ALL ranks' tokens (that is the sum-to-owner).
+
 Each step is given twice: the plain definition, and the loop of Algorithm 1 written out shard by shard (the tests
 prove the two agree for every D).  Everything is float64 on the bf16-rounded input values.  Every function is
 pinned by tests/test_attn_oracle_pins.py (brute force with exact summation, closed forms, invariants); none is
@@ -74,3 +82,55 @@ def qkv_rows(X, Wq, Wk, Wv, rows):
 
 def output_rows(A, Wo, rows):
     return output_projection(A[rows], Wo)
+
+
+# ----------------------------------------------------------------------------------------
+# backward
+# ----------------------------------------------------------------------------------------
+def qkv_projection_backward(X, Wq, Wk, Wv, dQ, dK, dV):
+    """Gradients of L = <dQ, Q> + <dK, K> + <dV, V>: returns dX [S, H], dWq [Hq, H], dWk, dWv [Hkv, H]."""
+    dX = dQ @ Wq + dK @ Wk + dV @ Wv
+    return dX, dQ.T @ X, dK.T @ X, dV.T @ X
+
+
+def output_projection_backward(A, Wo, dY):
+    """Gradients of L = <dY, Y>: returns dA [S, Hq] and dWo [H, Hq]."""
+    return dY @ Wo, dY.T @ A
+
+
+def sharded_qkv_projection_backward(X_ranks, Wq_shards, Wk_shards, Wv_shards, dQ_ranks, dK_ranks, dV_ranks):
+    """The same gradients formed the way the sharded schedule forms them.
+
+    X_ranks[p] [S_loc, H] are rank p's tokens, dQ_ranks[p] [S_loc, Hq] etc. its upstream gradients.  In iteration r
+    every rank p adds shard r's term to its dX and produces a partial gradient for shard r's rows; the partials of
+    all ranks are summed to the owner r.  Returns (list of dX per rank, dWq, dWk, dWv stacked in shard order).
+    """
+    D, P = len(Wq_shards), len(X_ranks)
+    q_w, kv_w = Wq_shards[0].shape[0], Wk_shards[0].shape[0]
+    dX = [np.zeros_like(X_ranks[p]) for p in range(P)]
+    dWq = [np.zeros_like(Wq_shards[r]) for r in range(D)]
+    dWk = [np.zeros_like(Wk_shards[r]) for r in range(D)]
+    dWv = [np.zeros_like(Wv_shards[r]) for r in range(D)]
+    for r in range(D):
+        q_cols, kv_cols = slice(r * q_w, (r + 1) * q_w), slice(r * kv_w, (r + 1) * kv_w)
+        for p in range(P):
+            dq, dk, dv = dQ_ranks[p][:, q_cols], dK_ranks[p][:, kv_cols], dV_ranks[p][:, kv_cols]
+            dX[p] = dX[p] + dq @ Wq_shards[r] + dk @ Wk_shards[r] + dv @ Wv_shards[r]
+            dWq[r] = dWq[r] + dq.T @ X_ranks[p]       # partial of rank p, summed to owner r
+            dWk[r] = dWk[r] + dk.T @ X_ranks[p]
+            dWv[r] = dWv[r] + dv.T @ X_ranks[p]
+    return dX, np.concatenate(dWq, axis=0), np.concatenate(dWk, axis=0), np.concatenate(dWv, axis=0)
+
+
+def sharded_output_projection_backward(A_ranks, Wo_shards, dY_ranks):
+    """dA per rank (heads of shard r in columns r*Hq/D ..) and dWo shards summed over the ranks' tokens."""
+    D, P = len(Wo_shards), len(A_ranks)
+    w = Wo_shards[0].shape[1]
+    dA = [np.zeros_like(A_ranks[p]) for p in range(P)]
+    dWo = [np.zeros_like(Wo_shards[r]) for r in range(D)]
+    for r in range(D):
+        cols = slice(r * w, (r + 1) * w)
+        for p in range(P):
+            dA[p][:, cols] = dY_ranks[p] @ Wo_shards[r]
+            dWo[r] = dWo[r] + dY_ranks[p].T @ A_ranks[p][:, cols]
+    return dA, dWo

@@ -146,3 +146,101 @@ def test_input_recipe_statistics_and_determinism():
     Y = orc.output_projection(inp.bf16_bits_to_f64(a.A), inp.bf16_bits_to_f64(a.Wo))
     assert abs(Y.std() - 1.0) < 0.05
     assert inp.shard_out_columns(a.Wo, 4).shape == (4, 128, 64)
+
+
+# ----------------------------------------------------------------------------------------------------- backward
+def _brute_aTb(A, B):
+    """out[i, j] = sum_s A[s, i] * B[s, j] with exactly rounded sums."""
+    return np.array([[math.fsum(float(A[s, i]) * float(B[s, j]) for s in range(A.shape[0])) for j in range(B.shape[1])]
+                     for i in range(A.shape[1])])
+
+
+def test_backward_brute_force():
+    r = _rng(10)
+    S, H, Hq, Hkv = 4, 5, 6, 2
+    X, Wq, Wk, Wv = r.standard_normal((S, H)), r.standard_normal((Hq, H)), r.standard_normal((Hkv, H)), \
+        r.standard_normal((Hkv, H))
+    dQ, dK, dV = r.standard_normal((S, Hq)), r.standard_normal((S, Hkv)), r.standard_normal((S, Hkv))
+    dX, dWq, dWk, dWv = orc.qkv_projection_backward(X, Wq, Wk, Wv, dQ, dK, dV)
+    # dX[s, h] = sum_j dQ[s, j] Wq[j, h] + ... : brute force via the transposed weights
+    ref_dX = _brute_xwT(dQ, Wq.T) + _brute_xwT(dK, Wk.T) + _brute_xwT(dV, Wv.T)
+    np.testing.assert_allclose(dX, ref_dX, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(dWq, _brute_aTb(dQ, X), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(dWk, _brute_aTb(dK, X), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(dWv, _brute_aTb(dV, X), rtol=0, atol=1e-13)
+    A, Wo, dY = r.standard_normal((S, Hq)), r.standard_normal((H, Hq)), r.standard_normal((S, H))
+    dA, dWo = orc.output_projection_backward(A, Wo, dY)
+    np.testing.assert_allclose(dA, _brute_xwT(dY, Wo.T), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(dWo, _brute_aTb(dY, A), rtol=0, atol=1e-13)
+
+
+def test_backward_finite_differences():
+    r = _rng(11)
+    S, H, Hq, Hkv = 5, 6, 8, 4
+    X, Wq, Wk, Wv = r.standard_normal((S, H)), r.standard_normal((Hq, H)), r.standard_normal((Hkv, H)), \
+        r.standard_normal((Hkv, H))
+    dQ, dK, dV = r.standard_normal((S, Hq)), r.standard_normal((S, Hkv)), r.standard_normal((S, Hkv))
+
+    def loss(X_, Wq_, Wk_, Wv_):
+        Q, K, V = orc.qkv_projection(X_, Wq_, Wk_, Wv_)
+        return float((dQ * Q).sum() + (dK * K).sum() + (dV * V).sum())
+
+    grads = orc.qkv_projection_backward(X, Wq, Wk, Wv, dQ, dK, dV)
+    args = [X, Wq, Wk, Wv]
+    eps = 1e-5
+    for which in range(4):
+        Vdir = r.standard_normal(args[which].shape)
+        plus = [a + eps * Vdir if i == which else a for i, a in enumerate(args)]
+        minus = [a - eps * Vdir if i == which else a for i, a in enumerate(args)]
+        fd = (loss(*plus) - loss(*minus)) / (2 * eps)
+        assert abs(fd - float((grads[which] * Vdir).sum())) <= 1e-7 * max(1.0, abs(fd))
+    A, Wo, dY = r.standard_normal((S, Hq)), r.standard_normal((H, Hq)), r.standard_normal((S, H))
+    dA, dWo = orc.output_projection_backward(A, Wo, dY)
+    for which, g in ((0, dA), (1, dWo)):
+        Vdir = r.standard_normal(g.shape)
+        f = lambda e: float((dY * orc.output_projection(A + e * Vdir if which == 0 else A,
+                                                        Wo + e * Vdir if which == 1 else Wo)).sum())
+        fd = (f(eps) - f(-eps)) / (2 * eps)
+        assert abs(fd - float((g * Vdir).sum())) <= 1e-7 * max(1.0, abs(fd))
+
+
+def test_backward_adjoint_identities():
+    # the layers are bilinear: <dWo, Wo> = <dA, A> = <dY, Y>, and <dX, X> = <dWq, Wq> + <dWk, Wk> + <dWv, Wv> = L
+    r = _rng(12)
+    S, H, Hq, Hkv = 7, 6, 10, 5
+    X, Wq, Wk, Wv = r.standard_normal((S, H)), r.standard_normal((Hq, H)), r.standard_normal((Hkv, H)), \
+        r.standard_normal((Hkv, H))
+    dQ, dK, dV = r.standard_normal((S, Hq)), r.standard_normal((S, Hkv)), r.standard_normal((S, Hkv))
+    Q, K, V = orc.qkv_projection(X, Wq, Wk, Wv)
+    L = (dQ * Q).sum() + (dK * K).sum() + (dV * V).sum()
+    dX, dWq, dWk, dWv = orc.qkv_projection_backward(X, Wq, Wk, Wv, dQ, dK, dV)
+    assert abs((dX * X).sum() - L) <= 1e-12 * abs(L)
+    assert abs((dWq * Wq).sum() + (dWk * Wk).sum() + (dWv * Wv).sum() - L) <= 1e-12 * abs(L)
+    assert abs((dWq * Wq).sum() - (dQ * Q).sum()) <= 1e-12 * abs(L)
+    A, Wo, dY = r.standard_normal((S, Hq)), r.standard_normal((H, Hq)), r.standard_normal((S, H))
+    LY = (dY * orc.output_projection(A, Wo)).sum()
+    dA, dWo = orc.output_projection_backward(A, Wo, dY)
+    assert abs((dA * A).sum() - LY) <= 1e-12 * abs(LY) and abs((dWo * Wo).sum() - LY) <= 1e-12 * abs(LY)
+    # zero upstream gradient -> zero gradients
+    z = orc.qkv_projection_backward(X, Wq, Wk, Wv, 0 * dQ, 0 * dK, 0 * dV)
+    assert not any(g.any() for g in z)
+
+
+@pytest.mark.parametrize("D", [1, 2, 4])
+def test_sharded_backward_sums_to_owner(D):
+    r = _rng(13)
+    S, H, Hq, Hkv = 8, 6, 8, 4
+    X, Wq, Wk, Wv = r.standard_normal((S, H)), r.standard_normal((Hq, H)), r.standard_normal((Hkv, H)), \
+        r.standard_normal((Hkv, H))
+    dQ, dK, dV = r.standard_normal((S, Hq)), r.standard_normal((S, Hkv)), r.standard_normal((S, Hkv))
+    ranks = lambda M: [M[p * (S // D):(p + 1) * (S // D)] for p in range(D)]
+    dXs, dWq, dWk, dWv = orc.sharded_qkv_projection_backward(ranks(X), _shard_rows(Wq, D), _shard_rows(Wk, D),
+                                                             _shard_rows(Wv, D), ranks(dQ), ranks(dK), ranks(dV))
+    ref = orc.qkv_projection_backward(X, Wq, Wk, Wv, dQ, dK, dV)
+    for got, want in zip((np.concatenate(dXs, axis=0), dWq, dWk, dWv), ref):
+        np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    A, Wo, dY = r.standard_normal((S, Hq)), r.standard_normal((H, Hq)), r.standard_normal((S, H))
+    dAs, dWos = orc.sharded_output_projection_backward(ranks(A), _shard_cols(Wo, D), ranks(dY))
+    rdA, rdWo = orc.output_projection_backward(A, Wo, dY)
+    np.testing.assert_allclose(np.concatenate(dAs, axis=0), rdA, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(np.concatenate(dWos, axis=1), rdWo, rtol=1e-12, atol=1e-12)
