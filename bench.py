@@ -590,8 +590,8 @@ def run_attn(args, wl):
     sampler.stop()
     assert b.tsp_attn_status(plan) == b.TSP_OK, "device-side wait timed out"
     ms_per_step = e0.elapsed_time(e1) / args.steps
-    qkv_ms = float(np.mean([b.tsp_attn_profile_read(plan, i) for i in range(0, n_prof, 2)]))
-    out_ms = float(np.mean([b.tsp_attn_profile_read(plan, i) for i in range(1, n_prof, 2)]))
+    qkv_ms = float(np.mean([b.tsp_attn_profile_read(plan, i)[0] for i in range(0, n_prof, 2)]))
+    out_ms = float(np.mean([b.tsp_attn_profile_read(plan, i)[0] for i in range(1, n_prof, 2)]))
     b.tsp_attn_profile_end(plan)
     flops = wl.qkv_flops() + wl.out_flops()
     peaks = measured_peaks()

@@ -7,7 +7,7 @@
  * and, after attention on those heads, adds their output through shard r of the output projection,
  *     Y <- Y + Flatten(A) W_O^(r)T                             W_O^(r) in R^{h x (h/D)},  Y starts at 0.
  * These entry points compute the two dense steps for all D shards resident on ONE GPU (no broadcast, no
- * collective); the attention core between them is not part of this library.
+ * collective), forward and backward; the attention core between them is not part of this library.
  *
  * Layouts (DEVICE pointers, row-major bf16, inputs 16-byte aligned, outputs 32-byte aligned):
  *     X        [S, H]               tokens of every rank (the projections are row-wise: any token order)
@@ -60,12 +60,34 @@ tsp_status_t tsp_attn_qkv_forward(tsp_attn_plan_t* plan, const void* X, const vo
 tsp_status_t tsp_attn_out_forward(tsp_attn_plan_t* plan, const void* A, const void* Wo, void* Y, int64_t S, int D,
                                   void* cuda_stream);
 
+/*
+ * Backward of the two steps (the backward pass mirrors the forward weight movement; the partial weight gradients
+ * the ranks produce for a shard are summed to its owner: Sections 4.3.4 and 4.7 - here all ranks' tokens are
+ * resident, so the sum over ranks is the contraction over all S tokens, in ascending token order).
+ *
+ * tsp_attn_qkv_backward: for upstream dQ [S, Hq], dK, dV [S, Hkv] (bf16):
+ *     dX  = dQ Wq + dK Wk + dV Wv                [S, H] bf16 (fp32 accumulation over all features, one rounding)
+ *     dWq = dQ^T X, dWk = dK^T X, dWv = dV^T X   fp32, in the layouts of Wq, Wk, Wv, overwritten
+ *   Two kernels.
+ * tsp_attn_out_backward: for upstream dY [S, H] (bf16):
+ *     dA  = dY Wo                                [S, Hq] bf16, heads of shard r in columns r*Hq/D ..
+ *     dWo = dY^T A                               fp32 [D][H][Hq/D], overwritten
+ *   Two kernels.
+ * Errors as for the forward calls; fp32 outputs must be 32-byte aligned.
+ */
+tsp_status_t tsp_attn_qkv_backward(tsp_attn_plan_t* plan, const void* X, const void* Wq, const void* Wk, const void* Wv,
+                                   const void* dQ, const void* dK, const void* dV, void* dX, float* dWq, float* dWk,
+                                   float* dWv, int64_t S, int D, void* cuda_stream);
+tsp_status_t tsp_attn_out_backward(tsp_attn_plan_t* plan, const void* A, const void* Wo, const void* dY, void* dA,
+                                   float* dWo, int64_t S, int D, void* cuda_stream);
+
 /* Device status word (after the stream has been synchronized): TSP_OK or TSP_ERR_DEVICE_TIMEOUT; clears it. */
 tsp_status_t tsp_attn_status(tsp_attn_plan_t* plan);
 
-/* Per-kernel timing with CUDA events on the launch stream, as tsp_mlp_profile_*: one kernel per call. */
+/* Per-kernel timing with CUDA events on the launch stream, as tsp_mlp_profile_*: a forward call records one
+ * kernel, a backward call two; ms_out must have room for 8 floats. */
 tsp_status_t tsp_attn_profile_begin(tsp_attn_plan_t* plan, int max_calls);
-tsp_status_t tsp_attn_profile_read(tsp_attn_plan_t* plan, int call_index, float* ms_out);
+tsp_status_t tsp_attn_profile_read(tsp_attn_plan_t* plan, int call_index, int* n_kernels_out, float* ms_out);
 tsp_status_t tsp_attn_profile_end(tsp_attn_plan_t* plan);
 
 #ifdef __cplusplus

@@ -58,7 +58,10 @@ SIGNATURES = {
     "tsp_attn_out_forward": (ctypes.c_int, [_P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_attn_status": (ctypes.c_int, [_P]),
     "tsp_attn_profile_begin": (ctypes.c_int, [_P, ctypes.c_int]),
-    "tsp_attn_profile_read": (ctypes.c_int, [_P, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]),
+    "tsp_attn_profile_read": (ctypes.c_int, [_P, ctypes.c_int, ctypes.POINTER(ctypes.c_int),
+                                             ctypes.POINTER(ctypes.c_float)]),
+    "tsp_attn_qkv_backward": (ctypes.c_int, [_P] * 12 + [ctypes.c_int64, ctypes.c_int, _P]),
+    "tsp_attn_out_backward": (ctypes.c_int, [_P] * 6 + [ctypes.c_int64, ctypes.c_int, _P]),
     "tsp_attn_profile_end": (ctypes.c_int, [_P]),
     "tsp_mlp_selftest_wait_expiry": (ctypes.c_int, [_P, ctypes.c_int, _P]),
     "tsp_mlp_status": (ctypes.c_int, [_P]),
@@ -318,10 +321,23 @@ def tsp_attn_profile_begin(plan, max_calls: int) -> None:
     _check(load_library().tsp_attn_profile_begin(plan, max_calls), "tsp_attn_profile_begin")
 
 
-def tsp_attn_profile_read(plan, call_index: int) -> float:
-    ms = ctypes.c_float()
-    _check(load_library().tsp_attn_profile_read(plan, call_index, ctypes.byref(ms)), "tsp_attn_profile_read")
-    return float(ms.value)
+def tsp_attn_profile_read(plan, call_index: int) -> list[float]:
+    """Kernel durations (ms) of one recorded call: one value for a forward call, two for a backward call."""
+    n = ctypes.c_int()
+    ms = (ctypes.c_float * 8)()
+    _check(load_library().tsp_attn_profile_read(plan, call_index, ctypes.byref(n), ms), "tsp_attn_profile_read")
+    return [float(ms[i]) for i in range(n.value)]
+
+
+def tsp_attn_qkv_backward(plan, X, Wq, Wk, Wv, dQ, dK, dV, dX, dWq, dWk, dWv, S: int, D: int, stream=None) -> None:
+    _check(load_library().tsp_attn_qkv_backward(plan, _ptr(X), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(dQ), _ptr(dK),
+                                                _ptr(dV), _ptr(dX), _ptr(dWq), _ptr(dWk), _ptr(dWv), S, D,
+                                                _stream_handle(stream)), "tsp_attn_qkv_backward")
+
+
+def tsp_attn_out_backward(plan, A, Wo, dY, dA, dWo, S: int, D: int, stream=None) -> None:
+    _check(load_library().tsp_attn_out_backward(plan, _ptr(A), _ptr(Wo), _ptr(dY), _ptr(dA), _ptr(dWo), S, D,
+                                                _stream_handle(stream)), "tsp_attn_out_backward")
 
 
 def tsp_attn_profile_end(plan) -> None:

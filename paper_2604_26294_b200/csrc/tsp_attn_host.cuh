@@ -97,19 +97,121 @@ tsp_status_t tsp_attn_out_forward(tsp_attn_plan_t* plan, const void* A, const vo
     return st;
 }
 
+tsp_status_t tsp_attn_qkv_backward(tsp_attn_plan_t* plan, const void* X, const void* Wq, const void* Wk, const void* Wv,
+                                   const void* dQ, const void* dK, const void* dV, void* dX, float* dWq, float* dWk,
+                                   float* dWv, int64_t S, int D, void* cuda_stream) {
+    if (!plan || D != plan->D || S < 1) return TSP_ERR_INVALID_ARG;
+    if (S > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X || !Wq || !Wk || !Wv || !dQ || !dK || !dV || !dX || !dWq || !dWk || !dWv) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(dQ) || !aligned16(dK) ||
+        !aligned16(dV) || !aligned32(dX) || !aligned32(dWq) || !aligned32(dWk) || !aligned32(dWv))
+        return TSP_ERR_INVALID_ARG;
+    tsp_mlp_plan_t* base = plan->base;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int H = plan->H, Hq = plan->Hq, Hkv = plan->Hkv;
+    Profiler prof(base, stream);
+    {
+        tsp::PairAttnDxPolicy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(base, &p.map_dq, dQ, S, Hq, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_dk, dK, S, Hkv, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_dv, dV, S, Hkv, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_wq, Wq, Hq, H, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_wk, Wk, Hkv, H, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_wv, Wv, Hkv, H, 64, 64)) return TSP_ERR_CUDA;
+        p.dX = static_cast<__nv_bfloat16*>(dX);
+        p.S = static_cast<int>(S); p.H = H;
+        p.q_kb = Hq / 64; p.kv_kb = Hkv / 64;
+        p.m_tiles = static_cast<int>((S + 255) / 256);
+        p.n_blocks = H / 256;
+        const int group = base->dx_group > 0 ? base->dx_group : 8;
+        p.group = p.m_tiles < group ? p.m_tiles : group;
+        fill_common(base, p, p.m_tiles * p.n_blocks);
+        tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDxPolicy>, p, stream);
+        if (st != TSP_OK) return st;
+        prof.mark();
+    }
+    {
+        tsp::PairAttnDwPolicy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(base, &p.map_m0, dQ, S, Hq, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_m1, dK, S, Hkv, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_m2, dV, S, Hkv, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_n, X, S, H, 64, 64)) return TSP_ERR_CUDA;
+        p.out0 = dWq; p.out1 = dWk; p.out2 = dWv;
+        p.m_tiles0 = Hq / 256; p.m_tiles1 = Hkv / 256; p.m_tiles2 = Hkv / 256;
+        p.rows0 = Hq; p.N = H; p.shard_w = 0;
+        p.S = static_cast<int>(S);
+        p.k_blocks = static_cast<int>((S + 63) / 64);
+        p.n_blocks = H / 256;
+        int n_group = base->dw_group > 0 ? base->dw_group : static_cast<int>((64ull << 20) / (512ull * static_cast<size_t>(S)));
+        if (n_group < 1) n_group = 1;
+        p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
+        fill_common(base, p, (p.m_tiles0 + p.m_tiles1 + p.m_tiles2) * p.n_blocks);
+        tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDwPolicy>, p, stream);
+        if (st != TSP_OK) return st;
+        prof.mark();
+    }
+    return TSP_OK;
+}
+
+tsp_status_t tsp_attn_out_backward(tsp_attn_plan_t* plan, const void* A, const void* Wo, const void* dY, void* dA,
+                                   float* dWo, int64_t S, int D, void* cuda_stream) {
+    if (!plan || D != plan->D || S < 1) return TSP_ERR_INVALID_ARG;
+    if (S > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!A || !Wo || !dY || !dA || !dWo) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(Wo) || !aligned16(dY) || !aligned32(dA) || !aligned32(dWo)) return TSP_ERR_INVALID_ARG;
+    tsp_mlp_plan_t* base = plan->base;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int H = plan->H, Hq = plan->Hq, Hq_d = plan->Hq / plan->D;
+    Profiler prof(base, stream);
+    {
+        tsp::PairAttnDaPolicy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(base, &p.map_dy, dY, S, H, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_sharded(base, &p.map_wo, Wo, D, H, Hq_d, 64, 64)) return TSP_ERR_CUDA;
+        p.dA = static_cast<__nv_bfloat16*>(dA);
+        p.S = static_cast<int>(S); p.H = H; p.Hq = Hq; p.Hq_d = Hq_d;
+        p.m_tiles = static_cast<int>((S + 255) / 256);
+        p.n_blocks = Hq / 256;
+        p.band = gate_band(base, p.m_tiles);
+        fill_common(base, p, p.m_tiles * p.n_blocks);
+        tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDaPolicy>, p, stream);
+        if (st != TSP_OK) return st;
+        prof.mark();
+    }
+    {
+        tsp::PairAttnDwPolicy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(base, &p.map_m0, dY, S, H, 64, 64)) return TSP_ERR_CUDA;
+        p.map_m1 = p.map_m0;
+        p.map_m2 = p.map_m0;
+        if (!encode_matrix(base, &p.map_n, A, S, Hq, 64, 64)) return TSP_ERR_CUDA;
+        p.out0 = dWo; p.out1 = dWo; p.out2 = dWo;
+        p.m_tiles0 = H / 256; p.m_tiles1 = 0; p.m_tiles2 = 0;
+        p.rows0 = H; p.N = Hq; p.shard_w = Hq_d;
+        p.S = static_cast<int>(S);
+        p.k_blocks = static_cast<int>((S + 63) / 64);
+        p.n_blocks = Hq / 256;
+        int n_group = base->dw_group > 0 ? base->dw_group : static_cast<int>((64ull << 20) / (512ull * static_cast<size_t>(S)));
+        if (n_group < 1) n_group = 1;
+        p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
+        fill_common(base, p, p.m_tiles0 * p.n_blocks);
+        tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDwPolicy>, p, stream);
+        if (st != TSP_OK) return st;
+        prof.mark();
+    }
+    return TSP_OK;
+}
+
 tsp_status_t tsp_attn_status(tsp_attn_plan_t* plan) { return plan ? tsp_mlp_status(plan->base) : TSP_ERR_INVALID_ARG; }
 
 tsp_status_t tsp_attn_profile_begin(tsp_attn_plan_t* plan, int max_calls) {
     return plan ? tsp_mlp_profile_begin(plan->base, max_calls) : TSP_ERR_INVALID_ARG;
 }
-tsp_status_t tsp_attn_profile_read(tsp_attn_plan_t* plan, int call_index, float* ms_out) {
-    if (!plan || !ms_out) return TSP_ERR_INVALID_ARG;
-    int n = 0;
-    float ms[kMaxKernelsPerCall] = {};
-    tsp_status_t st = tsp_mlp_profile_read(plan->base, call_index, &n, ms);
-    if (st != TSP_OK) return st;
-    *ms_out = n >= 1 ? ms[0] : 0.0f;
-    return TSP_OK;
+tsp_status_t tsp_attn_profile_read(tsp_attn_plan_t* plan, int call_index, int* n_kernels_out, float* ms_out) {
+    if (!plan) return TSP_ERR_INVALID_ARG;
+    return tsp_mlp_profile_read(plan->base, call_index, n_kernels_out, ms_out);
 }
 tsp_status_t tsp_attn_profile_end(tsp_attn_plan_t* plan) {
     return plan ? tsp_mlp_profile_end(plan->base) : TSP_ERR_INVALID_ARG;

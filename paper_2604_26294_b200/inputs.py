@@ -212,10 +212,15 @@ class AttnInputs:
     Wv: np.ndarray  # [Hkv, H]
     A: np.ndarray   # [S, Hq]   stand-in for the attention output fed to the output projection
     Wo: np.ndarray  # [H, Hq]
+    dQ: np.ndarray | None = None  # [S, Hq]   upstream gradients (stand-ins for what attention's backward hands over)
+    dK: np.ndarray | None = None  # [S, Hkv]
+    dV: np.ndarray | None = None  # [S, Hkv]
+    dY: np.ndarray | None = None  # [S, H]
 
 
-def make_attn_inputs(S: int, H: int, Hq: int, Hkv: int, seed: int = 0) -> AttnInputs:
-    """Draw order X, Wq, Wk, Wv, A, Wo; X, A ~ N(0,1); Wq, Wk, Wv ~ N(0, var 1/H); Wo ~ N(0, var 1/Hq)."""
+def make_attn_inputs(S: int, H: int, Hq: int, Hkv: int, seed: int = 0, with_grads: bool = False) -> AttnInputs:
+    """Draw order X, Wq, Wk, Wv, A, Wo (then dQ, dK, dV, dY); X, A, gradients ~ N(0,1); Wq, Wk, Wv ~ N(0, var 1/H);
+    Wo ~ N(0, var 1/Hq)."""
     rng = np.random.Generator(np.random.Philox(seed))
     X = _draw_bf16(rng, (S, H), 1.0)
     Wq = _draw_bf16(rng, (Hq, H), H ** -0.5)
@@ -223,7 +228,13 @@ def make_attn_inputs(S: int, H: int, Hq: int, Hkv: int, seed: int = 0) -> AttnIn
     Wv = _draw_bf16(rng, (Hkv, H), H ** -0.5)
     A = _draw_bf16(rng, (S, Hq), 1.0)
     Wo = _draw_bf16(rng, (H, Hq), Hq ** -0.5)
-    return AttnInputs(X, Wq, Wk, Wv, A, Wo)
+    out = AttnInputs(X, Wq, Wk, Wv, A, Wo)
+    if with_grads:
+        out.dQ = _draw_bf16(rng, (S, Hq), 1.0)
+        out.dK = _draw_bf16(rng, (S, Hkv), 1.0)
+        out.dV = _draw_bf16(rng, (S, Hkv), 1.0)
+        out.dY = _draw_bf16(rng, (S, H), 1.0)
+    return out
 
 
 def shard_out_columns(Wo: np.ndarray, D: int) -> np.ndarray:

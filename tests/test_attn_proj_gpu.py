@@ -150,3 +150,91 @@ def test_full_size_sampled_rows(name):
         assert rel_fro(g, ref) <= TOL
         assert worst_row_error(g, ref) <= 0.05
         assert bool(__import__("torch").isfinite(got.float()).all())
+
+
+# ------------------------------------------------------------------------------------------------------ backward
+def _run_backward(S, H, Hq, Hkv, D, seed=0):
+    import torch
+
+    host = inp.make_attn_inputs(S, H, Hq, Hkv, seed=seed, with_grads=True)
+    X, Wq, Wk, Wv, A = (bf16_tensor(a) for a in (host.X, host.Wq, host.Wk, host.Wv, host.A))
+    dQ, dK, dV, dY = (bf16_tensor(a) for a in (host.dQ, host.dK, host.dV, host.dY))
+    Wo = bf16_tensor(inp.shard_out_columns(host.Wo, D))
+    nan = float("nan")
+    dX = torch.full((S, H), nan, dtype=torch.bfloat16, device="cuda")
+    dA = torch.full((S, Hq), nan, dtype=torch.bfloat16, device="cuda")
+    dWq = torch.full((Hq, H), nan, dtype=torch.float32, device="cuda")
+    dWk = torch.full((Hkv, H), nan, dtype=torch.float32, device="cuda")
+    dWv = torch.full((Hkv, H), nan, dtype=torch.float32, device="cuda")
+    dWo = torch.full((D, H, Hq // D), nan, dtype=torch.float32, device="cuda")
+    plan = b.tsp_attn_plan(H, Hq, Hkv, D)
+    try:
+        b.tsp_attn_out_backward(plan, A, Wo, dY, dA, dWo, S, D)
+        b.tsp_attn_qkv_backward(plan, X, Wq, Wk, Wv, dQ, dK, dV, dX, dWq, dWk, dWv, S, D)
+        torch.cuda.synchronize()
+        assert b.tsp_attn_status(plan) == b.TSP_OK
+    finally:
+        b.tsp_attn_plan_destroy(plan)
+    return host, dX, dWq, dWk, dWv, dA, dWo
+
+
+@pytest.mark.parametrize("S,H,Hq,Hkv,D", [
+    (256, 256, 512, 256, 2),
+    (512, 256, 256, 256, 1),
+    (768, 512, 1024, 256, 4),
+    (1024, 256, 1536, 768, 3),
+    (1000, 256, 512, 512, 8),      # ragged token tail (also inside the last 64-token k-block), shard width 64
+    (77, 512, 256, 256, 2),
+    (4160, 256, 256, 256, 4),      # more token tiles than one group
+])
+def test_backward_matches_oracle(S, H, Hq, Hkv, D):
+    host, dX, dWq, dWk, dWv, dA, dWo = _run_backward(S, H, Hq, Hkv, D, seed=44)
+    f = _f64(host)
+    g = {n: inp.bf16_bits_to_f64(getattr(host, n)) for n in ("dQ", "dK", "dV", "dY")}
+    rdX, rdWq, rdWk, rdWv = orc.qkv_projection_backward(f["X"], f["Wq"], f["Wk"], f["Wv"], g["dQ"], g["dK"], g["dV"])
+    rdA, rdWo = orc.output_projection_backward(f["A"], f["Wo"], g["dY"])
+    got_dWo = inp.unshard_columns(tensor_to_f64(dWo))
+    for name, got, ref in (("dX", tensor_to_f64(dX), rdX), ("dA", tensor_to_f64(dA), rdA),
+                           ("dWq", tensor_to_f64(dWq), rdWq), ("dWk", tensor_to_f64(dWk), rdWk),
+                           ("dWv", tensor_to_f64(dWv), rdWv), ("dWo", got_dWo, rdWo)):
+        assert np.all(np.isfinite(got)), name
+        # bf16 outputs carry one rounding (1.7e-3); the fp32 weight gradients only fp32 accumulation error
+        tol = TOL if name in ("dX", "dA") else 1e-4
+        assert rel_fro(got, ref) <= tol, (name, rel_fro(got, ref))
+        assert worst_row_error(got, ref) <= 0.05, name
+
+
+def test_backward_is_deterministic_and_independent_of_shard_count():
+    import torch
+
+    S, H, Hq, Hkv = 512, 256, 1024, 512
+    ref = None
+    for D in (1, 4, 16, 4):
+        _, dX, dWq, dWk, dWv, dA, dWo = _run_backward(S, H, Hq, Hkv, D, seed=45)
+        cur = (dX.view(torch.int16), dWq, dWk, dWv, dA.view(torch.int16),
+               dWo.permute(1, 0, 2).reshape(H, Hq).contiguous())
+        if ref is None:
+            ref = cur
+        else:
+            for a, c in zip(ref, cur):
+                assert torch.equal(a, c)   # the shard count only changes where dWo's columns are stored
+
+
+def test_backward_argument_errors():
+    import torch
+
+    plan = b.tsp_attn_plan(256, 256, 256, 2)
+    try:
+        x = torch.zeros(256, 256, dtype=torch.bfloat16, device="cuda")
+        w = torch.zeros(256, 256, dtype=torch.float32, device="cuda")
+        with pytest.raises(b.TspError) as e:
+            b.tsp_attn_qkv_backward(plan, x, x, x, x, x, x, x, x, w, w, 0, 256, 2)
+        assert e.value.code == b.TSP_ERR_INVALID_ARG
+        with pytest.raises(b.TspError) as e:
+            b.tsp_attn_out_backward(plan, x, x, x, x, w.view(-1)[1:], 256, 2)     # fp32 output not 32-byte aligned
+        assert e.value.code == b.TSP_ERR_INVALID_ARG
+        with pytest.raises(b.TspError) as e:
+            b.tsp_attn_out_backward(plan, x, x, x, x, w, 256, 3)
+        assert e.value.code == b.TSP_ERR_INVALID_ARG
+    finally:
+        b.tsp_attn_plan_destroy(plan)
