@@ -556,7 +556,8 @@ def run_attn(args, wl):
     torch.cuda.set_device(0)
     _build.build_library()
     S, H, Hq, Hkv, D = wl.S, wl.H, wl.Hq, wl.Hkv, wl.D
-    host = inp.make_attn_inputs(S, H, Hq, Hkv, seed=0)
+    train = args.backward
+    host = inp.make_attn_inputs(S, H, Hq, Hkv, seed=0, with_grads=train)
 
     def dev(bits):
         return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
@@ -568,16 +569,27 @@ def run_attn(args, wl):
     V = torch.empty(S, Hkv, dtype=torch.bfloat16, device="cuda")
     Y = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
     plan = b.tsp_attn_plan(H, Hq, Hkv, D)
+    if train:
+        dQ, dK, dV, dY = dev(host.dQ), dev(host.dK), dev(host.dV), dev(host.dY)
+        dX, dA = torch.empty_like(X), torch.empty_like(A)
+        dWq = torch.empty(Hq, H, dtype=torch.float32, device="cuda")
+        dWk = torch.empty(Hkv, H, dtype=torch.float32, device="cuda")
+        dWv = torch.empty(Hkv, H, dtype=torch.float32, device="cuda")
+        dWo = torch.empty(D, H, Hq // D, dtype=torch.float32, device="cuda")
 
     def step():
         b.tsp_attn_qkv_forward(plan, X, Wq, Wk, Wv, Q, K, V, S, D)
         b.tsp_attn_out_forward(plan, A, Wo, Y, S, D)
+        if train:
+            b.tsp_attn_out_backward(plan, A, Wo, dY, dA, dWo, S, D)
+            b.tsp_attn_qkv_backward(plan, X, Wq, Wk, Wv, dQ, dK, dV, dX, dWq, dWk, dWv, S, D)
 
     for _ in range(max(3, args.warmup)):
         step()
     torch.cuda.synchronize()
     assert b.tsp_attn_status(plan) == b.TSP_OK
-    n_prof = min(4096, 2 * args.steps)
+    calls = 4 if train else 2
+    n_prof = min(4096, calls * args.steps)
     b.tsp_attn_profile_begin(plan, n_prof)
     sampler = ClockSampler(0)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -590,10 +602,18 @@ def run_attn(args, wl):
     sampler.stop()
     assert b.tsp_attn_status(plan) == b.TSP_OK, "device-side wait timed out"
     ms_per_step = e0.elapsed_time(e1) / args.steps
-    qkv_ms = float(np.mean([b.tsp_attn_profile_read(plan, i)[0] for i in range(0, n_prof, 2)]))
-    out_ms = float(np.mean([b.tsp_attn_profile_read(plan, i)[0] for i in range(1, n_prof, 2)]))
+    qkv_ms = float(np.mean([b.tsp_attn_profile_read(plan, i)[0] for i in range(0, n_prof, calls)]))
+    out_ms = float(np.mean([b.tsp_attn_profile_read(plan, i)[0] for i in range(1, n_prof, calls)]))
+    kernels_ms = {"pair_gemm_kernel<PairQkvPolicy>": qkv_ms, "pair_gemm_kernel<PairOutPolicy>": out_ms}
+    if train:
+        ob = np.mean([b.tsp_attn_profile_read(plan, i) for i in range(2, n_prof, calls)], axis=0)
+        qb = np.mean([b.tsp_attn_profile_read(plan, i) for i in range(3, n_prof, calls)], axis=0)
+        kernels_ms.update({"pair_gemm_kernel<PairAttnDaPolicy>": float(ob[0]),
+                           "pair_gemm_kernel<PairAttnDwPolicy> (dWo)": float(ob[1]),
+                           "pair_gemm_kernel<PairAttnDxPolicy>": float(qb[0]),
+                           "pair_gemm_kernel<PairAttnDwPolicy> (dWq, dWk, dWv)": float(qb[1])})
     b.tsp_attn_profile_end(plan)
-    flops = wl.qkv_flops() + wl.out_flops()
+    flops = (wl.qkv_flops() + wl.out_flops()) * (3.0 if train else 1.0)   # backward = twice the forward
     peaks = measured_peaks()
     achieved = wl.qkv_flops() / (qkv_ms * 1e-3) / 1e12
     # oracle timed on a bounded sample of rows (row-separable), host cores
@@ -608,21 +628,21 @@ def run_attn(args, wl):
             attn_orc.output_rows(f[4], f[5], rows)
             reps += 1
         dt = (time.perf_counter() - t0) / reps
-        cpu = {"value": flops * len(rows) / S / dt / 1e12, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
-               "kind": "oracle", "sample": f"{len(rows)} of {S} token rows, fp64, {reps} repetitions"}
+        cpu = {"value": (wl.qkv_flops() + wl.out_flops()) * len(rows) / S / dt / 1e12, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
+               "kind": "oracle", "sample": f"forward on {len(rows)} of {S} token rows, fp64, {reps} repetitions"}
     line = {
         "metric": "TSP attention projection GEMMs (Q/K/V + output projection) TFLOP/s on 1 B200",
         "value": flops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.name, "S": S, "H": H, "Hq": Hq, "Hkv": Hkv, "D": D, "model_flops_per_step": flops,
+        "config": {"workload": wl.name, "pass": "forward+backward" if train else "forward", "S": S, "H": H, "Hq": Hq, "Hkv": Hkv, "D": D, "model_flops_per_step": flops,
                    "l2": "inputs larger than L2 (X + weights + A = %.0f MB)" % (
                        (2 * S * H + 2 * H * (Hq + 2 * Hkv) + 2 * S * Hq + 2 * H * Hq) / 1e6)},
-        "clocks": sampler.summary(), "gpu_launches": int(2 * args.steps), "e2e": None,
+        "clocks": sampler.summary(), "gpu_launches": int((6 if train else 2) * args.steps), "e2e": None,
         "roofline": {"bound": "tensor", "kernel": "pair_gemm_kernel<PairQkvPolicy>", "achieved": achieved,
                      "peak": peaks["burst"], "unit": UNIT, "frac": achieved / peaks["burst"],
                      "peak_source": f"of {peaks['source']} (burst bf16 GEMM)", "traffic": None,
-                     "kernels_ms": {"pair_gemm_kernel<PairQkvPolicy>": qkv_ms, "pair_gemm_kernel<PairOutPolicy>": out_ms},
+                     "kernels_ms": kernels_ms,
                      "out_projection_tflops": wl.out_flops() / (out_ms * 1e-3) / 1e12},
         "cpu_baseline": cpu,
     }
