@@ -641,7 +641,10 @@ def run_attn(args, wl):
         "clocks": sampler.summary(), "gpu_launches": int((6 if train else 2) * args.steps), "e2e": None,
         "roofline": {"bound": "tensor", "kernel": "pair_gemm_kernel<PairQkvPolicy>", "achieved": achieved,
                      "peak": peaks["burst"], "unit": UNIT, "frac": achieved / peaks["burst"],
-                     "peak_source": f"of {peaks['source']} (burst bf16 GEMM)", "traffic": None,
+                     "peak_source": f"of {peaks['source']} (burst bf16 GEMM)",
+                     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the committed ncu capture
+                     "traffic": {"attn_7b_mha": 0.3305e9 + 0.1847e9}.get(wl.name),
+                     "algorithmic_bytes_per_launch": 2.0 * S * H + 2.0 * H * (Hq + 2 * Hkv) + 2.0 * S * (Hq + 2 * Hkv),
                      "kernels_ms": kernels_ms,
                      "out_projection_tflops": wl.out_flops() / (out_ms * 1e-3) / 1e12},
         "cpu_baseline": cpu,
