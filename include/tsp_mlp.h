@@ -107,7 +107,10 @@ tsp_status_t tsp_mlp_forward(tsp_mlp_plan_t* plan, const void* X, const void* Wg
  * recomputed from X; dA = dY Wd^T (kept in fp32); dU = dA*silu(G); dG = dA*U*silu'(G);
  * A, dG, dU are rounded once to bf16 into the workspace.  dX [S,H] bf16 accumulates over shards in
  * ring order; dWg, dWu [D][H][F/D] and dWd [D][F/D][H] are fp32 and contract over all S
- * tokens, rank order r = (k + t) mod D.
+ * tokens, rank order r = (k + t) mod D.  Beyond 2^18 tokens the token contraction of the weight
+ * gradients is cut into chunks of 2^18 tokens (ascending order, one launch per chunk, partial sums added
+ * in fp32 round-to-nearest): the tensor cores add into their accumulators with truncation, and an
+ * unbroken sum over millions of tokens would drift towards zero (about 2 % at 2^24 tokens).
  */
 tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu,
                               const void* Wd, const void* dY, void* dX, float* dWg, float* dWu,

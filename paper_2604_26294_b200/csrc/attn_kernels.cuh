@@ -256,6 +256,7 @@ struct PairAttnDwPolicy {
         int rows0;                         // rows of C of family 0 (needed for the sharded layout)
         int N;                             // columns of C
         int shard_w;                       // 0: C row-major [rows][N]; else C stored as [N / shard_w][rows][shard_w]
+        int accumulate;                    // 0: C overwritten; 1: the tile's sum is added to what C holds
         int S, k_blocks;
         int n_blocks, n_group;
         int num_tiles, stages;
@@ -315,6 +316,16 @@ struct PairAttnDwPolicy {
             } else {
                 const int r = col / p.shard_w;
                 dst = out + (static_cast<size_t>(r) * p.rows0 + j) * p.shard_w + (col - r * p.shard_w);
+            }
+            if (p.accumulate) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 prev = *reinterpret_cast<const float4*>(dst + q * 4);
+                    v[4 * q] = __float_as_uint(__uint_as_float(v[4 * q]) + prev.x);
+                    v[4 * q + 1] = __float_as_uint(__uint_as_float(v[4 * q + 1]) + prev.y);
+                    v[4 * q + 2] = __float_as_uint(__uint_as_float(v[4 * q + 2]) + prev.z);
+                    v[4 * q + 3] = __float_as_uint(__uint_as_float(v[4 * q + 3]) + prev.w);
+                }
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q)

@@ -372,6 +372,7 @@ struct BwdDwPolicy {
         float* dWu;          // [D][H][F/D]
         int S, H, F, D, S_loc;
         int k_linear;        // 0, or ceil(S / 64) when the tokens are contracted in ascending order (ragged ranks)
+        int accumulate;      // 0: dW overwritten; 1: the tile's sum is added to what dW holds
         int j_blocks, n_blocks, num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -416,16 +417,25 @@ struct BwdDwPolicy {
         if (tl.which == 0) {
             float4* dst = reinterpret_cast<float4*>(p.dWd + static_cast<size_t>(tl.jb * 128 + row) * p.H + tl.nb * 256 + c * 32);
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-                dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
-                                     __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+            for (int q = 0; q < 8; ++q) {
+                float4 o = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                       __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                if (p.accumulate) {
+                    const float4 prev = dst[q];
+                    o.x += prev.x; o.y += prev.y; o.z += prev.z; o.w += prev.w;
+                }
+                dst[q] = o;
+            }
         } else {
             const int F_d = p.F / p.D;
             float* base = (tl.which == 1 ? p.dWg : p.dWu) + static_cast<size_t>(tl.k) * p.H * F_d +
                           (tl.jb * 128 - tl.k * F_d) + row;
             const int h0 = tl.nb * 256 + c * 32;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) base[static_cast<size_t>(h0 + i) * F_d] = __uint_as_float(v[i]);
+            for (int i = 0; i < 32; ++i) {
+                float* dst = base + static_cast<size_t>(h0 + i) * F_d;
+                *dst = p.accumulate ? __uint_as_float(v[i]) + *dst : __uint_as_float(v[i]);
+            }
         }
     }
 };

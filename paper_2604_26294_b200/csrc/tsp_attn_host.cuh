@@ -131,27 +131,29 @@ tsp_status_t tsp_attn_qkv_backward(tsp_attn_plan_t* plan, const void* X, const v
         if (st != TSP_OK) return st;
         prof.mark();
     }
-    {
+    // weight gradients: token chunks, see for_token_chunks
+    tsp_status_t st = for_token_chunks(S, [&](int64_t c0, int64_t len, bool) {
         tsp::PairAttnDwPolicy::Params p;
         std::memset(&p, 0, sizeof(p));
-        if (!encode_matrix(base, &p.map_m0, dQ, S, Hq, 64, 64)) return TSP_ERR_CUDA;
-        if (!encode_matrix(base, &p.map_m1, dK, S, Hkv, 64, 64)) return TSP_ERR_CUDA;
-        if (!encode_matrix(base, &p.map_m2, dV, S, Hkv, 64, 64)) return TSP_ERR_CUDA;
-        if (!encode_matrix(base, &p.map_n, X, S, H, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_m0, row_offset(dQ, c0, Hq), len, Hq, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_m1, row_offset(dK, c0, Hkv), len, Hkv, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_m2, row_offset(dV, c0, Hkv), len, Hkv, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_n, row_offset(X, c0, H), len, H, 64, 64)) return TSP_ERR_CUDA;
         p.out0 = dWq; p.out1 = dWk; p.out2 = dWv;
         p.m_tiles0 = Hq / 256; p.m_tiles1 = Hkv / 256; p.m_tiles2 = Hkv / 256;
         p.rows0 = Hq; p.N = H; p.shard_w = 0;
-        p.S = static_cast<int>(S);
-        p.k_blocks = static_cast<int>((S + 63) / 64);
+        p.accumulate = c0 > 0;
+        p.S = static_cast<int>(len);
+        p.k_blocks = static_cast<int>((len + 63) / 64);
         p.n_blocks = H / 256;
-        int n_group = base->dw_group > 0 ? base->dw_group : static_cast<int>((64ull << 20) / (512ull * static_cast<size_t>(S)));
+        int n_group = base->dw_group > 0 ? base->dw_group : static_cast<int>((64ull << 20) / (512ull * static_cast<size_t>(len)));
         if (n_group < 1) n_group = 1;
         p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
         fill_common(base, p, (p.m_tiles0 + p.m_tiles1 + p.m_tiles2) * p.n_blocks);
-        tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDwPolicy>, p, stream);
-        if (st != TSP_OK) return st;
-        prof.mark();
-    }
+        return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDwPolicy>, p, stream);
+    });
+    if (st != TSP_OK) return st;
+    prof.mark();
     return TSP_OK;
 }
 
@@ -180,27 +182,28 @@ tsp_status_t tsp_attn_out_backward(tsp_attn_plan_t* plan, const void* A, const v
         if (st != TSP_OK) return st;
         prof.mark();
     }
-    {
+    tsp_status_t st = for_token_chunks(S, [&](int64_t c0, int64_t len, bool) {
         tsp::PairAttnDwPolicy::Params p;
         std::memset(&p, 0, sizeof(p));
-        if (!encode_matrix(base, &p.map_m0, dY, S, H, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_m0, row_offset(dY, c0, H), len, H, 64, 64)) return TSP_ERR_CUDA;
         p.map_m1 = p.map_m0;
         p.map_m2 = p.map_m0;
-        if (!encode_matrix(base, &p.map_n, A, S, Hq, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_matrix(base, &p.map_n, row_offset(A, c0, Hq), len, Hq, 64, 64)) return TSP_ERR_CUDA;
         p.out0 = dWo; p.out1 = dWo; p.out2 = dWo;
         p.m_tiles0 = H / 256; p.m_tiles1 = 0; p.m_tiles2 = 0;
         p.rows0 = H; p.N = Hq; p.shard_w = Hq_d;
-        p.S = static_cast<int>(S);
-        p.k_blocks = static_cast<int>((S + 63) / 64);
+        p.accumulate = c0 > 0;
+        p.S = static_cast<int>(len);
+        p.k_blocks = static_cast<int>((len + 63) / 64);
         p.n_blocks = Hq / 256;
-        int n_group = base->dw_group > 0 ? base->dw_group : static_cast<int>((64ull << 20) / (512ull * static_cast<size_t>(S)));
+        int n_group = base->dw_group > 0 ? base->dw_group : static_cast<int>((64ull << 20) / (512ull * static_cast<size_t>(len)));
         if (n_group < 1) n_group = 1;
         p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
         fill_common(base, p, p.m_tiles0 * p.n_blocks);
-        tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDwPolicy>, p, stream);
-        if (st != TSP_OK) return st;
-        prof.mark();
-    }
+        return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDwPolicy>, p, stream);
+    });
+    if (st != TSP_OK) return st;
+    prof.mark();
     return TSP_OK;
 }
 

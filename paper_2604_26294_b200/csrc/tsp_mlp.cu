@@ -282,7 +282,8 @@ tsp_status_t launch_bwd_dx(tsp_mlp_plan_t* plan, const void* dG, const void* dU,
 }
 
 tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
-                           const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream) {
+                           const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream,
+                           int accumulate = 0, bool linear = false) {
     const int H = plan->H, F = plan->F, D = plan->D;
     tsp::BwdDwPolicy::Params p;
     std::memset(&p, 0, sizeof(p));
@@ -294,7 +295,8 @@ tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, 
     p.dWd = dWd; p.dWg = dWg; p.dWu = dWu;
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.S_loc = static_cast<int>(S / D);
-    p.k_linear = (p.S_loc % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
+    p.k_linear = (linear || p.S_loc % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
+    p.accumulate = accumulate;
     p.j_blocks = F / 128;
     p.n_blocks = H / 256;
     p.num_tiles = 3 * p.j_blocks * p.n_blocks;
@@ -482,7 +484,7 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
 
 tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
                                 const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream,
-                                int accumulate = 0) {
+                                int accumulate = 0, bool linear = false) {
     const int H = plan->H, F = plan->F, D = plan->D;
     tsp::PairDwPolicy::Params p;
     std::memset(&p, 0, sizeof(p));
@@ -496,7 +498,7 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.F_d = F / D;
     p.S_loc = static_cast<int>(S / D);
-    p.k_linear = (p.S_loc % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
+    p.k_linear = (linear || p.S_loc % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
     p.j_tiles = F / 256;
     p.j_tiles_per_shard = p.F_d / 256;
     p.n_blocks = H / 256;
@@ -523,6 +525,46 @@ bool pairs_for_tokens(const tsp_mlp_plan_t* plan, int64_t S) {
     return padded_pair * 100 <= padded_single * 106;
 }
 bool pairs_for_dw(const tsp_mlp_plan_t* plan) { return plan->use_pairs && (plan->F / plan->D) % 256 == 0; }
+
+// The tensor cores add into their fp32 accumulators with truncation, so a contraction over very many tokens drifts
+// towards zero (measured: 1.9 % after 2^24 tokens, 0.4 % after 2^22).  The weight-gradient contractions are therefore
+// cut into chunks of at most kDwChunkTokens tokens, one launch per chunk in ascending token order; every launch after
+// the first adds its fp32 result to what the output holds (round to nearest), which bounds the drift at about 3e-4.
+// Up to kDwChunkTokens tokens (all the 7B-shaped workloads) there is one launch and the rank order of the sum is kept.
+constexpr int64_t kDwChunkTokens = 1 << 18;
+
+template <class Fn>
+tsp_status_t for_token_chunks(int64_t S, Fn fn) {
+    if (S <= kDwChunkTokens) return fn(static_cast<int64_t>(0), S, false);
+    for (int64_t c0 = 0; c0 < S; c0 += kDwChunkTokens) {
+        const int64_t len = S - c0 < kDwChunkTokens ? S - c0 : kDwChunkTokens;
+        tsp_status_t st = fn(c0, len, true);
+        if (st != TSP_OK) return st;
+    }
+    return TSP_OK;
+}
+
+inline const void* row_offset(const void* base, int64_t row, int64_t cols) {
+    return static_cast<const uint8_t*>(base) + static_cast<size_t>(row) * static_cast<size_t>(cols) * 2;
+}
+
+// All weight gradients of the MLP for S tokens; `accumulate`: add to what dW* hold instead of overwriting.
+tsp_status_t launch_dw_all(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
+                           const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream,
+                           int accumulate) {
+    const int H = plan->H, F = plan->F;
+    const bool pairs = pairs_for_dw(plan);
+    return for_token_chunks(S, [&](int64_t c0, int64_t len, bool chunked) {
+        const int acc = (accumulate || c0 > 0) ? 1 : 0;
+        const void* x = row_offset(X, c0, H);
+        const void* dy = row_offset(dY, c0, H);
+        const void* a = row_offset(A, c0, F);
+        const void* dg = row_offset(dG, c0, F);
+        const void* du = row_offset(dU, c0, F);
+        return pairs ? launch_bwd_dw_pair(plan, x, dy, a, dg, du, dWg, dWu, dWd, len, stream, acc, chunked)
+                     : launch_bwd_dw(plan, x, dy, a, dg, du, dWg, dWu, dWd, len, stream, acc, chunked);
+    });
+}
 
 // While alive, the plan describes ONE rank's problem: a single shard of width F/D applied to that rank's tokens
 // (the launch helpers read H, F, D from the plan).  Used by the per-rank ring-step entry points.
@@ -1001,8 +1043,8 @@ tsp_status_t tsp_mlp_ring_step_backward_dw(tsp_mlp_plan_t* plan, const void* X_p
     uint8_t* base = static_cast<uint8_t*>(plan->workspace);
     Profiler prof(plan, cs);
     OneShardView view(plan);
-    tsp_status_t st = launch_bwd_dw_pair(plan, X_p, dY_p, base, base + one, base + 2 * one, dWg_k, dWu_k, dWd_k, S_loc, cs,
-                                         accumulate);
+    tsp_status_t st = launch_dw_all(plan, X_p, dY_p, base, base + one, base + 2 * one, dWg_k, dWu_k, dWd_k, S_loc, cs,
+                                    accumulate);
     prof.mark();
     return st;
 }
@@ -1067,8 +1109,7 @@ tsp_status_t tsp_mlp_backward_saved(tsp_mlp_plan_t* plan, const void* X, const v
     st = launch_bwd_dx_pair(plan, dG, dU, Wg, Wu, dX, S, stream);
     if (st != TSP_OK) return st;
     prof.mark();
-    st = pairs_for_dw(plan) ? launch_bwd_dw_pair(plan, X, dY, sv, dG, dU, dWg, dWu, dWd, S, stream)
-                            : launch_bwd_dw(plan, X, dY, sv, dG, dU, dWg, dWu, dWd, S, stream);
+    st = launch_dw_all(plan, X, dY, sv, dG, dU, dWg, dWu, dWd, S, stream, 0);
     if (st != TSP_OK) return st;
     prof.mark();
     return TSP_OK;
@@ -1109,8 +1150,7 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
                : launch_bwd_dx(plan, dG, dU, Wg, Wu, dX, S, stream);
     if (st != TSP_OK) return st;
     prof.mark();
-    st = pairs_for_dw(plan) ? launch_bwd_dw_pair(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream)
-                            : launch_bwd_dw(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream);
+    st = launch_dw_all(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream, 0);
     if (st != TSP_OK) return st;
     prof.mark();
     plan->last_backward_kernels = (pairs && plan->F % 256 == 0) ? 4 : 3;
