@@ -5,7 +5,8 @@
 #include "attn_kernels.cuh"
 
 struct tsp_attn_plan {
-    tsp_mlp_plan_t* base;  // device properties, tensor-map encoder, status word, profiling events
+    tsp_mlp_plan_t* base;  // device-side part shared with the MLP plan: device properties, tensor-map encoder,
+                           // status word, profiling events
     int H, Hq, Hkv, D;
 };
 
@@ -19,7 +20,7 @@ tsp_status_t tsp_attn_plan(int H, int Hq, int Hkv, int D, tsp_attn_plan_t** out)
     if (Hq % D != 0 || Hkv % D != 0 || (Hq / D) % 64 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
     if (H > (1 << 20) || Hq > (1 << 20) || Hkv > (1 << 20)) return TSP_ERR_UNSUPPORTED_SHAPE;
     tsp_mlp_plan_t* base = nullptr;
-    tsp_status_t st = tsp_mlp_plan(H, 128, 1, &base);  // only the shared machinery of the plan is used
+    tsp_status_t st = make_plan(H, 0, 1, &base);  // device-side part only; the MLP fields stay unused
     if (st != TSP_OK) return st;
     tsp_attn_plan_t* plan = new (std::nothrow) tsp_attn_plan_t();
     if (!plan) {

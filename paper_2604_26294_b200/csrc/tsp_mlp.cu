@@ -688,12 +688,20 @@ tsp_status_t static_device_setup(int dev, StaticDeviceState** out) {
 // ---------------------------------------------------------------------------------------------
 extern "C" {
 
+// Device-side part of a plan, common to the MLP and the attention-projection entry points: device properties, the
+// tensor-map encoder, the status word, tunables.  The caller has validated the shape arguments it passes.
+static tsp_status_t make_plan(int H, int F, int D, tsp_mlp_plan_t** out);
+
 tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     if (!out) return TSP_ERR_INVALID_ARG;
     *out = nullptr;
     if (H <= 0 || F <= 0 || D <= 0 || D > 64) return TSP_ERR_INVALID_ARG;
     if (F % D != 0 || (F / D) % 128 != 0 || H % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
     if (H > (1 << 20) || F > (1 << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    return make_plan(H, F, D, out);
+}
+
+static tsp_status_t make_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return TSP_ERR_CUDA;
