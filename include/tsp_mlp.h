@@ -292,7 +292,8 @@ tsp_status_t tsp_mlp_profile_end(tsp_mlp_plan_t* plan);
 
 /* Number of kernels one forward call launches (pass=TSP_WS_FORWARD: 2), or that the most recent
  * tsp_mlp_backward on this plan launched (pass=TSP_WS_BACKWARD: 4 on the CTA-pair path with F % 256 == 0,
- * else 3; 3 before the first backward call). */
+ * else 3, plus one per further 2^18-token chunk of the weight-gradient contraction; 3 before the first backward
+ * call). */
 int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass);
 
 #ifdef __cplusplus

@@ -1161,7 +1161,8 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
     st = launch_dw_all(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream, 0);
     if (st != TSP_OK) return st;
     prof.mark();
-    plan->last_backward_kernels = (pairs && plan->F % 256 == 0) ? 4 : 3;
+    plan->last_backward_kernels = ((pairs && plan->F % 256 == 0) ? 4 : 3) +
+                                  static_cast<int>((S - 1) / kDwChunkTokens);   // one more dW launch per further chunk
     return TSP_OK;
 }
 
