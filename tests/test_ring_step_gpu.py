@@ -97,7 +97,7 @@ def test_ring_steps_forward_gelu():
     assert rel_fro(got, ref) <= TOL_ORACLE
 
 
-def _ring_backward_emulated(prob):
+def _ring_backward_emulated(prob, act=None):
     """Ranks in turn; the accumulator of shard k is one buffer that every rank holding k adds to (it 'travels')."""
     import torch
 
@@ -105,6 +105,8 @@ def _ring_backward_emulated(prob):
     S_loc, F_d = S // D, F // D
     plan = b.tsp_mlp_plan(H, F, D)
     try:
+        if act is not None:
+            b.tsp_mlp_set_activation(plan, act)
         nbytes = b.tsp_mlp_workspace_bytes_ring(plan, S_loc, b.TSP_WS_BACKWARD)
         ws = [torch.empty(nbytes, dtype=torch.uint8, device="cuda") for _ in range(D)]
         dX = torch.full((S, H), float("nan"), dtype=torch.bfloat16, device="cuda")
@@ -144,6 +146,16 @@ def test_ring_steps_backward_match_oracle_and_single_call(S, H, F, D):
         assert np.all(np.isfinite(g))
         assert rel_fro(g, ref_full) <= TOL_ORACLE
         assert rel_fro(g, unshard(tensor_to_f64(single))) <= TOL_MODES
+
+
+def test_ring_steps_backward_gelu():
+    prob = DeviceProblem(512, 256, 512, 2, seed=35, with_dy=True)
+    dX, dWg, dWu, dWd = _ring_backward_emulated(prob, act=b.TSP_ACT_GELU)
+    rdX, rdWg, rdWu, rdWd = orc.gated_mlp_backward(*prob.f64(), act="gelu")
+    assert rel_fro(tensor_to_f64(dX), rdX) <= TOL_ORACLE
+    assert rel_fro(inp.unshard_columns(tensor_to_f64(dWg)), rdWg) <= TOL_ORACLE
+    assert rel_fro(inp.unshard_columns(tensor_to_f64(dWu)), rdWu) <= TOL_ORACLE
+    assert rel_fro(inp.unshard_rows(tensor_to_f64(dWd)), rdWd) <= TOL_ORACLE
 
 
 def test_ring_mlp_object_single_rank():
