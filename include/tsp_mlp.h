@@ -290,10 +290,10 @@ tsp_status_t tsp_mlp_profile_begin(tsp_mlp_plan_t* plan, int max_calls);
 tsp_status_t tsp_mlp_profile_read(tsp_mlp_plan_t* plan, int call_index, int* n_kernels_out, float* ms_out);
 tsp_status_t tsp_mlp_profile_end(tsp_mlp_plan_t* plan);
 
-/* Number of kernels one forward call launches (pass=TSP_WS_FORWARD: 2), or that the most recent
- * tsp_mlp_backward on this plan launched (pass=TSP_WS_BACKWARD: 4 on the CTA-pair path with F % 256 == 0,
- * else 3, plus one per further 2^18-token chunk of the weight-gradient contraction; 3 before the first backward
- * call). */
+/* Number of kernels the most recent tsp_mlp_forward (pass=TSP_WS_FORWARD) or tsp_mlp_backward (pass=TSP_WS_BACKWARD)
+ * on this plan launched.  Up to 12288 tokens per phase a forward call is 2 kernels and a backward call 4 (CTA-pair
+ * path with F % 256 == 0, else 3); longer problems are cut into several launches per phase (token chunks), and the
+ * weight-gradient contraction into one launch per 2^18 tokens.  Before the first call: 2 and 3. */
 int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass);
 
 #ifdef __cplusplus

@@ -418,6 +418,7 @@ struct PairGateUpPolicyT {
         __nv_bfloat16* dU;    // [S, F] (backward only)
         int S, H, F, D, F_d, S_loc;
         int m_tiles, tiles_per_rank, jl_blocks, band, shared_order;
+        int mt_base;          // first token tile of this launch (a long problem is cut into several launches)
         int act;              // gate activation
         int rank_indexed;     // staged mode: one ring step per launch; the weight tensors hold, at index r, the
                               // shard rank r currently has in its receive buffer, and A is [S, F/D]
@@ -448,7 +449,7 @@ struct PairGateUpPolicyT {
         rem -= t * p.jl_blocks * band_sz;
         Tile o;
         o.jl = rem / band_sz;
-        o.mt = band_start + rem % band_sz;
+        o.mt = p.mt_base + band_start + rem % band_sz;
         int r;
         token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, r, o.row0, o.valid);
         o.k = p.rank_indexed ? r : (p.shared_order ? t : (r - t + p.D) % p.D);
@@ -578,6 +579,7 @@ struct PairDaPolicyT {
         __nv_bfloat16* dU;           // [S, F]
         int S, H, F, D, S_loc;
         int m_tiles, tiles_per_rank, j_tiles, band;
+        int mt_base;                 // first token tile of this launch
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -601,7 +603,7 @@ struct PairDaPolicyT {
         const int rem = tile - band_idx * per_band;
         Tile o;
         o.jt = rem / band_sz;
-        o.mt = band_start + rem % band_sz;
+        o.mt = p.mt_base + band_start + rem % band_sz;
         int r;
         token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, r, o.row0, o.valid);
         return o;
@@ -668,6 +670,7 @@ struct PairDownPolicy {
         int S, H, F, D, F_d, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;   // mixed-width kernel: number of 256 x 512 tiles at the head of the tile list
+        int mt_base;  // first token tile of this launch (a long problem is cut into several launches)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -696,7 +699,7 @@ struct PairDownPolicy {
         o.nb = rem / g_sz;
         // token tiles are taken from the last to the first: the producer kernel wrote the last rows most recently,
         // so they are the ones still in L2
-        o.mt = p.m_tiles - 1 - (g_start + rem % g_sz);
+        o.mt = p.mt_base + p.m_tiles - 1 - (g_start + rem % g_sz);
         token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }
@@ -714,6 +717,7 @@ struct PairDownPolicy {
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
         mixed_tile(t, p.wide_tiles, p.n_blocks, p.m_tiles, true, o.mt, o.nb, o.halves);
+        o.mt += p.mt_base;
         token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }
@@ -791,6 +795,7 @@ struct PairDxPolicy {
         int S, H, F, D, F_d, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;
+        int mt_base;   // first token tile of this launch
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -818,7 +823,7 @@ struct PairDxPolicy {
         o.nb = rem / g_sz;
         // token tiles are taken from the last to the first: the producer kernel wrote the last rows most recently,
         // so they are the ones still in L2
-        o.mt = p.m_tiles - 1 - (g_start + rem % g_sz);
+        o.mt = p.mt_base + p.m_tiles - 1 - (g_start + rem % g_sz);
         token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }
@@ -842,6 +847,7 @@ struct PairDxPolicy {
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
         mixed_tile(t, p.wide_tiles, p.n_blocks, p.m_tiles, true, o.mt, o.nb, o.halves);
+        o.mt += p.mt_base;
         token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, o.r, o.row0, o.valid);
         return o;
     }

@@ -53,11 +53,15 @@ struct tsp_mlp_plan {
     int shared_order;   // gate|up tile order: 1 = all ranks of a band on the same shard column block
     int group;          // token tiles per group in the down / dX tile order
     int pair_stages;
-    int last_backward_kernels;  // kernels launched by the most recent tsp_mlp_backward (3 or 4)
+    int last_backward_kernels;  // kernels launched by the most recent backward call
+    int last_forward_kernels;   // kernels launched by the most recent forward call
+    int launch_count;           // kernels launched since the current call began
     int dw_group;               // hidden blocks per group in the dW tile order
     int dx_group;               // token tiles per group in the dX tile order
     int act;                    // gate activation (TSP_ACT_*)
     int wide_mask;              // 256 x 512 tiles for: bit 0 down, bit 1 dX, bit 2 dW (env TSP_MLP_WIDE)
+    int chunk_bands;            // token bands per launch of the band-ordered kernels (gate|up, dA); 0 = one launch
+    int chunk_tiles;            // token tiles per launch of the group-ordered kernels (down, dX); 0 = one launch
     int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
     cudaStream_t host_copy_stream;           // tsp_mlp_forward_host: uploads Wd while the gate|up kernel runs
@@ -185,6 +189,7 @@ tsp_status_t launch_gate_up(tsp_mlp_plan_t* plan, const void* X, const void* Wg,
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
     tsp::gate_up_swiglu_kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    ++plan->launch_count;
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
@@ -212,6 +217,7 @@ tsp_status_t launch_down(tsp_mlp_plan_t* plan, const void* A, const void* Wd, vo
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
     tsp::down_accumulate_kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    ++plan->launch_count;
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
@@ -247,6 +253,7 @@ tsp_status_t launch_bwd_gate(tsp_mlp_plan_t* plan, const void* X, const void* Wg
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
     tsp::bwd_gate_kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    ++plan->launch_count;
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
@@ -277,6 +284,7 @@ tsp_status_t launch_bwd_dx(tsp_mlp_plan_t* plan, const void* dG, const void* dU,
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
     kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    ++plan->launch_count;
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
@@ -309,6 +317,7 @@ tsp_status_t launch_bwd_dw(tsp_mlp_plan_t* plan, const void* X, const void* dY, 
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int grid = p.num_tiles < plan->sm_count ? p.num_tiles : plan->sm_count;
     kernel<<<grid, tsp::kNumThreads, smem, stream>>>(p);
+    ++plan->launch_count;
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
@@ -337,6 +346,26 @@ int mixed_wide_tiles(const tsp_mlp_plan_t* plan, int bit, int n_blocks, int narr
     return 0;
 }
 
+// The CTA pairs of a launch take their tiles in a fixed round-robin order.  Over hundreds of tiles they drift apart in
+// time, and the tiles that were laid out to share an operand block through L2 no longer run together (measured at
+// S = 65536: 2.4 x the DRAM reads of the same tile order at S = 8192, 4-5 % of the time).  A long problem is therefore
+// cut into several launches of `chunk` token tiles each; every launch boundary realigns the pairs.  fn(first token
+// tile, token tiles) launches one chunk; `reverse` walks the chunks from the last to the first.
+template <class Fn>
+tsp_status_t for_tile_chunks(int m_tiles, int chunk, bool reverse, Fn fn) {
+    if (chunk <= 0 || m_tiles <= chunk + chunk / 2) return fn(0, m_tiles);
+    int n = m_tiles / chunk;                       // the remainder joins the last chunk if it is less than half a chunk
+    if (m_tiles - n * chunk >= chunk / 2 && m_tiles - n * chunk > 0) ++n;
+    for (int i = 0; i < n; ++i) {
+        const int c = reverse ? n - 1 - i : i;
+        const int first = c * chunk;
+        const int count = c == n - 1 ? m_tiles - first : chunk;
+        tsp_status_t st = fn(first, count);
+        if (st != TSP_OK) return st;
+    }
+    return TSP_OK;
+}
+
 template <class Params>
 void fill_common(tsp_mlp_plan_t* plan, Params& p, int num_tiles) {
     p.num_tiles = num_tiles;
@@ -354,6 +383,7 @@ tsp_status_t launch_pair_wide(tsp_mlp_plan_t* plan, Kernel kernel, Params& p, cu
     const int pairs_avail = plan->sm_count / 2;
     const int pairs = p.num_tiles < pairs_avail ? p.num_tiles : pairs_avail;
     kernel<<<2 * pairs, tsp::kNumThreads, smem, stream>>>(p);
+    ++plan->launch_count;
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
@@ -366,6 +396,7 @@ tsp_status_t launch_pair(tsp_mlp_plan_t* plan, Kernel kernel, const Params& p, c
     const int pairs_avail = plan->sm_count / 2;
     const int pairs = p.num_tiles < pairs_avail ? p.num_tiles : pairs_avail;
     kernel<<<2 * pairs, tsp::kNumThreads, smem, stream>>>(p);
+    ++plan->launch_count;
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
@@ -393,8 +424,12 @@ tsp_status_t launch_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* W
     p.band = gate_band(plan, p.m_tiles);
     p.shared_order = plan->shared_order;
     p.act = plan->act;
-    fill_common(plan, p, p.m_tiles * D * p.jl_blocks);
-    return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
+    return for_tile_chunks(p.m_tiles, plan->chunk_bands * p.band, false, [&](int first, int count) {
+        p.mt_base = first;
+        p.m_tiles = count;
+        fill_common(plan, p, count * D * p.jl_blocks);
+        return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
+    });
 }
 
 tsp_status_t launch_gate_up_pair(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A, int64_t S,
@@ -423,8 +458,12 @@ tsp_status_t launch_da_pair_t(tsp_mlp_plan_t* plan, const void* dY, const void* 
     p.m_tiles = D * p.tiles_per_rank;
     p.j_tiles = F / 256;
     p.band = gate_band(plan, p.m_tiles);
-    fill_common(plan, p, p.m_tiles * p.j_tiles);
-    return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
+    return for_tile_chunks(p.m_tiles, plan->chunk_bands * p.band, false, [&](int first, int count) {
+        p.mt_base = first;
+        p.m_tiles = count;
+        fill_common(plan, p, count * p.j_tiles);
+        return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
+    });
 }
 
 tsp_status_t launch_da_pair(tsp_mlp_plan_t* plan, const void* dY, const void* Wd, float* dA, int64_t S, cudaStream_t stream) {
@@ -444,14 +483,19 @@ tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* W
     p.m_tiles = D * p.tiles_per_rank;
     p.n_blocks = H / 256;
     const int group = plan->group > 0 ? plan->group : 8;
-    p.group = p.m_tiles < group ? p.m_tiles : group;
-    p.wide_tiles = mixed_wide_tiles(plan, 1, p.n_blocks, p.m_tiles * p.n_blocks, F / 64);
-    if (p.wide_tiles > 0) {
-        fill_common(plan, p, p.m_tiles * p.n_blocks - p.wide_tiles);   // wide tiles count once in the list
-        return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDownPolicy>, p, stream);
-    }
-    fill_common(plan, p, p.m_tiles * p.n_blocks);
-    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownPolicy>, p, stream);
+    // chunks from the last token tiles to the first: the rows the gate|up kernel wrote last are still in L2
+    return for_tile_chunks(p.m_tiles, plan->chunk_tiles, true, [&](int first, int count) {
+        p.mt_base = first;
+        p.m_tiles = count;
+        p.group = count < group ? count : group;
+        p.wide_tiles = mixed_wide_tiles(plan, 1, p.n_blocks, count * p.n_blocks, F / 64);
+        if (p.wide_tiles > 0) {
+            fill_common(plan, p, count * p.n_blocks - p.wide_tiles);   // wide tiles count once in the list
+            return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDownPolicy>, p, stream);
+        }
+        fill_common(plan, p, count * p.n_blocks);
+        return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownPolicy>, p, stream);
+    });
 }
 
 tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void* dU, const void* Wg, const void* Wu,
@@ -472,14 +516,18 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
     p.m_tiles = D * p.tiles_per_rank;
     p.n_blocks = H / 256;
     const int group = plan->dx_group > 0 ? plan->dx_group : 8;
-    p.group = p.m_tiles < group ? p.m_tiles : group;
-    p.wide_tiles = mixed_wide_tiles(plan, 2, p.n_blocks, p.m_tiles * p.n_blocks, 2 * F / 64);
-    if (p.wide_tiles > 0) {
-        fill_common(plan, p, p.m_tiles * p.n_blocks - p.wide_tiles);
-        return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDxPolicy>, p, stream);
-    }
-    fill_common(plan, p, p.m_tiles * p.n_blocks);
-    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDxPolicy>, p, stream);
+    return for_tile_chunks(p.m_tiles, plan->chunk_tiles, true, [&](int first, int count) {
+        p.mt_base = first;
+        p.m_tiles = count;
+        p.group = count < group ? count : group;
+        p.wide_tiles = mixed_wide_tiles(plan, 2, p.n_blocks, count * p.n_blocks, 2 * F / 64);
+        if (p.wide_tiles > 0) {
+            fill_common(plan, p, count * p.n_blocks - p.wide_tiles);
+            return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDxPolicy>, p, stream);
+        }
+        fill_common(plan, p, count * p.n_blocks);
+        return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDxPolicy>, p, stream);
+    });
 }
 
 tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
@@ -736,11 +784,15 @@ static tsp_status_t make_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->group = env_int("TSP_MLP_GROUP", 0);
     plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
     plan->last_backward_kernels = 3;
+    plan->last_forward_kernels = 2;
+    plan->launch_count = 0;
     plan->host_ready = false;
     plan->phase_mask = env_int("TSP_MLP_PHASES", 3);
     plan->act = TSP_ACT_SILU;
     plan->wide_mask = env_int("TSP_MLP_WIDE", -1);   // -1: decide per launch from the tile counts
     plan->dw_group = env_int("TSP_MLP_DW_GROUP", 0);
+    plan->chunk_bands = env_int("TSP_MLP_CHUNK_BANDS", 3);
+    plan->chunk_tiles = env_int("TSP_MLP_CHUNK_TILES", 96);
     plan->dx_group = env_int("TSP_MLP_DX_GROUP", 0);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
@@ -821,6 +873,7 @@ static tsp_status_t forward_impl(tsp_mlp_plan_t* plan, const void* X, const void
     if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes(plan, S, TSP_WS_FORWARD))
         return TSP_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    plan->launch_count = 0;
     Profiler prof(plan, stream);
     const bool pairs = pairs_for_tokens(plan, S);
     if (plan->phase_mask & 1) {
@@ -839,6 +892,7 @@ static tsp_status_t forward_impl(tsp_mlp_plan_t* plan, const void* X, const void
         if (st != TSP_OK) return st;
     }
     prof.mark();
+    plan->last_forward_kernels = plan->launch_count;
     return TSP_OK;
 }
 
@@ -1140,6 +1194,7 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
     void* A = base;
     void* dG = base + one;
     void* dU = base + 2 * one;
+    plan->launch_count = 0;
     Profiler prof(plan, stream);
     const bool pairs = pairs_for_tokens(plan, S);
     if (pairs && plan->F % 256 == 0) {
@@ -1161,8 +1216,7 @@ tsp_status_t tsp_mlp_backward(tsp_mlp_plan_t* plan, const void* X, const void* W
     st = launch_dw_all(plan, X, dY, A, dG, dU, dWg, dWu, dWd, S, stream, 0);
     if (st != TSP_OK) return st;
     prof.mark();
-    plan->last_backward_kernels = ((pairs && plan->F % 256 == 0) ? 4 : 3) +
-                                  static_cast<int>((S - 1) / kDwChunkTokens);   // one more dW launch per further chunk
+    plan->last_backward_kernels = plan->launch_count;
     return TSP_OK;
 }
 
@@ -1293,7 +1347,7 @@ tsp_status_t tsp_mlp_profile_end(tsp_mlp_plan_t* plan) {
 
 int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass) {
     if (!plan) return 0;
-    return pass == TSP_WS_BACKWARD ? plan->last_backward_kernels : 2;
+    return pass == TSP_WS_BACKWARD ? plan->last_backward_kernels : plan->last_forward_kernels;
 }
 
 }  // extern "C"
