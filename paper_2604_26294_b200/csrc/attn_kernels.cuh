@@ -23,6 +23,7 @@ struct PairQkvPolicy {
         __nv_bfloat16* V;   // [S, Hkv]
         int S, H, Hq, Hkv;
         int m_tiles, q_blocks, kv_blocks, n_blocks, band;
+        int mt_base;        // first token tile of this launch (long problems are cut into several launches)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -48,7 +49,7 @@ struct PairQkvPolicy {
         const int b_sz = min(p.band, p.m_tiles - b_start);
         const int rem = tile - b * per_band;
         const int nb = rem / b_sz;
-        const int mt = b_start + rem - nb * b_sz;
+        const int mt = p.mt_base + b_start + rem - nb * b_sz;
         Tile o;
         o.row0 = mt * 256;
         o.valid = min(256, p.S - o.row0);
@@ -86,6 +87,7 @@ struct PairOutPolicy {
         __nv_bfloat16* Y;           // [S, H]
         int S, H, Hq, D, Hq_d;
         int m_tiles, n_blocks, group;
+        int mt_base;
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -109,7 +111,7 @@ struct PairOutPolicy {
         const int rem = tile - g * per_group;
         Tile o;
         o.nb = rem / g_sz;
-        const int mt = g_start + rem - o.nb * g_sz;
+        const int mt = p.mt_base + g_start + rem - o.nb * g_sz;
         o.row0 = mt * 256;
         o.valid = min(256, p.S - o.row0);
         return o;
@@ -136,6 +138,7 @@ struct PairAttnDxPolicy {
         __nv_bfloat16* dX;                   // [S, H]
         int S, H, q_kb, kv_kb;               // k-blocks of 64 features per matrix
         int m_tiles, n_blocks, group;
+        int mt_base;
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -160,7 +163,7 @@ struct PairAttnDxPolicy {
         const int rem = tile - g * per_group;
         Tile o;
         o.nb = rem / g_sz;
-        const int mt = g_start + rem - o.nb * g_sz;
+        const int mt = p.mt_base + g_start + rem - o.nb * g_sz;
         o.row0 = mt * 256;
         o.valid = min(256, p.S - o.row0);
         return o;
@@ -196,6 +199,7 @@ struct PairAttnDaPolicy {
         __nv_bfloat16* dA;           // [S, Hq]
         int S, H, Hq, Hq_d;
         int m_tiles, n_blocks, band;
+        int mt_base;
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -219,7 +223,7 @@ struct PairAttnDaPolicy {
         const int rem = tile - b * per_band;
         Tile o;
         o.nb = rem / b_sz;
-        const int mt = b_start + rem - o.nb * b_sz;
+        const int mt = p.mt_base + b_start + rem - o.nb * b_sz;
         o.row0 = mt * 256;
         o.valid = min(256, p.S - o.row0);
         const int c = o.nb * 256;

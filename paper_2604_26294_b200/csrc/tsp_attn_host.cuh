@@ -65,9 +65,13 @@ tsp_status_t tsp_attn_qkv_forward(tsp_attn_plan_t* plan, const void* X, const vo
     p.kv_blocks = Hkv / 256;
     p.n_blocks = p.q_blocks + 2 * p.kv_blocks;
     p.band = gate_band(base, p.m_tiles);   // the band's rows of X take about 32 MB of L2
-    fill_common(base, p, p.m_tiles * p.n_blocks);
     Profiler prof(base, stream);
-    tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairQkvPolicy>, p, stream);
+    tsp_status_t st = for_tile_chunks(p.m_tiles, base->chunk_bands * p.band, false, [&](int first, int count) {
+        p.mt_base = first;
+        p.m_tiles = count;
+        fill_common(base, p, count * p.n_blocks);
+        return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairQkvPolicy>, p, stream);
+    });
     prof.mark();
     return st;
 }
@@ -91,9 +95,14 @@ tsp_status_t tsp_attn_out_forward(tsp_attn_plan_t* plan, const void* A, const vo
     p.n_blocks = H / 256;
     const int group = base->group > 0 ? base->group : 8;
     p.group = p.m_tiles < group ? p.m_tiles : group;
-    fill_common(base, p, p.m_tiles * p.n_blocks);
     Profiler prof(base, stream);
-    tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairOutPolicy>, p, stream);
+    tsp_status_t st = for_tile_chunks(p.m_tiles, base->chunk_tiles, false, [&](int first, int count) {
+        p.mt_base = first;
+        p.m_tiles = count;
+        p.group = count < group ? count : group;
+        fill_common(base, p, count * p.n_blocks);
+        return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairOutPolicy>, p, stream);
+    });
     prof.mark();
     return st;
 }
@@ -127,8 +136,13 @@ tsp_status_t tsp_attn_qkv_backward(tsp_attn_plan_t* plan, const void* X, const v
         p.n_blocks = H / 256;
         const int group = base->dx_group > 0 ? base->dx_group : 8;
         p.group = p.m_tiles < group ? p.m_tiles : group;
-        fill_common(base, p, p.m_tiles * p.n_blocks);
-        tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDxPolicy>, p, stream);
+        tsp_status_t st = for_tile_chunks(p.m_tiles, base->chunk_tiles, false, [&](int first, int count) {
+            p.mt_base = first;
+            p.m_tiles = count;
+            p.group = count < group ? count : group;
+            fill_common(base, p, count * p.n_blocks);
+            return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDxPolicy>, p, stream);
+        });
         if (st != TSP_OK) return st;
         prof.mark();
     }
@@ -178,8 +192,12 @@ tsp_status_t tsp_attn_out_backward(tsp_attn_plan_t* plan, const void* A, const v
         p.m_tiles = static_cast<int>((S + 255) / 256);
         p.n_blocks = Hq / 256;
         p.band = gate_band(base, p.m_tiles);
-        fill_common(base, p, p.m_tiles * p.n_blocks);
-        tsp_status_t st = launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDaPolicy>, p, stream);
+        tsp_status_t st = for_tile_chunks(p.m_tiles, base->chunk_bands * p.band, false, [&](int first, int count) {
+            p.mt_base = first;
+            p.m_tiles = count;
+            fill_common(base, p, count * p.n_blocks);
+            return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDaPolicy>, p, stream);
+        });
         if (st != TSP_OK) return st;
         prof.mark();
     }
