@@ -879,6 +879,7 @@ struct PairDwPolicy {
         int k_linear;  // 0, or ceil(S / 64) when the token contraction runs in ascending order (ragged ranks)
         int accumulate;  // 0: dW overwritten; 1: the tile's sum is added to what dW holds (partial sums of other ranks)
         int wide_tiles;
+        int tile_base;   // first entry of the tile list this launch covers (a long list is cut into several launches)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -905,6 +906,7 @@ struct PairDwPolicy {
     }
     __device__ static __forceinline__ Tile decode(const Params& p, int tile) {
         // family (dWd, dWg, dWu) -> group of hidden blocks -> intermediate tile -> hidden block of the group
+        tile += p.tile_base;
         Tile o;
         const int per_which = p.j_tiles * p.n_blocks;
         o.which = tile / per_which;
@@ -971,7 +973,7 @@ struct PairDwPolicy {
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
         int row;
-        mixed_tile(t, p.wide_tiles, p.n_blocks, 3 * p.j_tiles, false, row, o.nb, o.halves);
+        mixed_tile(t + p.tile_base, p.wide_tiles, p.n_blocks, 3 * p.j_tiles, false, row, o.nb, o.halves);
         o.which = row / p.j_tiles;
         o.jt = row - o.which * p.j_tiles;
         o.k = o.jt / p.j_tiles_per_shard;

@@ -61,6 +61,8 @@ struct tsp_mlp_plan {
     int act;                    // gate activation (TSP_ACT_*)
     int wide_mask;              // 256 x 512 tiles for: bit 0 down, bit 1 dX, bit 2 dW (env TSP_MLP_WIDE)
     int chunk_bands;            // token bands per launch of the band-ordered kernels (gate|up, dA); 0 = one launch
+    int dw_chunk_rounds;        // rounds of the CTA pairs per launch of the weight-gradient kernel; 0 = about 3 ms of
+                                // work per launch, negative = one launch
     int chunk_tiles;            // token tiles per launch of the group-ordered kernels (down, dX); 0 = one launch
     int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
@@ -555,13 +557,23 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     int n_group = plan->dw_group > 0 ? plan->dw_group : static_cast<int>((64ull << 20) / (512ull * static_cast<size_t>(S)));
     if (n_group < 1) n_group = 1;
     p.wide_tiles = mixed_wide_tiles(plan, 4, p.n_blocks, 3 * p.j_tiles * p.n_blocks, static_cast<int>(S / 64));
-    if (p.wide_tiles > 0) {
-        fill_common(plan, p, 3 * p.j_tiles * p.n_blocks - p.wide_tiles);
-        return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDwPolicy>, p, stream);
-    }
     p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
-    fill_common(plan, p, 3 * p.j_tiles * p.n_blocks);
-    return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDwPolicy>, p, stream);
+    // the tile list is cut into launches of `dw_chunk_rounds` rounds of the CTA pairs (see for_tile_chunks)
+    const int list = 3 * p.j_tiles * p.n_blocks - p.wide_tiles;
+    // about 3 ms of work per launch: a tile takes about 0.44 us per 64-token k-block (twice that for a wide tile)
+    int rounds = plan->dw_chunk_rounds;
+    if (rounds == 0) {
+        const double tile_us = 0.44 * static_cast<double>((S + 63) / 64) * (p.wide_tiles > 0 ? 2.0 : 1.0);
+        rounds = static_cast<int>(3000.0 / tile_us + 0.5);
+        if (rounds < 1) rounds = 1;
+    }
+    const int chunk = rounds > 0 ? rounds * (plan->sm_count / 2) : 0;
+    return for_tile_chunks(list, chunk, false, [&](int first, int count) {
+        p.tile_base = first;
+        fill_common(plan, p, count);
+        return p.wide_tiles > 0 ? launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDwPolicy>, p, stream)
+                                : launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDwPolicy>, p, stream);
+    });
 }
 
 // CTA pairs work on 256-row token tiles, single CTAs on 128-row tiles; a rank's last tile is padded.  Pairs are the
@@ -793,6 +805,7 @@ static tsp_status_t make_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->dw_group = env_int("TSP_MLP_DW_GROUP", 0);
     plan->chunk_bands = env_int("TSP_MLP_CHUNK_BANDS", 3);
     plan->chunk_tiles = env_int("TSP_MLP_CHUNK_TILES", 96);
+    plan->dw_chunk_rounds = env_int("TSP_MLP_DW_CHUNK_ROUNDS", 0);
     plan->dx_group = env_int("TSP_MLP_DX_GROUP", 0);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
