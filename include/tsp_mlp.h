@@ -30,6 +30,10 @@
  *   - A plan must not be used from two host threads at once, nor on two streams at
  *     once (the workspace and status word are shared).
  *   - Results are deterministic: no atomics, fixed accumulation order.
+ *   - "One kernel" / "two kernels" below name the distinct kernels of a call.  A long problem runs each of them
+ *     as several launches over consecutive token ranges (beyond about 18 000 tokens; the launch boundaries keep
+ *     the thread blocks aligned in time so that they keep sharing operand blocks through L2); outputs do not
+ *     depend on where the cuts fall.  tsp_mlp_kernels_per_call reports the launches actually made.
  */
 #ifndef TSP_MLP_H
 #define TSP_MLP_H
