@@ -185,7 +185,8 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
  *   t = D-1:      Y_p   = bf16(Yacc + ...)                          (D = 1: Y_p = bf16(...) directly)
  * X_p, Y_p: [S_loc, H] bf16 (this rank's tokens only); Wg_k, Wu_k: [H, F/D] bf16 and Wd_k: [F/D, H] bf16, the
  * shard the rank holds at this step (k = (p - t) mod D when the caller follows the ring; the kernels do not
- * care which).  The fp32 accumulator Yacc [S_loc, H] and the bf16 scratch A [S_loc, F/D] live in the plan's
+ * care which).  The fp32 accumulator Yacc [S_loc, H] and two bf16 scratch buffers A [S_loc, F/D] (even / odd
+ * steps) live in the plan's
  * workspace (tsp_mlp_workspace_bytes_ring(plan, S_loc, TSP_WS_FORWARD) bytes) and carry the state from step to
  * step, so the D calls of one forward pass must use the same plan, workspace and S_loc, in the order t = 0..D-1 on
  * one stream (or otherwise ordered).  Two kernels per call (gate|up with the activation epilogue; down projection
@@ -197,6 +198,19 @@ tsp_status_t tsp_mlp_forward_staged(tsp_mlp_plan_t* plan, const void* X, const v
 size_t tsp_mlp_workspace_bytes_ring(const tsp_mlp_plan_t* plan, int64_t S_loc, int pass);
 tsp_status_t tsp_mlp_ring_step(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
                                const void* Wd_k, void* Y_p, int64_t S_loc, int t, int D, void* cuda_stream);
+
+/*
+ * The two halves of tsp_mlp_ring_step as calls of their own: _gate writes A = act(X_p Wg_k) * (X_p Wu_k) into the
+ * scratch buffer of step t (buffer t & 1), _down adds A Wd_k to the accumulator (or stores Y_p at t = D-1).  With
+ * few tokens per rank one step is less than a full round of tiles, so a caller can fill the GPU by running the
+ * down projection of step t on a second stream while the gate|up GEMM of step t+1 runs on the first.  Ordering
+ * the caller must provide: _down(t) after _gate(t); _gate(t+2) after _down(t) (it reuses the scratch buffer);
+ * _down(t+1) after _down(t) (the accumulator).  Same bits as tsp_mlp_ring_step.
+ */
+tsp_status_t tsp_mlp_ring_step_gate(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
+                                    int64_t S_loc, int t, int D, void* cuda_stream);
+tsp_status_t tsp_mlp_ring_step_down(tsp_mlp_plan_t* plan, const void* Wd_k, void* Y_p, int64_t S_loc, int t, int D,
+                                    void* cuda_stream);
 
 /*
  * Backward pass of one ring step on one rank's data (the backward mirrors the forward weight movement, and the

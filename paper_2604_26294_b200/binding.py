@@ -49,6 +49,8 @@ SIGNATURES = {
                                                      _P]),
     "tsp_mlp_ring_step_backward_dw": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                                      _P]),
+    "tsp_mlp_ring_step_gate": (ctypes.c_int, [_P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
+    "tsp_mlp_ring_step_down": (ctypes.c_int, [_P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_ring_step": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_forward_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, _P,
                                               ctypes.c_int64, ctypes.POINTER(ctypes.c_int), _P]),
@@ -205,6 +207,18 @@ def tsp_mlp_ring_step(plan, X_p, Wg_k, Wu_k, Wd_k, Y_p, S_loc: int, t: int, D: i
     """One ring step of Algorithm 2 on one rank's tokens and the one shard it holds at step t."""
     _check(load_library().tsp_mlp_ring_step(plan, _ptr(X_p), _ptr(Wg_k), _ptr(Wu_k), _ptr(Wd_k), _ptr(Y_p), S_loc, t, D,
                                             _stream_handle(stream)), "tsp_mlp_ring_step", plan)
+
+
+def tsp_mlp_ring_step_gate(plan, X_p, Wg_k, Wu_k, S_loc: int, t: int, D: int, stream=None) -> None:
+    """First half of a ring step: the gate|up GEMM with the activation epilogue into the scratch buffer of step t."""
+    _check(load_library().tsp_mlp_ring_step_gate(plan, _ptr(X_p), _ptr(Wg_k), _ptr(Wu_k), S_loc, t, D,
+                                                 _stream_handle(stream)), "tsp_mlp_ring_step_gate", plan)
+
+
+def tsp_mlp_ring_step_down(plan, Wd_k, Y_p, S_loc: int, t: int, D: int, stream=None) -> None:
+    """Second half of a ring step: the shard's down projection added to the carried fp32 sum."""
+    _check(load_library().tsp_mlp_ring_step_down(plan, _ptr(Wd_k), _ptr(Y_p), S_loc, t, D, _stream_handle(stream)),
+           "tsp_mlp_ring_step_down", plan)
 
 
 def tsp_mlp_ring_step_backward_dx(plan, X_p, Wg_k, Wu_k, Wd_k, dY_p, dX_p, S_loc: int, t: int, D: int, stream=None) -> None:

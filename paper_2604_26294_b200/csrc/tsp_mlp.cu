@@ -644,9 +644,8 @@ struct OneShardView {
 // One ring step for `n_ranks` ranks at once (S tokens in all): gate|up GEMM of every rank's tokens against the shard
 // in that rank's buffer slot into the [S, F/D] scratch, then the down projection of that shard added to the fp32
 // accumulator.  mode: 0 first step, 1 middle, 2 last (rounds to bf16 Y), 3 only step.
-tsp_status_t launch_forward_step(tsp_mlp_plan_t* plan, const void* X, const void* cur_g, const void* cur_u,
-                                 const void* cur_d, void* A_step, float* Yacc, void* Y, int64_t S, int n_ranks, int mode,
-                                 cudaStream_t cs) {
+tsp_status_t launch_step_gate(tsp_mlp_plan_t* plan, const void* X, const void* cur_g, const void* cur_u, void* A_step,
+                              int64_t S, int n_ranks, cudaStream_t cs) {
     const int H = plan->H, F_d = plan->F / plan->D, D = n_ranks;
     tsp_status_t st;
     {
@@ -669,6 +668,13 @@ tsp_status_t launch_forward_step(tsp_mlp_plan_t* plan, const void* X, const void
         st = launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, cs);
         if (st != TSP_OK) return st;
     }
+    return TSP_OK;
+}
+
+tsp_status_t launch_step_down(tsp_mlp_plan_t* plan, const void* cur_d, const void* A_step, float* Yacc, void* Y, int64_t S,
+                              int n_ranks, int mode, cudaStream_t cs) {
+    const int H = plan->H, F_d = plan->F / plan->D, D = n_ranks;
+    tsp_status_t st;
     {
         tsp::PairDownStagedPolicy::Params p;
         std::memset(&p, 0, sizeof(p));
@@ -689,6 +695,14 @@ tsp_status_t launch_forward_step(tsp_mlp_plan_t* plan, const void* X, const void
         if (st != TSP_OK) return st;
     }
     return TSP_OK;
+}
+
+tsp_status_t launch_forward_step(tsp_mlp_plan_t* plan, const void* X, const void* cur_g, const void* cur_u,
+                                 const void* cur_d, void* A_step, float* Yacc, void* Y, int64_t S, int n_ranks, int mode,
+                                 cudaStream_t cs) {
+    tsp_status_t st = launch_step_gate(plan, X, cur_g, cur_u, A_step, S, n_ranks, cs);
+    if (st != TSP_OK) return st;
+    return launch_step_down(plan, cur_d, A_step, Yacc, Y, S, n_ranks, mode, cs);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1046,29 +1060,62 @@ size_t tsp_mlp_workspace_bytes_ring(const tsp_mlp_plan_t* plan, int64_t S_loc, i
     if (!plan || S_loc <= 0) return 0;
     const size_t one = align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2, 256);
     const size_t acc = align_up(static_cast<size_t>(S_loc) * plan->H * 4, 256);
-    if (pass == TSP_WS_FORWARD) return one + acc;                       // A | Yacc
+    if (pass == TSP_WS_FORWARD) return 2 * one + acc;                   // A of even steps | A of odd steps | Yacc
     if (pass == TSP_WS_BACKWARD) return 3 * one + 2 * one + acc;        // A, dG, dU | dA (fp32) | dXacc
     return 0;
 }
 
-tsp_status_t tsp_mlp_ring_step(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
-                               const void* Wd_k, void* Y_p, int64_t S_loc, int t, int D, void* cuda_stream) {
+namespace {
+// argument checks shared by the forward ring-step entry points; on success the scratch of step t and the accumulator
+tsp_status_t ring_step_setup(tsp_mlp_plan_t* plan, int64_t S_loc, int t, int D, void** A_step, float** Yacc) {
     if (!plan || D != plan->D || t < 0 || t >= D) return TSP_ERR_INVALID_ARG;
     if (S_loc < 1 || S_loc > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
-    if (!X_p || !Wg_k || !Wu_k || !Wd_k || !Y_p) return TSP_ERR_INVALID_ARG;
-    if (!aligned16(X_p) || !aligned16(Wg_k) || !aligned16(Wu_k) || !aligned16(Wd_k) || !aligned32(Y_p))
-        return TSP_ERR_INVALID_ARG;
     if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_ring(plan, S_loc, TSP_WS_FORWARD))
         return TSP_ERR_WORKSPACE;
-    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    const size_t one = align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2, 256);
     uint8_t* base = static_cast<uint8_t*>(plan->workspace);
-    void* A_step = base;
-    float* Yacc = reinterpret_cast<float*>(base + align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2, 256));
+    *A_step = base + static_cast<size_t>(t & 1) * one;   // two scratch buffers alternate, so that the down projection
+    *Yacc = reinterpret_cast<float*>(base + 2 * one);    // of step t may overlap the gate|up GEMM of step t + 1
+    return TSP_OK;
+}
+}  // namespace
+
+tsp_status_t tsp_mlp_ring_step_gate(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
+                                    int64_t S_loc, int t, int D, void* cuda_stream) {
+    void* A_step = nullptr;
+    float* Yacc = nullptr;
+    tsp_status_t st = ring_step_setup(plan, S_loc, t, D, &A_step, &Yacc);
+    if (st != TSP_OK) return st;
+    if (!X_p || !Wg_k || !Wu_k) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X_p) || !aligned16(Wg_k) || !aligned16(Wu_k)) return TSP_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
     Profiler prof(plan, cs);
-    tsp_status_t st = launch_forward_step(plan, X_p, Wg_k, Wu_k, Wd_k, A_step, Yacc, Y_p, S_loc, 1,
-                                          D == 1 ? 3 : (t == 0 ? 0 : (t == D - 1 ? 2 : 1)), cs);
+    st = launch_step_gate(plan, X_p, Wg_k, Wu_k, A_step, S_loc, 1, cs);
     prof.mark();
     return st;
+}
+
+tsp_status_t tsp_mlp_ring_step_down(tsp_mlp_plan_t* plan, const void* Wd_k, void* Y_p, int64_t S_loc, int t, int D,
+                                    void* cuda_stream) {
+    void* A_step = nullptr;
+    float* Yacc = nullptr;
+    tsp_status_t st = ring_step_setup(plan, S_loc, t, D, &A_step, &Yacc);
+    if (st != TSP_OK) return st;
+    if (!Wd_k || !Y_p) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(Wd_k) || !aligned32(Y_p)) return TSP_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    Profiler prof(plan, cs);
+    st = launch_step_down(plan, Wd_k, A_step, Yacc, Y_p, S_loc, 1, D == 1 ? 3 : (t == 0 ? 0 : (t == D - 1 ? 2 : 1)), cs);
+    prof.mark();
+    return st;
+}
+
+tsp_status_t tsp_mlp_ring_step(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
+                               const void* Wd_k, void* Y_p, int64_t S_loc, int t, int D, void* cuda_stream) {
+    if (!Wd_k || !Y_p || !aligned16(Wd_k) || !aligned32(Y_p)) return TSP_ERR_INVALID_ARG;   // before anything is launched
+    tsp_status_t st = tsp_mlp_ring_step_gate(plan, X_p, Wg_k, Wu_k, S_loc, t, D, cuda_stream);
+    if (st != TSP_OK) return st;
+    return tsp_mlp_ring_step_down(plan, Wd_k, Y_p, S_loc, t, D, cuda_stream);
 }
 
 tsp_status_t tsp_mlp_ring_step_backward_dx(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,

@@ -47,18 +47,25 @@ def _wait(reqs) -> None:
 
 
 def ring_forward(compute: Callable[[int, int, torch.Tensor], None], own_shard: torch.Tensor,
-                 recv_bufs: Sequence[torch.Tensor], rank: int, D: int, group=None) -> None:
+                 recv_bufs: Sequence[torch.Tensor], rank: int, D: int, group=None,
+                 before_exchange: Callable[[int], None] | None = None) -> None:
     """The loop of Algorithm 2 on one rank.
 
     compute(t, k, shard) runs ring step t with the packed shard k = (rank - t) mod D it is handed;
-    own_shard is this rank's packed shard (never written); recv_bufs are two buffers of the same shape
-    that alternate as receive target.  The transfer for step t+1 is posted before step t computes.
+    own_shard is this rank's packed shard (never written); recv_bufs are n >= 2 buffers of the same shape that
+    take turns as receive target (step t receives into buffer t mod n, which step t - n + 1 was the last to read).
+    The transfer for step t+1 is posted before step t computes.  before_exchange(t), if given, runs before the
+    transfer of step t is posted: a caller whose compute is asynchronous uses it to make sure the target buffer's
+    last reader has finished.
     """
+    n = len(recv_bufs)
     cur = own_shard
     for t in range(D):
         reqs = []
         if t < D - 1:
-            nxt = recv_bufs[t & 1]
+            if before_exchange is not None:
+                before_exchange(t)
+            nxt = recv_bufs[t % n]
             reqs = _exchange(cur, nxt, rank, D, group)
         compute(t, shard_at_step(rank, t, D), cur)
         _wait(reqs)                      # Wait(): the next shard has arrived, the current one has left
@@ -112,6 +119,10 @@ def unpack_shard(buf: torch.Tensor, H: int, F_d: int):
 class TspRingMlp:
     """One rank of the TSP gated ring MLP on its own GPU: the schedule above driving the library's step kernels."""
 
+    # up to this many tokens per rank the two halves of a forward step run on two streams (measured on one rank's
+    # step sequence: +3 % at 1024 tokens, +6 % at 2048, -2 % at 8192)
+    TWO_STREAM_MAX_TOKENS = 4096
+
     def __init__(self, H: int, F: int, D: int, rank: int, S_loc: int, group=None, training: bool = False,
                  activation: int | None = None):
         from . import binding as b   # fails loudly without the CUDA library or a GPU
@@ -126,8 +137,13 @@ class TspRingMlp:
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
         b.tsp_mlp_set_workspace(self.plan, self.workspace)
         n = 3 * H * self.F_d
-        self.recv_bufs = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(2)] if D > 1 else []
+        # three receive buffers: the down projection of step t may still read its shard while the transfer for
+        # step t+2 is posted (the two halves of a step run on two streams, see forward())
+        self.recv_bufs = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(3)] if D > 1 else []
         self.dw_bufs = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(2 if D > 1 else 1)] if training else []
+        self.down_stream = torch.cuda.Stream(device=dev)
+        self._gate_done = [torch.cuda.Event() for _ in range(D)]
+        self._down_done = [torch.cuda.Event() for _ in range(D)]
 
     def close(self) -> None:
         if self.plan is not None:
@@ -135,15 +151,41 @@ class TspRingMlp:
             self.plan = None
 
     def forward(self, X_p: torch.Tensor, shard: torch.Tensor, Y_p: torch.Tensor | None = None) -> torch.Tensor:
-        """Y_p = rows of this rank of the gated MLP over all D shards; `shard` is this rank's packed own shard."""
+        """Y_p = rows of this rank of the gated MLP over all D shards; `shard` is this rank's packed own shard.
+
+        The gate|up GEMM of step t runs on the current stream, the down projection of step t on a second stream, so
+        that the down projection overlaps the next step's gate|up GEMM (with few tokens per rank neither fills the
+        GPU alone; with many tokens per rank everything stays on the current stream).  On return the current stream
+        has been made to wait for the last down projection.
+        """
         if Y_p is None:
             Y_p = torch.empty_like(X_p)
+        main = torch.cuda.current_stream()
+        if self.S_loc > self.TWO_STREAM_MAX_TOKENS:   # a step fills the GPU by itself: one stream, no event traffic
+            def compute_one_stream(t, k, buf):
+                Wg, Wu, Wd = unpack_shard(buf, self.H, self.F_d)
+                self.b.tsp_mlp_ring_step(self.plan, X_p, Wg, Wu, Wd, Y_p, self.S_loc, t, self.D, main)
+
+            ring_forward(compute_one_stream, shard, self.recv_bufs, self.rank, self.D, self.group)
+            return Y_p
+        self.down_stream.wait_stream(main)            # whatever produced X_p, shard and freed Y_p comes first
+
+        def before_exchange(t):
+            if t >= 2:                                # the receive buffer of step t was last read by step t - 2
+                main.wait_event(self._down_done[t - 2])
 
         def compute(t, k, buf):
             Wg, Wu, Wd = unpack_shard(buf, self.H, self.F_d)
-            self.b.tsp_mlp_ring_step(self.plan, X_p, Wg, Wu, Wd, Y_p, self.S_loc, t, self.D)
+            if t >= 2:                                # scratch buffer t & 1 is free once down(t - 2) has run
+                main.wait_event(self._down_done[t - 2])
+            self.b.tsp_mlp_ring_step_gate(self.plan, X_p, Wg, Wu, self.S_loc, t, self.D, main)
+            self._gate_done[t].record(main)
+            self.down_stream.wait_event(self._gate_done[t])
+            self.b.tsp_mlp_ring_step_down(self.plan, Wd, Y_p, self.S_loc, t, self.D, self.down_stream)
+            self._down_done[t].record(self.down_stream)
 
-        ring_forward(compute, shard, self.recv_bufs, self.rank, self.D, self.group)
+        ring_forward(compute, shard, self.recv_bufs, self.rank, self.D, self.group, before_exchange)
+        main.wait_stream(self.down_stream)
         return Y_p
 
     def backward(self, X_p: torch.Tensor, shard: torch.Tensor, dY_p: torch.Tensor, dX_p: torch.Tensor | None = None):

@@ -32,8 +32,8 @@ def main():
     cols = slice(rank * F_d, (rank + 1) * F_d)                  # ... and keeps only its own shards
     own = ring.pack_shard(torch.from_numpy(Wg[:, cols].copy()), torch.from_numpy(Wu[:, cols].copy()),
                           torch.from_numpy(Wd[cols, :].copy()))
-    recv = [torch.empty_like(own) for _ in range(2)]
-    visited = []
+    recv = [torch.empty_like(own) for _ in range(3)]    # three take turns in the forward pass, the first two in the backward
+    visited, hook_calls = [], []
 
     # ---- forward
     Yp = np.zeros((S_loc, H))
@@ -44,7 +44,7 @@ def main():
         visited.append(k)
         Yp[...] += orc.gated_mlp_forward(Xp, wg, wu, wd)
 
-    ring.ring_forward(compute, own, recv, rank, D)
+    ring.ring_forward(compute, own, recv, rank, D, before_exchange=hook_calls.append)
 
     # ---- backward
     dXp = np.zeros((S_loc, H))
@@ -75,7 +75,7 @@ def main():
     def err(a, ref):
         return float(np.max(np.abs(a - ref)) / np.max(np.abs(ref)))
 
-    out = {"rank": rank, "D": D, "visited": visited,
+    out = {"rank": rank, "D": D, "visited": visited, "hook_calls": hook_calls,
            "err_Y": err(Yp, Y_ref[rows]), "err_dX": err(dXp, rdX[rows]),
            "err_dWg": err(dWg_own, rdWg[:, cols]), "err_dWu": err(dWu_own, rdWu[:, cols]),
            "err_dWd": err(dWd_own, rdWd[cols, :])}

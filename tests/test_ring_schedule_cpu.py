@@ -24,5 +24,6 @@ def test_ring_schedules_reach_the_unsharded_result(tmp_path, world):
     for r in range(world):
         o = json.load(open(tmp_path / f"rank{r}.json"))
         assert o["visited"] == [(r - t) % world for t in range(world)]
+        assert o["hook_calls"] == list(range(world - 1))      # once before every transfer, none after the last step
         for key in ("err_Y", "err_dX", "err_dWg", "err_dWu", "err_dWd"):
             assert o[key] <= 1e-12, (r, key, o[key])

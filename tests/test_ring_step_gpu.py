@@ -215,3 +215,50 @@ def test_ring_step_argument_errors():
         assert b.tsp_mlp_workspace_bytes_ring(plan, 0, b.TSP_WS_FORWARD) == 0
     finally:
         b.tsp_mlp_plan_destroy(plan)
+
+
+def test_gate_and_down_halves_on_two_streams_keep_the_bits():
+    # one rank, all shards local: the down projection of step t on a second stream overlaps the gate|up GEMM of
+    # step t + 1 (ordering by events, as the header prescribes); the result must equal the one-stream sequence
+    import torch
+
+    S_loc, H, F, D = 512, 256, 2048, 8
+    prob = DeviceProblem(S_loc, H, F, D, seed=36)       # X of one rank; D shards
+    plan = b.tsp_mlp_plan(H, F, D)
+    try:
+        ws = torch.empty(b.tsp_mlp_workspace_bytes_ring(plan, S_loc, b.TSP_WS_FORWARD), dtype=torch.uint8, device="cuda")
+        b.tsp_mlp_set_workspace(plan, ws)
+        Y1 = torch.full((S_loc, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        for t in range(D):
+            k = ring.shard_at_step(0, t, D)
+            b.tsp_mlp_ring_step(plan, prob.X, prob.Wg[k], prob.Wu[k], prob.Wd[k], Y1, S_loc, t, D)
+        torch.cuda.synchronize()
+        Y2 = torch.full((S_loc, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        s_gate, s_down = torch.cuda.Stream(), torch.cuda.Stream()
+        gate_done = [torch.cuda.Event() for _ in range(D)]
+        down_done = [torch.cuda.Event() for _ in range(D)]
+        for rep in range(2):                              # twice: the scratch buffers are reused across passes
+            s_gate.wait_stream(s_down)
+            for t in range(D):
+                k = ring.shard_at_step(0, t, D)
+                if t >= 2:
+                    s_gate.wait_event(down_done[t - 2])
+                b.tsp_mlp_ring_step_gate(plan, prob.X, prob.Wg[k], prob.Wu[k], S_loc, t, D, s_gate)
+                gate_done[t].record(s_gate)
+                s_down.wait_event(gate_done[t])
+                b.tsp_mlp_ring_step_down(plan, prob.Wd[k], Y2, S_loc, t, D, s_down)
+                down_done[t].record(s_down)
+            s_down.synchronize()
+            s_gate.synchronize()
+            assert b.tsp_mlp_status(plan) == b.TSP_OK
+            assert torch.equal(Y1.view(torch.int16), Y2.view(torch.int16))
+            Y2.fill_(float("nan")) if rep == 0 else None
+        with pytest.raises(b.TspError) as e:
+            b.tsp_mlp_ring_step_down(plan, prob.Wd[0], 0, S_loc, 0, D)
+        assert e.value.code == b.TSP_ERR_INVALID_ARG
+    finally:
+        b.tsp_mlp_plan_destroy(plan)
+    # and against the definition: rank 0 of a problem whose other ranks' tokens do not matter for these rows
+    X, Wg, Wu, Wd = prob.f64()
+    ref = orc.gated_mlp_forward(X, Wg, Wu, Wd)
+    assert rel_fro(tensor_to_f64(Y1), ref) <= TOL_ORACLE
