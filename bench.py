@@ -38,6 +38,9 @@ FALLBACK_BF16_TFLOPS = 1590.0
 NCU_DRAM_BYTES = {
     ("gate_up", "7b_short"): 0.6946e9 + 0.2263e9,   # profiles/ncu_full_pair_kernels_7b_train.txt (same shapes)
     ("gate_up", "train"): 0.6946e9 + 0.2263e9,
+    # summed over the six launches the gate|up phase takes at this length
+    # (profiles/dram_bytes_forward_kernels_vs_token_count.txt)
+    ("gate_up", "7b_long"): 3.237e9 + 0.802e9,
 }
 
 
