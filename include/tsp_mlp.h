@@ -147,8 +147,9 @@ tsp_status_t tsp_mlp_backward_saved(tsp_mlp_plan_t* plan, const void* X, const v
  * tsp_mlp_forward_host - the same forward for callers whose tensors live in HOST
  * memory (pinned memory gives asynchronous copies).  Copies X, Wg, Wu to device
  * staging inside the workspace, runs the gate|up kernel while Wd is still being
- * copied on a plan-owned side stream (created on first use), runs the down projection,
- * copies Y back; ordered with respect to `cuda_stream`.  Needs a workspace of tsp_mlp_workspace_bytes_host(plan, S) bytes.
+ * copied on a plan-owned side stream (created on first use), runs the down projection in four
+ * launches over token ranges and copies each range of Y back on the side stream while the next range is
+ * computed; ordered with respect to `cuda_stream` (synchronizing it is enough to read Y_host).  Needs a workspace of tsp_mlp_workspace_bytes_host(plan, S) bytes.
  */
 size_t tsp_mlp_workspace_bytes_host(const tsp_mlp_plan_t* plan, int64_t S);
 tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, const void* Wg_host,

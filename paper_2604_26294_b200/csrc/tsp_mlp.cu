@@ -67,7 +67,7 @@ struct tsp_mlp_plan {
     int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
     cudaStream_t host_copy_stream;           // tsp_mlp_forward_host: uploads Wd while the gate|up kernel runs
-    cudaEvent_t host_events[3];
+    cudaEvent_t host_events[8];
     bool host_ready;
 };
 
@@ -472,7 +472,9 @@ tsp_status_t launch_da_pair(tsp_mlp_plan_t* plan, const void* dY, const void* Wd
     return launch_da_pair_t<false>(plan, dY, Wd, dA, nullptr, nullptr, nullptr, nullptr, S, stream);
 }
 
-tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* Wd, void* Y, int64_t S, cudaStream_t stream) {
+// tile_first / tile_count: restrict the launch to a range of token tiles (default: all of them)
+tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* Wd, void* Y, int64_t S, cudaStream_t stream,
+                              int tile_first = 0, int tile_count = -1) {
     const int H = plan->H, F = plan->F, D = plan->D;
     tsp::PairDownPolicy::Params p;
     std::memset(&p, 0, sizeof(p));
@@ -485,9 +487,10 @@ tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* W
     p.m_tiles = D * p.tiles_per_rank;
     p.n_blocks = H / 256;
     const int group = plan->group > 0 ? plan->group : 8;
+    if (tile_count < 0) tile_count = p.m_tiles - tile_first;
     // chunks from the last token tiles to the first: the rows the gate|up kernel wrote last are still in L2
-    return for_tile_chunks(p.m_tiles, plan->chunk_tiles, true, [&](int first, int count) {
-        p.mt_base = first;
+    return for_tile_chunks(tile_count, plan->chunk_tiles, true, [&](int first, int count) {
+        p.mt_base = tile_first + first;
         p.m_tiles = count;
         p.group = count < group ? count : group;
         p.wide_tiles = mixed_wide_tiles(plan, 1, p.n_blocks, count * p.n_blocks, F / 64);
@@ -957,9 +960,45 @@ tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, cons
     if ((e = cudaMemcpyAsync(dWd, Wd_host, wb, cudaMemcpyHostToDevice, side)) != cudaSuccess) return cuda_fail(plan, e);
     if ((e = cudaEventRecord(plan->host_events[1], side)) != cudaSuccess) return cuda_fail(plan, e);
     // The forward proper uses only the first `a` bytes of the workspace.
-    st = forward_impl(plan, dX, dWg, dWu, dWd, dY, S, D, cuda_stream, plan->host_events[1]);
+    const int tiles_per_rank = static_cast<int>((S / D + 255) / 256), m_tiles = D * tiles_per_rank;
+    constexpr int kParts = 4;
+    if (!pairs_for_tokens(plan, S) || m_tiles < 2 * kParts || plan->phase_mask != 3) {
+        st = forward_impl(plan, dX, dWg, dWu, dWd, dY, S, D, cuda_stream, plan->host_events[1]);
+        if (st != TSP_OK) return st;
+        if ((e = cudaMemcpyAsync(Y_host, dY, xb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(plan, e);
+        return TSP_OK;
+    }
+    // The down projection runs in kParts launches over token ranges, last range first; each range of Y goes back to the
+    // host on the side stream while the next range is computed.
+    auto row_of = [&](int mt) {
+        const int64_t r = mt / tiles_per_rank, j = mt % tiles_per_rank;
+        const int64_t row = r * (S / D) + j * 256;
+        return row < S ? row : S;
+    };
+    plan->launch_count = 0;
+    Profiler prof(plan, stream);
+    st = launch_gate_up_pair(plan, dX, dWg, dWu, plan->workspace, S, stream);
     if (st != TSP_OK) return st;
-    if ((e = cudaMemcpyAsync(Y_host, dY, xb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    prof.mark();
+    if ((e = cudaStreamWaitEvent(stream, plan->host_events[1], 0)) != cudaSuccess) return cuda_fail(plan, e);   // Wd has arrived
+    const int per = m_tiles / kParts;
+    for (int q = kParts - 1; q >= 0; --q) {
+        const int first = q * per, count = q == kParts - 1 ? m_tiles - first : per;
+        st = launch_down_pair(plan, plan->workspace, dWd, dY, S, stream, first, count);
+        if (st != TSP_OK) return st;
+        const int64_t r0 = row_of(first), r1 = q == kParts - 1 ? S : row_of(first + count);
+        cudaEvent_t ev = plan->host_events[3 + q];
+        if ((e = cudaEventRecord(ev, stream)) != cudaSuccess) return cuda_fail(plan, e);
+        if ((e = cudaStreamWaitEvent(side, ev, 0)) != cudaSuccess) return cuda_fail(plan, e);
+        const size_t off = static_cast<size_t>(r0) * plan->H * 2, len = static_cast<size_t>(r1 - r0) * plan->H * 2;
+        if ((e = cudaMemcpyAsync(static_cast<uint8_t*>(Y_host) + off, dY + off, len, cudaMemcpyDeviceToHost, side)) != cudaSuccess)
+            return cuda_fail(plan, e);
+    }
+    prof.mark();
+    plan->last_forward_kernels = plan->launch_count;
+    // the caller synchronizes `stream`: make it wait for the copies on the side stream
+    if ((e = cudaEventRecord(plan->host_events[2], side)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaStreamWaitEvent(stream, plan->host_events[2], 0)) != cudaSuccess) return cuda_fail(plan, e);
     return TSP_OK;
 }
 
