@@ -548,7 +548,6 @@ def run_ring(args, wl):
 def run_attn(args, wl):
     import torch
 
-    from oracle import tsp_attn_proj_oracle as attn_orc  # cpu_baseline leg only
     from paper_2604_26294_b200 import binding as b
     from paper_2604_26294_b200 import build as _build
 
@@ -622,6 +621,8 @@ def run_attn(args, wl):
     # oracle timed on a bounded sample of rows (row-separable), host cores
     cpu = None
     if not args.no_cpu_baseline:
+        from oracle import tsp_attn_proj_oracle as attn_orc   # the only use of the oracle in this arm
+
         f = [inp.bf16_bits_to_f64(a) for a in (host.X, host.Wq, host.Wk, host.Wv, host.A, host.Wo)]
         rows = np.arange(0, S, max(1, S // 256))[:256]
         t0 = time.perf_counter()
