@@ -238,3 +238,42 @@ def test_backward_argument_errors():
         assert e.value.code == b.TSP_ERR_INVALID_ARG
     finally:
         b.tsp_attn_plan_destroy(plan)
+
+
+def test_random_shapes_and_tile_orders(monkeypatch):
+    """Seeded sweep over shapes, ragged token counts and tile-order tunables (read when a plan is created); the
+    reference here is the oracle's formulas evaluated per case on the CPU."""
+    import random
+
+    rnd = random.Random(7)
+    tun = ("TSP_MLP_BAND", "TSP_MLP_CHUNK_BANDS", "TSP_MLP_CHUNK_TILES", "TSP_MLP_GROUP", "TSP_MLP_DX_GROUP", "TSP_MLP_DW_GROUP")
+    done = 0
+    while done < 16:
+        D = rnd.choice([1, 2, 4, 8])
+        H, Hq = rnd.choice([256, 512]), rnd.choice([512, 1024])
+        Hkv = rnd.choice([h for h in (256, 512, 1024) if h <= Hq])
+        S = rnd.choice([1, 63, 200, 257, 511, 777, 1300])
+        for k in tun:
+            monkeypatch.delenv(k, raising=False)
+        if done % 4:      # every fourth case runs with the defaults
+            monkeypatch.setenv("TSP_MLP_BAND", rnd.choice(["1", "2"]))
+            monkeypatch.setenv("TSP_MLP_CHUNK_BANDS", rnd.choice(["0", "1", "2"]))
+            monkeypatch.setenv("TSP_MLP_CHUNK_TILES", rnd.choice(["0", "1", "3"]))
+            monkeypatch.setenv("TSP_MLP_GROUP", rnd.choice(["1", "3"]))
+            monkeypatch.setenv("TSP_MLP_DX_GROUP", rnd.choice(["0", "2"]))
+            monkeypatch.setenv("TSP_MLP_DW_GROUP", rnd.choice(["0", "1", "3"]))
+        host, dX, dWq, dWk, dWv, dA, dWo = _run_backward(S, H, Hq, Hkv, D, seed=100 + done)
+        _, Q, K, V, Y = _run(S, H, Hq, Hkv, D, host=host)
+        f = _f64(host)
+        g = {n: inp.bf16_bits_to_f64(getattr(host, n)) for n in ("dQ", "dK", "dV", "dY")}
+        rQ, rK, rV = orc.qkv_projection(f["X"], f["Wq"], f["Wk"], f["Wv"])
+        rY = orc.output_projection(f["A"], f["Wo"])
+        rdX, rdWq, rdWk, rdWv = orc.qkv_projection_backward(f["X"], f["Wq"], f["Wk"], f["Wv"], g["dQ"], g["dK"], g["dV"])
+        rdA, rdWo = orc.output_projection_backward(f["A"], f["Wo"], g["dY"])
+        pairs = [(Q, rQ), (K, rK), (V, rV), (Y, rY), (dX, rdX), (dA, rdA), (dWq, rdWq), (dWk, rdWk), (dWv, rdWv),
+                 (inp.unshard_columns(tensor_to_f64(dWo)), rdWo)]
+        for got, ref in pairs:
+            got = got if isinstance(got, np.ndarray) else tensor_to_f64(got)
+            assert np.all(np.isfinite(got)), (S, H, Hq, Hkv, D)
+            assert rel_fro(got, ref) <= TOL, (S, H, Hq, Hkv, D, rel_fro(got, ref))
+        done += 1
