@@ -206,7 +206,8 @@ tsp_status_t tsp_mlp_ring_step(tsp_mlp_plan_t* plan, const void* X_p, const void
  * few tokens per rank one step is less than a full round of tiles, so a caller can fill the GPU by running the
  * down projection of step t on a second stream while the gate|up GEMM of step t+1 runs on the first.  Ordering
  * the caller must provide: _down(t) after _gate(t); _gate(t+2) after _down(t) (it reuses the scratch buffer);
- * _down(t+1) after _down(t) (the accumulator).  Same bits as tsp_mlp_ring_step.
+ * _down(t+1) after _down(t) (the accumulator).  Same bits as tsp_mlp_ring_step.  (These two calls are the one
+ * exception to the rule that a plan is used on one stream at a time; the host thread is still one.)
  */
 tsp_status_t tsp_mlp_ring_step_gate(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
                                     int64_t S_loc, int t, int D, void* cuda_stream);
