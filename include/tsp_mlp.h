@@ -215,6 +215,25 @@ tsp_status_t tsp_mlp_ring_step_down(tsp_mlp_plan_t* plan, const void* Wd_k, void
                                     void* cuda_stream);
 
 /*
+ * tsp_mlp_ring_steps - n consecutive ring steps t_first .. t_first + n - 1 of ONE rank in one call (two kernels
+ * instead of 2 n): with few tokens per rank a single step is less than one round of tiles and its launches cost as
+ * much as its math, so a rank that has already received the next n shards applies them together.  The n shards
+ * are n packed buffers at a constant distance: shard i has its gate / up / down matrices at Wg_first, Wu_first,
+ * Wd_first + i * shard_stride ELEMENTS (bf16; shard_stride a multiple of 8 and at least H * F/D; ignored for n = 1),
+ * in the order the rank meets them.  The fp32 sum is carried across calls exactly as by tsp_mlp_ring_step (first call
+ * t_first = 0, last call ends at D), and the shards of a call are accumulated in tensor memory in the order given,
+ * so the result differs from the step-by-step one only in fp32 summation grouping.  Workspace:
+ * tsp_mlp_workspace_bytes_ring_group(plan, S_loc, n) bytes for the largest n used (the accumulator, then
+ * A [S_loc, n * F/D]); the calls of a pass may use different n, but not be mixed with tsp_mlp_ring_step calls (which
+ * lay the workspace out differently).  Errors as tsp_mlp_ring_step; INVALID_ARG also for a bad stride
+ * or t_first + n > D.
+ */
+size_t tsp_mlp_workspace_bytes_ring_group(const tsp_mlp_plan_t* plan, int64_t S_loc, int n_shards);
+tsp_status_t tsp_mlp_ring_steps(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_first, const void* Wu_first,
+                                const void* Wd_first, int64_t shard_stride, int n_shards, void* Y_p, int64_t S_loc,
+                                int t_first, int D, void* cuda_stream);
+
+/*
  * Backward pass of one ring step on one rank's data (the backward mirrors the forward weight movement, and the
  * partial weight gradients the ranks produce for a shard are summed to its owner: Sections 4.3.4 and 4.7).  Split
  * in two calls so that the caller can let a travelling dW accumulator arrive while the first call computes:

@@ -51,6 +51,9 @@ SIGNATURES = {
                                                      _P]),
     "tsp_mlp_ring_step_gate": (ctypes.c_int, [_P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_ring_step_down": (ctypes.c_int, [_P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
+    "tsp_mlp_workspace_bytes_ring_group": (ctypes.c_size_t, [_P, ctypes.c_int64, ctypes.c_int]),
+    "tsp_mlp_ring_steps": (ctypes.c_int, [_P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P, ctypes.c_int64,
+                                          ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_ring_step": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_forward_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, _P,
                                               ctypes.c_int64, ctypes.POINTER(ctypes.c_int), _P]),
@@ -219,6 +222,18 @@ def tsp_mlp_ring_step_down(plan, Wd_k, Y_p, S_loc: int, t: int, D: int, stream=N
     """Second half of a ring step: the shard's down projection added to the carried fp32 sum."""
     _check(load_library().tsp_mlp_ring_step_down(plan, _ptr(Wd_k), _ptr(Y_p), S_loc, t, D, _stream_handle(stream)),
            "tsp_mlp_ring_step_down", plan)
+
+
+def tsp_mlp_workspace_bytes_ring_group(plan, S_loc: int, n_shards: int) -> int:
+    return int(load_library().tsp_mlp_workspace_bytes_ring_group(plan, S_loc, n_shards))
+
+
+def tsp_mlp_ring_steps(plan, X_p, Wg_first, Wu_first, Wd_first, shard_stride: int, n_shards: int, Y_p, S_loc: int,
+                       t_first: int, D: int, stream=None) -> None:
+    """n consecutive ring steps of one rank in one call; the n packed shards lie shard_stride elements apart."""
+    _check(load_library().tsp_mlp_ring_steps(plan, _ptr(X_p), _ptr(Wg_first), _ptr(Wu_first), _ptr(Wd_first),
+                                             shard_stride, n_shards, _ptr(Y_p), S_loc, t_first, D,
+                                             _stream_handle(stream)), "tsp_mlp_ring_steps", plan)
 
 
 def tsp_mlp_ring_step_backward_dx(plan, X_p, Wg_k, Wu_k, Wd_k, dY_p, dX_p, S_loc: int, t: int, D: int, stream=None) -> None:

@@ -745,15 +745,20 @@ struct PairDownStagedPolicy {
         float* Yacc;                // [S, H] fp32
         __nv_bfloat16* Y;           // [S, H]
         int S, H, F_d, D, mode, S_loc;
+        int n_shards;               // 0: one ring step of every rank (buffer slot = rank).  n > 0: ONE rank, n consecutive
+                                    // ring steps in one launch: A is [S, n * F/D], the weight map holds the n shards in
+                                    // the order they are met
         int m_tiles, n_blocks, tiles_per_rank, group;
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
     };
     using Tile = PairDownPolicy::Tile;
-    __device__ static __forceinline__ int outer(const Params&) { return 1; }
+    __device__ static __forceinline__ int outer(const Params& p) { return p.n_shards > 0 ? p.n_shards : 1; }
     __device__ static __forceinline__ int inner(const Params& p) { return p.F_d / kBK; }
-    __device__ static __forceinline__ int select(const Params&, const Tile& tl, int) { return tl.r; }
+    __device__ static __forceinline__ int select(const Params& p, const Tile& tl, int t) {
+        return p.n_shards > 0 ? t : tl.r;
+    }
     __device__ static __forceinline__ void prefetch(const Params& p) {
         tma_prefetch_desc(&p.map_a);
         tma_prefetch_desc(&p.map_wd);
@@ -774,7 +779,7 @@ struct PairDownStagedPolicy {
     }
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int r, int i, uint32_t cta, uint32_t sa,
                                                 uint32_t sb, uint32_t bar) {
-        pair_load_kmajor(sa, &p.map_a, bar, i * kBK, tl.row0 + cta * 128, 0);
+        pair_load_kmajor(sa, &p.map_a, bar, (p.n_shards > 0 ? r * p.F_d : 0) + i * kBK, tl.row0 + cta * 128, 0);
         pair_load_mnmajor(sb, &p.map_wd, bar, tl.nb * 256 + cta * 128, i * kBK, r, 2);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {

@@ -708,6 +708,63 @@ tsp_status_t launch_forward_step(tsp_mlp_plan_t* plan, const void* X, const void
     return launch_step_down(plan, cur_d, A_step, Yacc, Y, S, n_ranks, mode, cs);
 }
 
+// [n][rows][cols] bf16 with an arbitrary distance between consecutive matrices (packed shard buffers in a row).
+bool encode_strided(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, uint64_t n, uint64_t rows, uint64_t cols,
+                    uint64_t stride_bytes, uint32_t box0, uint32_t box1) {
+    return encode_map(plan, map, base, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, cols, rows, n, cols * 2, stride_bytes, box0, box1);
+}
+
+// n consecutive ring steps of ONE rank in two launches: gate|up of the rank's tokens against the n shards (A becomes
+// [S, n * F/D]), then one down projection whose K loop runs over the n shards in the order given.
+tsp_status_t launch_steps_group(tsp_mlp_plan_t* plan, const void* X, const void* Wg0, const void* Wu0, const void* Wd0,
+                                size_t stride_bytes, int n, void* A, float* Yacc, void* Y, int64_t S, int mode,
+                                cudaStream_t cs) {
+    const int H = plan->H, F_d = plan->F / plan->D;
+    {
+        using Policy = tsp::PairGateUpPolicyT<0>;
+        Policy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_strided(plan, &p.map_wg, Wg0, n, H, F_d, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_strided(plan, &p.map_wu, Wu0, n, H, F_d, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
+        p.A = static_cast<__nv_bfloat16*>(A);
+        p.S = static_cast<int>(S); p.H = H; p.F = n * F_d; p.D = n; p.F_d = F_d;
+        p.S_loc = static_cast<int>(S);          // one rank: every token tile belongs to it
+        p.tiles_per_rank = (p.S_loc + 255) / 256;
+        p.m_tiles = p.tiles_per_rank;
+        p.jl_blocks = F_d / 128;
+        p.band = gate_band(plan, p.m_tiles);
+        p.shared_order = 1;                     // tile order: band -> shard -> column block -> token tile
+        p.act = plan->act;
+        tsp_status_t st = for_tile_chunks(p.m_tiles, plan->chunk_bands * p.band, false, [&](int first, int count) {
+            p.mt_base = first;
+            p.m_tiles = count;
+            fill_common(plan, p, count * n * p.jl_blocks);
+            return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, cs);
+        });
+        if (st != TSP_OK) return st;
+    }
+    {
+        tsp::PairDownStagedPolicy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(plan, &p.map_a, A, S, static_cast<uint64_t>(n) * F_d, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_strided(plan, &p.map_wd, Wd0, n, F_d, H, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
+        p.Yacc = Yacc;
+        p.Y = static_cast<__nv_bfloat16*>(Y);
+        p.S = static_cast<int>(S); p.H = H; p.F_d = F_d; p.D = 1;
+        p.mode = mode;
+        p.n_shards = n;
+        p.S_loc = static_cast<int>(S);
+        p.tiles_per_rank = (p.S_loc + 255) / 256;
+        p.m_tiles = p.tiles_per_rank;
+        p.n_blocks = H / 256;
+        const int group = plan->group > 0 ? plan->group : 8;
+        p.group = p.m_tiles < group ? p.m_tiles : group;
+        fill_common(plan, p, p.m_tiles * p.n_blocks);
+        return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownStagedPolicy>, p, cs);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Fixed scratch for tsp_mlp_forward_static: part of the library image, so every GPU that loads the
 // library holds these bytes until the process exits.  First 256 bytes: device status word; the rest:
@@ -1155,6 +1212,40 @@ tsp_status_t tsp_mlp_ring_step(tsp_mlp_plan_t* plan, const void* X_p, const void
     tsp_status_t st = tsp_mlp_ring_step_gate(plan, X_p, Wg_k, Wu_k, S_loc, t, D, cuda_stream);
     if (st != TSP_OK) return st;
     return tsp_mlp_ring_step_down(plan, Wd_k, Y_p, S_loc, t, D, cuda_stream);
+}
+
+size_t tsp_mlp_workspace_bytes_ring_group(const tsp_mlp_plan_t* plan, int64_t S_loc, int n_shards) {
+    if (!plan || S_loc <= 0 || n_shards < 1 || n_shards > plan->D) return 0;
+    return align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2 * n_shards, 256) +
+           align_up(static_cast<size_t>(S_loc) * plan->H * 4, 256);            // Yacc | A of the group
+}
+
+tsp_status_t tsp_mlp_ring_steps(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_first, const void* Wu_first,
+                                const void* Wd_first, int64_t shard_stride, int n_shards, void* Y_p, int64_t S_loc,
+                                int t_first, int D, void* cuda_stream) {
+    if (!plan || D != plan->D || n_shards < 1 || t_first < 0 || t_first + n_shards > D) return TSP_ERR_INVALID_ARG;
+    if (S_loc < 1 || S_loc > (1ll << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X_p || !Wg_first || !Wu_first || !Wd_first || !Y_p) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X_p) || !aligned16(Wg_first) || !aligned16(Wu_first) || !aligned16(Wd_first) || !aligned32(Y_p))
+        return TSP_ERR_INVALID_ARG;
+    const int64_t shard_elems = static_cast<int64_t>(plan->H) * (plan->F / plan->D);
+    if (n_shards > 1 && (shard_stride < shard_elems || shard_stride % 8 != 0)) return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_ring_group(plan, S_loc, n_shards))
+        return TSP_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    // the accumulator comes first, so that its place does not depend on the size of the group
+    float* Yacc = static_cast<float*>(plan->workspace);
+    uint8_t* base = static_cast<uint8_t*>(plan->workspace) + align_up(static_cast<size_t>(S_loc) * plan->H * 4, 256);
+    const bool first = t_first == 0, last = t_first + n_shards == D;
+    const int mode = first && last ? 3 : (first ? 0 : (last ? 2 : 1));
+    const size_t stride_bytes = n_shards > 1 ? static_cast<size_t>(shard_stride) * 2 : static_cast<size_t>(shard_elems) * 2;
+    plan->launch_count = 0;
+    Profiler prof(plan, cs);
+    tsp_status_t st = launch_steps_group(plan, X_p, Wg_first, Wu_first, Wd_first, stride_bytes, n_shards, base, Yacc, Y_p,
+                                         S_loc, mode, cs);
+    prof.mark();
+    plan->last_forward_kernels = plan->launch_count;
+    return st;
 }
 
 tsp_status_t tsp_mlp_ring_step_backward_dx(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,

@@ -73,6 +73,48 @@ def ring_forward(compute: Callable[[int, int, torch.Tensor], None], own_shard: t
             cur = nxt
 
 
+def ring_forward_grouped(compute: Callable[[int, int, int], None], own_shard: torch.Tensor, slots: torch.Tensor,
+                         rank: int, D: int, g: int, group=None, ordered_transport: bool = False) -> None:
+    """Algorithm 2 with g ring steps per compute call.
+
+    With few tokens per rank one ring step does not fill a GPU, so a rank lets the transfers run ahead and applies
+    g shards at a time.  slots [2g, n] is a ring of packed-shard buffers: the shard of step t lives in row t mod 2g,
+    so the g shards of a group are consecutive rows (what `tsp_mlp_ring_steps` wants).  The rank's own shard is
+    copied into row 0.  Every rank still forwards each shard it receives to p+1 exactly once: transfer t sends row
+    (t-1) mod 2g and receives row t mod 2g.  Before group j computes, the transfers for groups j and j+1 are posted,
+    so the next group's shards arrive while this one computes.
+    compute(t_first, n_steps, first_row) applies steps t_first .. t_first + n_steps - 1, whose shards are rows
+    first_row .. first_row + n_steps - 1.
+    ordered_transport: True when consecutive transfers are executed in posting order (NCCL: one stream), so that
+    a received shard can be forwarded without waiting for it on the host; False (gloo) waits before forwarding.
+    """
+    n_slots = slots.shape[0]
+    assert n_slots >= 2 * g and g >= 1
+    slots[0].copy_(own_shard)
+    reqs: dict[int, list] = {}
+    posted = 0                                        # transfers 1 .. posted have been posted
+
+    def post_up_to(t_last: int) -> None:
+        nonlocal posted
+        while posted < min(t_last, D - 1):
+            t = posted + 1                            # delivers the shard of step t
+            if not ordered_transport and t - 1 in reqs:
+                _wait(reqs[t - 1])                    # the shard about to be forwarded has arrived
+                reqs[t - 1] = []                      # (a request is waited for once only: gloo blocks on a second wait)
+            reqs[t] = _exchange(slots[(t - 1) % n_slots], slots[t % n_slots], rank, D, group)
+            posted = t
+
+    for t0 in range(0, D, g):
+        n = min(g, D - t0)
+        post_up_to(t0 + n - 1 + g)                    # this group's shards and the next group's
+        for t in range(t0, t0 + n):
+            if t in reqs:
+                _wait(reqs.pop(t))
+        compute(t0, n, t0 % n_slots)
+    for r in reqs.values():                           # sends of the last transfers
+        _wait(r)
+
+
 def ring_backward(compute_dx: Callable[[int, int, torch.Tensor], None],
                   compute_dw: Callable[[int, int, torch.Tensor, bool], None], own_shard: torch.Tensor,
                   recv_bufs: Sequence[torch.Tensor], dw_bufs: Sequence[torch.Tensor], rank: int, D: int,
@@ -124,7 +166,7 @@ class TspRingMlp:
     TWO_STREAM_MAX_TOKENS = 4096
 
     def __init__(self, H: int, F: int, D: int, rank: int, S_loc: int, group=None, training: bool = False,
-                 activation: int | None = None):
+                 activation: int | None = None, steps_per_launch: int | None = None):
         from . import binding as b   # fails loudly without the CUDA library or a GPU
 
         self.b, self.H, self.F, self.D, self.rank, self.S_loc, self.group = b, H, F, D, rank, S_loc, group
@@ -133,7 +175,14 @@ class TspRingMlp:
         self.plan = b.tsp_mlp_plan(H, F, D)
         if activation is not None:
             b.tsp_mlp_set_activation(self.plan, activation)
-        nbytes = b.tsp_mlp_workspace_bytes_ring(self.plan, S_loc, b.TSP_WS_BACKWARD if training else b.TSP_WS_FORWARD)
+        # ring steps applied per launch in the forward pass (measured on one rank's step sequence at H = 4096,
+        # F/D = 1792: 1024 tokens per rank 746 -> 1030 / 1223 TFLOP/s with 2 / 4 steps per launch; 8192 tokens 1240 -> 1373 /
+        # 1427); more steps per launch also mean more shards in flight (2 g receive buffers)
+        if steps_per_launch is None:
+            steps_per_launch = 4 if S_loc <= 2048 else 2
+        self.g = max(1, min(steps_per_launch, D))
+        nbytes = max(b.tsp_mlp_workspace_bytes_ring(self.plan, S_loc, b.TSP_WS_BACKWARD if training else b.TSP_WS_FORWARD),
+                     b.tsp_mlp_workspace_bytes_ring_group(self.plan, S_loc, self.g))
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
         b.tsp_mlp_set_workspace(self.plan, self.workspace)
         n = 3 * H * self.F_d
@@ -141,6 +190,7 @@ class TspRingMlp:
         # step t+2 is posted (the two halves of a step run on two streams, see forward())
         self.recv_bufs = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(3)] if D > 1 else []
         self.dw_bufs = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(2 if D > 1 else 1)] if training else []
+        self.slots = torch.empty(2 * self.g, n, dtype=torch.bfloat16, device=dev) if (D > 1 and self.g > 1) else None
         self.down_stream = torch.cuda.Stream(device=dev)
         self._gate_done = [torch.cuda.Event() for _ in range(D)]
         self._down_done = [torch.cuda.Event() for _ in range(D)]
@@ -161,6 +211,16 @@ class TspRingMlp:
         if Y_p is None:
             Y_p = torch.empty_like(X_p)
         main = torch.cuda.current_stream()
+        if self.slots is not None:                    # g ring steps per launch
+            n = 3 * self.H * self.F_d
+
+            def compute_group(t_first, n_steps, first_row):
+                Wg, Wu, Wd = unpack_shard(self.slots[first_row], self.H, self.F_d)
+                self.b.tsp_mlp_ring_steps(self.plan, X_p, Wg, Wu, Wd, n, n_steps, Y_p, self.S_loc, t_first, self.D, main)
+
+            ring_forward_grouped(compute_group, shard, self.slots, self.rank, self.D, self.g, self.group,
+                                 ordered_transport=True)
+            return Y_p
         if self.S_loc > self.TWO_STREAM_MAX_TOKENS:   # a step fills the GPU by itself: one stream, no event traffic
             def compute_one_stream(t, k, buf):
                 Wg, Wu, Wd = unpack_shard(buf, self.H, self.F_d)

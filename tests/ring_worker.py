@@ -46,6 +46,21 @@ def main():
 
     ring.ring_forward(compute, own, recv, rank, D, before_exchange=hook_calls.append)
 
+    # ---- forward again, two ring steps per compute call (the transfers run ahead through a ring of 4 buffers)
+    Yg = np.zeros((S_loc, H))
+    groups = []
+    slots = torch.full((4, own.numel()), float("nan"), dtype=own.dtype)
+
+    def compute_group(t_first, n_steps, first_row):
+        groups.append((t_first, n_steps, first_row))
+        for i in range(n_steps):
+            k = ring.shard_at_step(rank, t_first + i, D)
+            wg, wu, wd = (a.numpy() for a in ring.unpack_shard(slots[first_row + i], H, F_d))
+            assert np.array_equal(wu, Wu[:, k * F_d:(k + 1) * F_d]), "row does not hold the shard of that step"
+            Yg[...] += orc.gated_mlp_forward(Xp, wg, wu, wd)
+
+    ring.ring_forward_grouped(compute_group, own, slots, rank, D, 2)
+
     # ---- backward
     dXp = np.zeros((S_loc, H))
     parts = {}
@@ -76,6 +91,7 @@ def main():
         return float(np.max(np.abs(a - ref)) / np.max(np.abs(ref)))
 
     out = {"rank": rank, "D": D, "visited": visited, "hook_calls": hook_calls,
+           "groups": groups, "err_Y_grouped": err(Yg, Y_ref[rows]),
            "err_Y": err(Yp, Y_ref[rows]), "err_dX": err(dXp, rdX[rows]),
            "err_dWg": err(dWg_own, rdWg[:, cols]), "err_dWu": err(dWu_own, rdWu[:, cols]),
            "err_dWd": err(dWd_own, rdWd[cols, :])}

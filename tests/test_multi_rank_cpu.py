@@ -1,6 +1,7 @@
 """The N > 1 path of bench.py on CPU: world size 2 over gloo (replicas, max-over-ranks timing)."""
 import json
 import os
+import signal
 import socket
 import subprocess
 import sys
@@ -14,11 +15,20 @@ def _free_port():
         return s.getsockname()[1]
 
 
-def _torchrun(script_args, nproc=2, timeout=300):
+def _torchrun(script_args, nproc=2, timeout=180):
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={nproc}",
            "--master-addr", "127.0.0.1", "--master-port", str(_free_port())] + script_args
     env = dict(os.environ, OMP_NUM_THREADS="2")
-    return subprocess.run(cmd, capture_output=True, text=True, timeout=timeout, cwd=ROOT, env=env)
+    # own session, so that a hung run can be ended as a whole (launcher and workers) by its process group id
+    proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, cwd=ROOT, env=env,
+                            start_new_session=True)
+    try:
+        out, err = proc.communicate(timeout=timeout)
+    except subprocess.TimeoutExpired:
+        os.killpg(proc.pid, signal.SIGKILL)
+        out, err = proc.communicate()
+        return subprocess.CompletedProcess(cmd, -9, out, "timed out after %d s\n" % timeout + err)
+    return subprocess.CompletedProcess(cmd, proc.returncode, out, err)
 
 
 def test_max_over_ranks_and_whole_job_value(tmp_path):

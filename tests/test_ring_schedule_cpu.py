@@ -17,7 +17,7 @@ def test_neighbours_and_shard_index():
             assert all(ring.shard_at_step((r + 1) % D, t + 1, D) == met[t] for t in range(D - 1))  # it moves to p+1
 
 
-@pytest.mark.parametrize("world", [2, 3, 4])   # 3 and 4: p+1 and p-1 are different ranks, a reversed ring would show
+@pytest.mark.parametrize("world", [2, 3, 4, 5])   # 3 and 4: p+1 and p-1 are different ranks, a reversed ring would show
 def test_ring_schedules_reach_the_unsharded_result(tmp_path, world):
     res = _torchrun([os.path.join(ROOT, "tests", "ring_worker.py"), str(tmp_path)], nproc=world)
     assert res.returncode == 0, res.stderr[-3000:]
@@ -25,5 +25,7 @@ def test_ring_schedules_reach_the_unsharded_result(tmp_path, world):
         o = json.load(open(tmp_path / f"rank{r}.json"))
         assert o["visited"] == [(r - t) % world for t in range(world)]
         assert o["hook_calls"] == list(range(world - 1))      # once before every transfer, none after the last step
-        for key in ("err_Y", "err_dX", "err_dWg", "err_dWu", "err_dWd"):
+        assert [g[:2] for g in o["groups"]] == [[t0, min(2, world - t0)] for t0 in range(0, world, 2)]
+        assert [g[2] for g in o["groups"]] == [t0 % 4 for t0 in range(0, world, 2)]
+        for key in ("err_Y", "err_Y_grouped", "err_dX", "err_dWg", "err_dWu", "err_dWd"):
             assert o[key] <= 1e-12, (r, key, o[key])

@@ -262,3 +262,48 @@ def test_gate_and_down_halves_on_two_streams_keep_the_bits():
     X, Wg, Wu, Wd = prob.f64()
     ref = orc.gated_mlp_forward(X, Wg, Wu, Wd)
     assert rel_fro(tensor_to_f64(Y1), ref) <= TOL_ORACLE
+
+
+@pytest.mark.parametrize("S_loc,H,F,D,n", [(512, 256, 2048, 8, 4), (1000, 256, 1024, 4, 2), (300, 512, 768, 6, 3),
+                                           (256, 256, 1280, 5, 2), (64, 256, 512, 4, 4)])
+def test_grouped_ring_steps_match_oracle_and_single_steps(S_loc, H, F, D, n):
+    # one rank, its D shards in packed buffers a constant distance apart, n ring steps per call
+    import torch
+
+    prob = DeviceProblem(S_loc, H, F, D, seed=37)
+    F_d = F // D
+    order = [ring.shard_at_step(0, t, D) for t in range(D)]                 # the order rank 0 meets the shards
+    slot = 3 * H * F_d + 64                                                  # some slack between the packed buffers
+    packed = torch.zeros(D, slot, dtype=torch.bfloat16, device="cuda")
+    for t, k in enumerate(order):
+        packed[t, :3 * H * F_d] = ring.pack_shard(prob.Wg[k], prob.Wu[k], prob.Wd[k])
+    plan = b.tsp_mlp_plan(H, F, D)
+    try:
+        nbytes = max(b.tsp_mlp_workspace_bytes_ring_group(plan, S_loc, n), b.tsp_mlp_workspace_bytes_ring(plan, S_loc, 0))
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        b.tsp_mlp_set_workspace(plan, ws)
+        Yg = torch.full((S_loc, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        for t0 in range(0, D, n):
+            m = min(n, D - t0)                                               # the last group may be shorter
+            Wg, Wu, Wd = ring.unpack_shard(packed[t0], H, F_d)
+            b.tsp_mlp_ring_steps(plan, prob.X, Wg, Wu, Wd, slot, m, Yg, S_loc, t0, D)
+        Ys = torch.full((S_loc, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        for t, k in enumerate(order):
+            b.tsp_mlp_ring_step(plan, prob.X, prob.Wg[k], prob.Wu[k], prob.Wd[k], Ys, S_loc, t, D)
+        torch.cuda.synchronize()
+        assert b.tsp_mlp_status(plan) == b.TSP_OK
+        with pytest.raises(b.TspError) as e:
+            b.tsp_mlp_ring_steps(plan, prob.X, prob.Wg[0], prob.Wu[0], prob.Wd[0], slot, 2, Yg, S_loc, D - 1, D)
+        assert e.value.code == b.TSP_ERR_INVALID_ARG                         # t_first + n > D
+        with pytest.raises(b.TspError) as e:
+            b.tsp_mlp_ring_steps(plan, prob.X, prob.Wg[0], prob.Wu[0], prob.Wd[0], 12, 2, Yg, S_loc, 0, D)
+        assert e.value.code == b.TSP_ERR_INVALID_ARG                         # stride shorter than a matrix
+    finally:
+        b.tsp_mlp_plan_destroy(plan)
+    X, Wg64, Wu64, Wd64 = prob.f64()
+    ref = orc.gated_mlp_forward(X, Wg64, Wu64, Wd64)
+    got = tensor_to_f64(Yg)
+    assert np.all(np.isfinite(got))
+    assert rel_fro(got, ref) <= TOL_ORACLE, rel_fro(got, ref)
+    assert worst_row_error(got, ref) <= 0.08
+    assert rel_fro(got, tensor_to_f64(Ys)) <= TOL_MODES
