@@ -657,6 +657,88 @@ def run_attn(args, wl):
     b.tsp_attn_plan_destroy(plan)
 
 
+# ------------------------------------------------------------------------------------------------
+# One rank's share of the ring (opt-in, --mode rank-steps): the tokens of ONE rank (S / D of the workload) and all D
+# shards resident on this GPU, applied by the per-rank step entry points, g ring steps per launch pair.  No
+# transfers: this is the compute side of what each GPU of a D-GPU ring does per forward (and backward) pass.
+# ------------------------------------------------------------------------------------------------
+def run_rank_steps(args, wl):
+    import torch
+
+    from paper_2604_26294_b200 import binding as b
+    from paper_2604_26294_b200 import build as _build
+    from paper_2604_26294_b200 import ring
+
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("--mode rank-steps runs on one GPU")
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(0)
+    _build.build_library()
+    train = wl.name == "train" or args.backward
+    S, H, F, D = wl.S, wl.H, wl.F, wl.D
+    S_loc, F_d, g = S // D, F // D, max(1, min(args.steps_per_launch, D))
+    host = inp.make_inputs(S_loc, H, F, seed=0, with_dy=train)      # rank 0's tokens, the whole layer's weights
+
+    def dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    X_p = dev(host.X)
+    Wg, Wu, Wd = dev(inp.shard_columns(host.Wg, D)), dev(inp.shard_columns(host.Wu, D)), dev(inp.shard_rows(host.Wd, D))
+    order = [ring.shard_at_step(0, t, D) for t in range(D)]
+    packed = torch.stack([ring.pack_shard(Wg[k], Wu[k], Wd[k]) for k in order])      # row t = the shard met at step t
+    Y_p = torch.empty_like(X_p)
+    plan = b.tsp_mlp_plan(H, F, D)
+    ws = torch.empty(max(b.tsp_mlp_workspace_bytes_ring(plan, S_loc, b.TSP_WS_BACKWARD),
+                         b.tsp_mlp_workspace_bytes_ring_group(plan, S_loc, g)), dtype=torch.uint8, device="cuda")
+    b.tsp_mlp_set_workspace(plan, ws)
+    if train:
+        dY_p, dX_p = dev(host.dY), torch.empty_like(X_p)
+        dW = torch.empty(D, 3 * H * F_d, dtype=torch.float32, device="cuda")
+
+    def step():
+        for t0 in range(0, D, g):
+            a, u, d = ring.unpack_shard(packed[t0], H, F_d)
+            b.tsp_mlp_ring_steps(plan, X_p, a, u, d, packed.shape[1], min(g, D - t0), Y_p, S_loc, t0, D)
+        if train:
+            for t in range(D):
+                a, u, d = ring.unpack_shard(packed[t], H, F_d)
+                ga, gu, gd = ring.unpack_shard(dW[t], H, F_d)
+                b.tsp_mlp_ring_step_backward_dx(plan, X_p, a, u, d, dY_p, dX_p, S_loc, t, D)
+                b.tsp_mlp_ring_step_backward_dw(plan, X_p, dY_p, ga, gu, gd, S_loc, 0, D)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    assert b.tsp_mlp_status(plan) == b.TSP_OK
+    sampler = ClockSampler(0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.stop()
+    assert b.tsp_mlp_status(plan) == b.TSP_OK, "device-side wait timed out"
+    ms = e0.elapsed_time(e1) / args.steps
+    flops = (6.0 + (12.0 if train else 0.0)) * S_loc * H * F
+    launches = 2 * ((D + g - 1) // g) + (4 * D if train else 0)
+    line = {
+        "metric": METRIC, "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "pass": "forward+backward (G, U recomputed)" if train else "forward",
+                   "mode": "rank-steps (one rank's tokens, all shards local, per-rank step entry points)",
+                   "S_loc": S_loc, "H": H, "F": F, "D": D, "ring_steps_per_launch_forward": g,
+                   "us_per_ring_step": 1e3 * ms / D},
+        "clocks": sampler.summary(), "gpu_launches": int(args.steps * launches), "e2e": None, "roofline": None,
+        "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+    b.tsp_mlp_plan_destroy(plan)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -666,9 +748,12 @@ def main():
     ap.add_argument("--backward", action="store_true", help="time forward + backward (as the `train` workload does)")
     ap.add_argument("--stored-activations", action="store_true",
                     help="training step through tsp_mlp_forward_save / tsp_mlp_backward_saved (no recomputation)")
-    ap.add_argument("--mode", default="direct", choices=["direct", "staged", "ring"],
+    ap.add_argument("--steps-per-launch", type=int, default=1,
+                    help="--mode rank-steps: ring steps applied per launch pair in the forward pass")
+    ap.add_argument("--mode", default="direct", choices=["direct", "staged", "ring", "rank-steps"],
                     help="staged: Algorithm 2 step by step with the shard transfer emulated on a side stream; "
-                         "ring: D = N ranks on N GPUs, the shards travel between the GPUs")
+                         "ring: D = N ranks on N GPUs, the shards travel between the GPUs; "
+                         "rank-steps: one rank's tokens against all D shards through the per-rank step calls")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the torch-eager context measurement")
@@ -683,6 +768,8 @@ def main():
         run_reference(args, wl)
     elif args.mode == "ring":
         run_ring(args, wl)
+    elif args.mode == "rank-steps":
+        run_rank_steps(args, wl)
     else:
         run_gpu(args, wl)
 
