@@ -73,6 +73,70 @@ tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out);
 tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan);
 
 /*
+ * Plan options: how the kernels of a plan walk their tiles.  None of them changes WHAT is computed (Algorithm 2
+ * and its gradients, ring accumulation order k = (r - t) mod D included); they select kernel families, tile
+ * orders and launch cuts, i.e. speed and, for a few of them, the grouping of fp32 partial sums.  The paper has no
+ * counterpart (it runs library GEMMs); the fields exist so that every path can be selected per plan, from tests
+ * and sweeps, without touching the process environment.
+ * Fill the struct with tsp_mlp_options_default, change what is wanted, pass it to tsp_mlp_plan_ex.
+ * In every field TSP_OPT_AUTO (-1) means "the library decides from the shape".
+ *   use_pairs        1: CTA-pair (cta_group::2) kernels where the token count allows (auto); 0: single-CTA kernels only
+ *   gate_band        token tiles (256 rows) per band of the gate|up and dA tile order (auto: rows worth 32 MB of L2)
+ *   gate_order       1 (auto): all ranks of a band work on the same column block of the same shard;
+ *                    0: ring-faithful, every rank of a band on the shard it holds at that step (same results: the
+ *                    gate|up tiles are independent; 8x the weight traffic)
+ *   down_group       token tiles per group of the narrow down-projection tile order (auto: 8)
+ *   dx_group         the same for the dX kernel (auto: 8)
+ *   dw_group         hidden blocks (256 columns) per group of the weight-gradient tile order (auto: from S)
+ *   wide_mask        bit 0 down, bit 1 dX, bit 2 dW: force 256 x 512 tiles for that kernel; 0 forces 256 x 256
+ *                    everywhere; auto: a mixed list chosen per launch from the tile counts
+ *   pair_stages      shared-memory stages of the 256 x 256 pair kernels (auto: 6)
+ *   chunk_bands      token bands per launch of gate|up / dA (auto: 3; 0 = one launch however long)
+ *   chunk_tiles      token tiles per launch of down / dX (auto: 96; 0 = one launch)
+ *   dw_chunk_rounds  rounds of the CTA pairs per launch of the weight-gradient kernel (auto: about 3 ms of tiles;
+ *                    n > 0: n rounds; 0 = one launch)
+ *   phase_mask       profiling aid: bit 0 run gate|up, bit 1 run down in tsp_mlp_forward (auto: both)
+ *   timeout_ms       limit of every device-side wait (auto: 2000)
+ *   dynamic_tiles    bit mask of the kernels whose CTA pairs draw tiles from a device counter instead of taking them
+ *                    round-robin: bit 0 the short-K kernels (gate|up, dA, Q/K/V), bit 1 down projection (and the
+ *                    attention output projection), bit 2 dX, bit 3 weight gradients.  Same tiles, same bits: the
+ *                    tile -> accumulator order does not depend on which pair runs a tile.
+ *   fuse_ring_steps  1: tsp_mlp_ring_step / tsp_mlp_ring_steps run the gate|up GEMM and the down projection of their
+ *                    shard(s) as ONE launch (up to 261888 tokens per rank): gate|up tiles first, then down-projection
+ *                    tiles that wait, per 256 token rows, for the rows of A they read; 0 (auto): two launches.  Same
+ *                    bits either way.  (Measured on B200: on a par at best, so not the default.)
+ * Environment variables of the same meaning (TSP_MLP_PAIR, TSP_MLP_BAND, TSP_MLP_GATE_ORDER, TSP_MLP_GROUP,
+ * TSP_MLP_DX_GROUP, TSP_MLP_DW_GROUP, TSP_MLP_WIDE, TSP_MLP_PAIR_STAGES, TSP_MLP_CHUNK_BANDS, TSP_MLP_CHUNK_TILES,
+ * TSP_MLP_DW_CHUNK_ROUNDS (negative = one launch), TSP_MLP_PHASES, TSP_MLP_TIMEOUT_MS, TSP_MLP_DYNAMIC,
+ * TSP_MLP_FUSE_STEPS) are read
+ * when a plan is created and fill only the fields the caller left at TSP_OPT_AUTO: an explicit option wins.
+ * struct_bytes must be sizeof(tsp_mlp_options_t) as the caller was compiled (tsp_mlp_options_default sets it);
+ * a different size is refused with INVALID_ARG, as is a field outside its range.
+ */
+#define TSP_OPT_AUTO (-1)
+typedef struct {
+    uint32_t struct_bytes;
+    int use_pairs;
+    int gate_band;
+    int gate_order;
+    int down_group;
+    int dx_group;
+    int dw_group;
+    int wide_mask;
+    int pair_stages;
+    int chunk_bands;
+    int chunk_tiles;
+    int dw_chunk_rounds;
+    int phase_mask;
+    int timeout_ms;
+    int dynamic_tiles;
+    int fuse_ring_steps;
+} tsp_mlp_options_t;
+void tsp_mlp_options_default(tsp_mlp_options_t* options);
+/* tsp_mlp_plan with options (NULL options = tsp_mlp_plan).  Errors as tsp_mlp_plan. */
+tsp_status_t tsp_mlp_plan_ex(int H, int F, int D, const tsp_mlp_options_t* options, tsp_mlp_plan_t** out);
+
+/*
  * tsp_mlp_set_activation - choose the gate activation sigma of Algorithm 2 ("Activation sigma"; the paper
  * names SwiGLU as the example of a gated MLP).  TSP_ACT_SILU (default): sigma(z) = z / (1 + e^-z);
  * TSP_ACT_GELU: sigma(z) = z * Phi(z), Phi the standard normal CDF (erf form, not the tanh approximation);
@@ -274,7 +338,9 @@ tsp_status_t tsp_mlp_ring_step_backward_dw(tsp_mlp_plan_t* plan, const void* X_p
  * The caller passes only inputs and outputs, all DEVICE pointers with the layouts given at the top of this
  * file, plus optionally `timed_out_host`: a HOST int that, after `cuda_stream` has been synchronized,
  * is 0 if the kernels completed and non-zero if a bounded device-side wait expired (Y is then invalid).
- * Pass NULL to skip that copy.
+ * The int is filled by a 4-byte asynchronous copy at the end of the call: give it PINNED host memory
+ * (cudaHostAlloc / cudaHostRegister).  With ordinary pageable memory the copy makes the calling thread wait
+ * until both kernels have finished, which a latency-critical caller does not want.  Pass NULL to skip the copy.
  *
  * Limits and rules:
  *   - S * F * 2 bytes must not exceed TSP_MLP_STATIC_SCRATCH_BYTES (8 MiB: e.g. S=1024, F=4096), otherwise
@@ -285,7 +351,10 @@ tsp_status_t tsp_mlp_ring_step_backward_dw(tsp_mlp_plan_t* plan, const void* X_p
  *     entry point clears the status word on `cuda_stream` before launching; the intermediate is fully
  *     rewritten before it is read.  Two calls that overlap on the GPU (different streams, or different
  *     host threads) race on the array: serialize them on one stream.
- *   - Errors: INVALID_ARG, UNSUPPORTED_SHAPE, UNSUPPORTED_DEVICE, STATIC_LIMIT, CUDA.
+ *   - The limit of the device-side waits is 2 s, or TSP_MLP_TIMEOUT_MS milliseconds if that environment
+ *     variable is set when the first call on the device is made.
+ *   - Errors: INVALID_ARG, UNSUPPORTED_SHAPE, UNSUPPORTED_DEVICE, STATIC_LIMIT, CUDA (there is no plan to ask:
+ *     tsp_mlp_last_cuda_error(NULL) returns the cudaError_t of the last CUDA call that failed in this entry point).
  */
 #define TSP_MLP_STATIC_SCRATCH_BYTES (8u << 20)
 tsp_status_t tsp_mlp_forward_static(int H, int F, int D, const void* X, const void* Wg, const void* Wu,
@@ -309,7 +378,8 @@ tsp_status_t tsp_mlp_selftest_wait_expiry(tsp_mlp_plan_t* plan, int limit_ms, vo
 
 /* Static, never-null description of a status code. */
 const char* tsp_mlp_error_string(tsp_status_t status);
-/* The cudaError_t / CUresult value of the last failed CUDA call on this plan (0 if none). */
+/* The cudaError_t / CUresult value of the last failed CUDA call on this plan (0 if none); with plan == NULL, of the
+ * last failed CUDA call inside tsp_mlp_forward_static. */
 int tsp_mlp_last_cuda_error(const tsp_mlp_plan_t* plan);
 
 /*

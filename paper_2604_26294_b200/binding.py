@@ -31,6 +31,8 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtsp_mlp.
 _P = ctypes.c_void_p
 SIGNATURES = {
     "tsp_mlp_plan": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(_P)]),
+    "tsp_mlp_options_default": (None, [_P]),
+    "tsp_mlp_plan_ex": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, ctypes.POINTER(_P)]),
     "tsp_mlp_plan_destroy": (ctypes.c_int, [_P]),
     "tsp_mlp_set_activation": (ctypes.c_int, [_P, ctypes.c_int]),
     "tsp_mlp_workspace_bytes": (ctypes.c_size_t, [_P, ctypes.c_int64, ctypes.c_int]),
@@ -149,6 +151,34 @@ def tsp_mlp_plan(H: int, F: int, D: int):
     """Create a plan for hidden H, intermediate width F, D shards on the current device."""
     out = ctypes.c_void_p()
     _check(load_library().tsp_mlp_plan(H, F, D, ctypes.byref(out)), "tsp_mlp_plan")
+    return out
+
+
+class TspMlpOptions(ctypes.Structure):
+    """Mirror of tsp_mlp_options_t (include/tsp_mlp.h); every field defaults to TSP_OPT_AUTO."""
+
+    _fields_ = [("struct_bytes", ctypes.c_uint32)] + [(n, ctypes.c_int) for n in (
+        "use_pairs", "gate_band", "gate_order", "down_group", "dx_group", "dw_group", "wide_mask", "pair_stages",
+        "chunk_bands", "chunk_tiles", "dw_chunk_rounds", "phase_mask", "timeout_ms", "dynamic_tiles", "fuse_ring_steps")]
+
+
+def tsp_mlp_options_default() -> TspMlpOptions:
+    o = TspMlpOptions()
+    load_library().tsp_mlp_options_default(ctypes.byref(o))
+    return o
+
+
+def tsp_mlp_plan_ex(H: int, F: int, D: int, options: TspMlpOptions | None = None, **fields):
+    """tsp_mlp_plan with options: pass a TspMlpOptions, or the fields to change as keywords."""
+    if options is None and fields:
+        options = tsp_mlp_options_default()
+    for k, v in fields.items():
+        if k not in dict(TspMlpOptions._fields_):
+            raise TypeError(f"tsp_mlp_options_t has no field {k!r}")
+        setattr(options, k, v)
+    out = ctypes.c_void_p()
+    ref = ctypes.byref(options) if options is not None else None
+    _check(load_library().tsp_mlp_plan_ex(H, F, D, ref, ctypes.byref(out)), "tsp_mlp_plan_ex")
     return out
 
 

@@ -24,6 +24,7 @@ struct PairQkvPolicy {
         int S, H, Hq, Hkv;
         int m_tiles, q_blocks, kv_blocks, n_blocks, band;
         int mt_base;        // first token tile of this launch (long problems are cut into several launches)
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -88,6 +89,7 @@ struct PairOutPolicy {
         int S, H, Hq, D, Hq_d;
         int m_tiles, n_blocks, group;
         int mt_base;
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -139,6 +141,7 @@ struct PairAttnDxPolicy {
         int S, H, q_kb, kv_kb;               // k-blocks of 64 features per matrix
         int m_tiles, n_blocks, group;
         int mt_base;
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -200,6 +203,7 @@ struct PairAttnDaPolicy {
         int S, H, Hq, Hq_d;
         int m_tiles, n_blocks, band;
         int mt_base;
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -263,6 +267,7 @@ struct PairAttnDwPolicy {
         int accumulate;                    // 0: C overwritten; 1: the tile's sum is added to what C holds
         int S, k_blocks;
         int n_blocks, n_group;
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;

@@ -298,7 +298,8 @@ pair_wide_kernel(const __grid_constant__ typename Policy::Params p) {
             bool ok = true;
             uint32_t uses[2] = {0u, 0u};   // how often each column half has been filled so far
             for (int tile = pair_id; tile < p.num_tiles && ok; tile += n_pairs) {
-                const int halves = tile < p.wide_tiles ? 2 : 1;
+                // the policy decides (its list index may be offset when a long list is cut into several launches)
+                const int halves = Policy::halves_of(p, tile);
                 for (int kb = 0; kb < k_blocks && ok; ++kb) {
                     if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
                     tc_fence_after_sync();
@@ -368,12 +369,21 @@ __device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t
 __device__ __forceinline__ void carry_row256(float* acc_row, __nv_bfloat16* out, uint32_t t_row, bool live, bool add_prev,
                                              bool to_fp32) {
     float4* acc = reinterpret_cast<float4*>(acc_row);
+    // the carried values of chunk c + 1 are requested while chunk c is processed, so only the first request's latency
+    // is exposed (the loads are independent of the accumulator)
+    float4 nxt[8] = {};
+    if (live && add_prev) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) nxt[q] = acc[q];
+    }
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
-        float4 prev[8] = {};
-        if (live && add_prev) {
+        float4 prev[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) prev[q] = acc[c * 8 + q];
+        for (int q = 0; q < 8; ++q) prev[q] = nxt[q];
+        if (live && add_prev && c < 7) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) nxt[q] = acc[(c + 1) * 8 + q];
         }
         uint32_t v[32];
         tmem_ld32(t_row + c * 32, v);
@@ -401,6 +411,31 @@ __device__ __forceinline__ void carry_row256(float* acc_row, __nv_bfloat16* out,
     }
 }
 
+// One accumulator row of a gate|up tile: tensor-memory columns 0..127 hold G, 128..255 hold U; writes
+// A = act(G) * U for the 128 intermediate columns, rounded once to bf16.  Rows that are not live only drain.
+__device__ __forceinline__ void gated_row128(__nv_bfloat16* out, uint32_t t_row, bool live, int act) {
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+        uint32_t g[32], u[32];
+        tmem_ld32(t_row + c * 32, g);
+        tmem_ld32(t_row + 128 + c * 32, u);
+        tmem_ld_wait();
+        uint32_t packed[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+            packed[i] = pack_bf16x2(gate_act(g0, act) * __uint_as_float(u[2 * i]),
+                                    gate_act(g1, act) * __uint_as_float(u[2 * i + 1]));
+        }
+        if (live) {
+            st_global_256(out + c * 32, packed[0], packed[1], packed[2], packed[3], packed[4], packed[5], packed[6],
+                          packed[7]);
+            st_global_256(out + c * 32 + 16, packed[8], packed[9], packed[10], packed[11], packed[12], packed[13],
+                          packed[14], packed[15]);
+        }
+    }
+}
+
 // ---- gate | up + SwiGLU: tile = 256 tokens x 128 intermediate columns; CTA 0 loads the Wg half of B, CTA 1 the Wu half.
 // kMode 0 (forward)            : epilogue writes A = sigma(G) * U.
 // kMode 1 (backward, recompute): epilogue also reads dA (fp32, from the dA GEMM) and writes A, dG = dA*U*sigma'(G),
@@ -422,6 +457,7 @@ struct PairGateUpPolicyT {
         int act;              // gate activation
         int rank_indexed;     // staged mode: one ring step per launch; the weight tensors hold, at index r, the
                               // shard rank r currently has in its receive buffer, and A is [S, F/D]
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -466,27 +502,7 @@ struct PairGateUpPolicyT {
         const size_t off = static_cast<size_t>(tl.row0 + cta * 128 + row) * p.F +
                            (p.rank_indexed ? 0 : static_cast<size_t>(tl.k) * p.F_d) + tl.jl * 128;
         if constexpr (kMode == 0) {
-            __nv_bfloat16* out = p.A + off;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t g[32], u[32];
-                tmem_ld32(t_row + c * 32, g);
-                tmem_ld32(t_row + 128 + c * 32, u);
-                tmem_ld_wait();
-                uint32_t packed[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-                    packed[i] = pack_bf16x2(gate_act(g0, p.act) * __uint_as_float(u[2 * i]),
-                                            gate_act(g1, p.act) * __uint_as_float(u[2 * i + 1]));
-                }
-                if (live) {
-                    st_global_256(out + c * 32, packed[0], packed[1], packed[2], packed[3], packed[4], packed[5], packed[6],
-                                  packed[7]);
-                    st_global_256(out + c * 32 + 16, packed[8], packed[9], packed[10], packed[11], packed[12], packed[13],
-                                  packed[14], packed[15]);
-                }
-            }
+            gated_row128(p.A + off, t_row, live, p.act);
         } else if constexpr (kMode == 2) {
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {
@@ -580,6 +596,7 @@ struct PairDaPolicyT {
         int S, H, F, D, S_loc;
         int m_tiles, tiles_per_rank, j_tiles, band;
         int mt_base;                 // first token tile of this launch
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -671,6 +688,7 @@ struct PairDownPolicy {
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;   // mixed-width kernel: number of 256 x 512 tiles at the head of the tile list
         int mt_base;  // first token tile of this launch (a long problem is cut into several launches)
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -714,6 +732,7 @@ struct PairDownPolicy {
                           static_cast<int>(cta) * 128 + row < tl.valid);
     }
     // mixed-width kernel: tl.nb is the first 256-column block, tl.halves the number of column blocks
+    __device__ static __forceinline__ int halves_of(const Params& p, int t) { return t < p.wide_tiles ? 2 : 1; }
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
         mixed_tile(t, p.wide_tiles, p.n_blocks, p.m_tiles, true, o.mt, o.nb, o.halves);
@@ -749,6 +768,7 @@ struct PairDownStagedPolicy {
                                     // ring steps in one launch: A is [S, n * F/D], the weight map holds the n shards in
                                     // the order they are met
         int m_tiles, n_blocks, tiles_per_rank, group;
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -801,6 +821,7 @@ struct PairDxPolicy {
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;
         int mt_base;   // first token tile of this launch
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -849,6 +870,7 @@ struct PairDxPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_block(p, tl, cta, row, t_row, tl.nb);
     }
+    __device__ static __forceinline__ int halves_of(const Params& p, int t) { return t < p.wide_tiles ? 2 : 1; }
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
         mixed_tile(t, p.wide_tiles, p.n_blocks, p.m_tiles, true, o.mt, o.nb, o.halves);
@@ -885,6 +907,7 @@ struct PairDwPolicy {
         int accumulate;  // 0: dW overwritten; 1: the tile's sum is added to what dW holds (partial sums of other ranks)
         int wide_tiles;
         int tile_base;   // first entry of the tile list this launch covers (a long list is cut into several launches)
+        int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
         int* status;
         unsigned long long timeout_ns;
@@ -974,7 +997,9 @@ struct PairDwPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_cols(p, tl, cta, row, t_row, tl.nb * 256);
     }
-    // mixed-width kernel: rows of the tile grid are (family, intermediate tile)
+    // mixed-width kernel: rows of the tile grid are (family, intermediate tile); the list index is offset by tile_base
+    // when a long list is cut into several launches
+    __device__ static __forceinline__ int halves_of(const Params& p, int t) { return t + p.tile_base < p.wide_tiles ? 2 : 1; }
     __device__ static __forceinline__ Tile decode_mixed(const Params& p, int t) {
         Tile o;
         int row;

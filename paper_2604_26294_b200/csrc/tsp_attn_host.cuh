@@ -20,7 +20,7 @@ tsp_status_t tsp_attn_plan(int H, int Hq, int Hkv, int D, tsp_attn_plan_t** out)
     if (Hq % D != 0 || Hkv % D != 0 || (Hq / D) % 64 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
     if (H > (1 << 20) || Hq > (1 << 20) || Hkv > (1 << 20)) return TSP_ERR_UNSUPPORTED_SHAPE;
     tsp_mlp_plan_t* base = nullptr;
-    tsp_status_t st = make_plan(H, 0, 1, &base);  // device-side part only; the MLP fields stay unused
+    tsp_status_t st = make_plan(H, 0, 1, nullptr, &base);  // device-side part only; the MLP fields stay unused
     if (st != TSP_OK) return st;
     tsp_attn_plan_t* plan = new (std::nothrow) tsp_attn_plan_t();
     if (!plan) {
@@ -70,7 +70,7 @@ tsp_status_t tsp_attn_qkv_forward(tsp_attn_plan_t* plan, const void* X, const vo
         p.mt_base = first;
         p.m_tiles = count;
         fill_common(base, p, count * p.n_blocks);
-        return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairQkvPolicy>, p, stream);
+        return launch_pair<tsp::PairQkvPolicy>(base, p, stream);
     });
     prof.mark();
     return st;
@@ -101,7 +101,7 @@ tsp_status_t tsp_attn_out_forward(tsp_attn_plan_t* plan, const void* A, const vo
         p.m_tiles = count;
         p.group = count < group ? count : group;
         fill_common(base, p, count * p.n_blocks);
-        return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairOutPolicy>, p, stream);
+        return launch_pair<tsp::PairOutPolicy>(base, p, stream, kDynDown);
     });
     prof.mark();
     return st;
@@ -141,7 +141,7 @@ tsp_status_t tsp_attn_qkv_backward(tsp_attn_plan_t* plan, const void* X, const v
             p.m_tiles = count;
             p.group = count < group ? count : group;
             fill_common(base, p, count * p.n_blocks);
-            return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDxPolicy>, p, stream);
+            return launch_pair<tsp::PairAttnDxPolicy>(base, p, stream, kDynDx);
         });
         if (st != TSP_OK) return st;
         prof.mark();
@@ -165,7 +165,7 @@ tsp_status_t tsp_attn_qkv_backward(tsp_attn_plan_t* plan, const void* X, const v
         if (n_group < 1) n_group = 1;
         p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
         fill_common(base, p, (p.m_tiles0 + p.m_tiles1 + p.m_tiles2) * p.n_blocks);
-        return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDwPolicy>, p, stream);
+        return launch_pair<tsp::PairAttnDwPolicy>(base, p, stream, kDynDw);
     });
     if (st != TSP_OK) return st;
     prof.mark();
@@ -196,7 +196,7 @@ tsp_status_t tsp_attn_out_backward(tsp_attn_plan_t* plan, const void* A, const v
             p.mt_base = first;
             p.m_tiles = count;
             fill_common(base, p, count * p.n_blocks);
-            return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDaPolicy>, p, stream);
+            return launch_pair<tsp::PairAttnDaPolicy>(base, p, stream);
         });
         if (st != TSP_OK) return st;
         prof.mark();
@@ -219,7 +219,7 @@ tsp_status_t tsp_attn_out_backward(tsp_attn_plan_t* plan, const void* A, const v
         if (n_group < 1) n_group = 1;
         p.n_group = n_group > p.n_blocks ? p.n_blocks : n_group;
         fill_common(base, p, p.m_tiles0 * p.n_blocks);
-        return launch_pair(base, tsp::pair_gemm_kernel<tsp::PairAttnDwPolicy>, p, stream);
+        return launch_pair<tsp::PairAttnDwPolicy>(base, p, stream, kDynDw);
     });
     if (st != TSP_OK) return st;
     prof.mark();

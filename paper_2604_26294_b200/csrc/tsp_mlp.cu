@@ -15,6 +15,7 @@
 #include "bwd_kernels.cuh"
 #include "fwd_kernels.cuh"
 #include "pair_kernels.cuh"
+#include "dyn_kernels.cuh"
 
 namespace {
 
@@ -26,6 +27,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kMaxKernelsPerCall = 8;
+
+// Device control block of a plan (ints): [0] status word; [16 + 2 i] scheduler words of slot i (dynamic tile
+// hand-out: next list index, leaders done); [64 ...] two sets of per-token-tile "rows of A are ready" counters
+// of the fused ring step, which alternate from launch to launch.
+constexpr int kCtlSchedBase = 16, kCtlSchedSlots = 8;
+constexpr int kCtlReadyBase = 64, kCtlReadyCount = 1024;
+constexpr size_t kCtlBytes = (kCtlReadyBase + 2 * kCtlReadyCount) * sizeof(int);
 
 struct ProfileCall {
     cudaEvent_t ev[kMaxKernelsPerCall + 1];
@@ -65,6 +73,9 @@ struct tsp_mlp_plan {
                                 // work per launch, negative = one launch
     int chunk_tiles;            // token tiles per launch of the group-ordered kernels (down, dX); 0 = one launch
     int phase_mask;             // profiling aid (env TSP_MLP_PHASES): bit 0 = gate|up, bit 1 = down; default both
+    int dynamic_tiles;          // CTA pairs draw their tiles from a device counter instead of a fixed round-robin
+    int fuse_steps;             // per-rank ring steps: gate|up and down projection in one launch
+    int ready_parity;           // which of the two ready-counter sets the next fused launch uses
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
     cudaStream_t host_copy_stream;           // tsp_mlp_forward_host: uploads Wd while the gate|up kernel runs
     cudaEvent_t host_events[8];
@@ -369,17 +380,23 @@ tsp_status_t for_tile_chunks(int m_tiles, int chunk, bool reverse, Fn fn) {
 }
 
 template <class Params>
-void fill_common(tsp_mlp_plan_t* plan, Params& p, int num_tiles) {
+void fill_common(tsp_mlp_plan_t* plan, Params& p, int num_tiles, int sched_slot = 0) {
     p.num_tiles = num_tiles;
+    p.sched = plan->status_dev + kCtlSchedBase + 2 * sched_slot;
     p.stages = pick_stages(plan, tsp::kPairStageBytes, plan->pair_stages > 0 ? plan->pair_stages : 6);
     p.status = plan->status_dev;
     p.timeout_ns = plan->timeout_ns;
 }
 
-template <class Kernel, class Params>
-tsp_status_t launch_pair_wide(tsp_mlp_plan_t* plan, Kernel kernel, Params& p, cudaStream_t stream) {
+// Which kernels draw their tiles dynamically (bits of the plan's dynamic_tiles mask).
+constexpr int kDynGate = 1, kDynDown = 2, kDynDx = 4, kDynDw = 8;
+
+template <class Policy>
+tsp_status_t launch_pair_wide(tsp_mlp_plan_t* plan, typename Policy::Params& p, cudaStream_t stream, int kind) {
     p.stages = pick_stages(plan, tsp::kWideStageBytes, 4);
-    const size_t smem = p.stages * tsp::kWideStageBytes + sizeof(tsp::SharedCtl) + 1024;
+    const bool dynamic = (plan->dynamic_tiles & kind) != 0;
+    const size_t smem = p.stages * tsp::kWideStageBytes + sizeof(tsp::SharedCtl) + (dynamic ? sizeof(tsp::DynCtl) : 0) + 1024;
+    auto kernel = dynamic ? tsp::pair_wide_dyn_kernel<Policy> : tsp::pair_wide_kernel<Policy>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int pairs_avail = plan->sm_count / 2;
@@ -391,8 +408,8 @@ tsp_status_t launch_pair_wide(tsp_mlp_plan_t* plan, Kernel kernel, Params& p, cu
 }
 
 template <class Kernel, class Params>
-tsp_status_t launch_pair(tsp_mlp_plan_t* plan, Kernel kernel, const Params& p, cudaStream_t stream) {
-    const size_t smem = p.stages * tsp::kPairStageBytes + sizeof(tsp::SharedCtl) + 1024;
+tsp_status_t launch_pair_kernel(tsp_mlp_plan_t* plan, Kernel kernel, const Params& p, size_t extra_smem, cudaStream_t stream) {
+    const size_t smem = p.stages * tsp::kPairStageBytes + sizeof(tsp::SharedCtl) + extra_smem + 1024;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int pairs_avail = plan->sm_count / 2;
@@ -401,6 +418,14 @@ tsp_status_t launch_pair(tsp_mlp_plan_t* plan, Kernel kernel, const Params& p, c
     ++plan->launch_count;
     e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
+}
+
+// 256 x 256 tiles of `Policy`: CTA pairs take them round-robin, or draw them from the plan's scheduler words
+template <class Policy>
+tsp_status_t launch_pair(tsp_mlp_plan_t* plan, const typename Policy::Params& p, cudaStream_t stream, int kind = kDynGate) {
+    if (plan->dynamic_tiles & kind)
+        return launch_pair_kernel(plan, tsp::pair_dyn_kernel<tsp::DynOf<Policy>>, p, sizeof(tsp::DynCtl), stream);
+    return launch_pair_kernel(plan, tsp::pair_gemm_kernel<Policy>, p, 0, stream);
 }
 
 template <int kMode>
@@ -430,7 +455,7 @@ tsp_status_t launch_gate_pair(tsp_mlp_plan_t* plan, const void* X, const void* W
         p.mt_base = first;
         p.m_tiles = count;
         fill_common(plan, p, count * D * p.jl_blocks);
-        return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
+        return launch_pair<Policy>(plan, p, stream);
     });
 }
 
@@ -464,7 +489,7 @@ tsp_status_t launch_da_pair_t(tsp_mlp_plan_t* plan, const void* dY, const void* 
         p.mt_base = first;
         p.m_tiles = count;
         fill_common(plan, p, count * p.j_tiles);
-        return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
+        return launch_pair<Policy>(plan, p, stream);
     });
 }
 
@@ -496,10 +521,10 @@ tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* W
         p.wide_tiles = mixed_wide_tiles(plan, 1, p.n_blocks, count * p.n_blocks, F / 64);
         if (p.wide_tiles > 0) {
             fill_common(plan, p, count * p.n_blocks - p.wide_tiles);   // wide tiles count once in the list
-            return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDownPolicy>, p, stream);
+            return launch_pair_wide<tsp::PairDownPolicy>(plan, p, stream, kDynDown);
         }
         fill_common(plan, p, count * p.n_blocks);
-        return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownPolicy>, p, stream);
+        return launch_pair<tsp::PairDownPolicy>(plan, p, stream, kDynDown);
     });
 }
 
@@ -528,10 +553,10 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
         p.wide_tiles = mixed_wide_tiles(plan, 2, p.n_blocks, count * p.n_blocks, 2 * F / 64);
         if (p.wide_tiles > 0) {
             fill_common(plan, p, count * p.n_blocks - p.wide_tiles);
-            return launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDxPolicy>, p, stream);
+            return launch_pair_wide<tsp::PairDxPolicy>(plan, p, stream, kDynDx);
         }
         fill_common(plan, p, count * p.n_blocks);
-        return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDxPolicy>, p, stream);
+        return launch_pair<tsp::PairDxPolicy>(plan, p, stream, kDynDx);
     });
 }
 
@@ -574,8 +599,8 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     return for_tile_chunks(list, chunk, false, [&](int first, int count) {
         p.tile_base = first;
         fill_common(plan, p, count);
-        return p.wide_tiles > 0 ? launch_pair_wide(plan, tsp::pair_wide_kernel<tsp::PairDwPolicy>, p, stream)
-                                : launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDwPolicy>, p, stream);
+        return p.wide_tiles > 0 ? launch_pair_wide<tsp::PairDwPolicy>(plan, p, stream, kDynDw)
+                                : launch_pair<tsp::PairDwPolicy>(plan, p, stream, kDynDw);
     });
 }
 
@@ -668,7 +693,7 @@ tsp_status_t launch_step_gate(tsp_mlp_plan_t* plan, const void* X, const void* c
         p.rank_indexed = 1;
         p.act = plan->act;
         fill_common(plan, p, p.m_tiles * p.jl_blocks);
-        st = launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, cs);
+        st = launch_pair<Policy>(plan, p, cs);
         if (st != TSP_OK) return st;
     }
     return TSP_OK;
@@ -693,8 +718,8 @@ tsp_status_t launch_step_down(tsp_mlp_plan_t* plan, const void* cur_d, const voi
         p.n_blocks = H / 256;
         const int group = plan->group > 0 ? plan->group : 8;
         p.group = p.m_tiles < group ? p.m_tiles : group;
-        fill_common(plan, p, p.m_tiles * p.n_blocks);
-        st = launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownStagedPolicy>, p, cs);
+        fill_common(plan, p, p.m_tiles * p.n_blocks, 1);   // own scheduler words: may run beside the next step's gate|up GEMM
+        st = launch_pair<tsp::PairDownStagedPolicy>(plan, p, cs, kDynDown);
         if (st != TSP_OK) return st;
     }
     return TSP_OK;
@@ -740,7 +765,7 @@ tsp_status_t launch_steps_group(tsp_mlp_plan_t* plan, const void* X, const void*
             p.mt_base = first;
             p.m_tiles = count;
             fill_common(plan, p, count * n * p.jl_blocks);
-            return launch_pair(plan, tsp::pair_gemm_kernel<Policy>, p, cs);
+            return launch_pair<Policy>(plan, p, cs);
         });
         if (st != TSP_OK) return st;
     }
@@ -761,8 +786,51 @@ tsp_status_t launch_steps_group(tsp_mlp_plan_t* plan, const void* X, const void*
         const int group = plan->group > 0 ? plan->group : 8;
         p.group = p.m_tiles < group ? p.m_tiles : group;
         fill_common(plan, p, p.m_tiles * p.n_blocks);
-        return launch_pair(plan, tsp::pair_gemm_kernel<tsp::PairDownStagedPolicy>, p, cs);
+        return launch_pair<tsp::PairDownStagedPolicy>(plan, p, cs, kDynDown);
     }
+}
+
+// The same n ring steps of one rank as ONE launch (PairFusedStepPolicy): gate|up tiles, then down-projection tiles
+// that wait for their token rows of A.  Same tiles, same K order, same epilogues as launch_steps_group: same bits.
+bool fused_steps_possible(const tsp_mlp_plan_t* plan, int64_t S) {
+    return plan->fuse_steps && (S + 255) / 256 < kCtlReadyCount;   // one counter per token tile + one for all of them
+}
+
+tsp_status_t launch_steps_fused(tsp_mlp_plan_t* plan, const void* X, const void* Wg0, const void* Wu0, const void* Wd0,
+                                size_t stride_bytes, int n, void* A, float* Yacc, void* Y, int64_t S, int mode,
+                                cudaStream_t cs) {
+    using Policy = tsp::PairFusedStepPolicy;
+    const int H = plan->H, F_d = plan->F / plan->D;
+    Policy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_strided(plan, &p.map_wg, Wg0, n, H, F_d, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_strided(plan, &p.map_wu, Wu0, n, H, F_d, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_matrix(plan, &p.map_a, A, S, static_cast<uint64_t>(n) * F_d, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_strided(plan, &p.map_wd, Wd0, n, F_d, H, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
+    p.A = static_cast<__nv_bfloat16*>(A);
+    p.Yacc = Yacc;
+    p.Y = static_cast<__nv_bfloat16*>(Y);
+    p.S_loc = static_cast<int>(S); p.H = H; p.F_d = F_d; p.n_shards = n;
+    p.mode = mode;
+    p.act = plan->act;
+    p.m_tiles = static_cast<int>((S + 255) / 256);
+    p.jl_blocks = F_d / 128;
+    p.n_blocks = H / 256;
+    p.gate_tiles = p.m_tiles * p.jl_blocks * n;
+    p.band = gate_band(plan, p.m_tiles);
+    const int group = plan->group > 0 ? plan->group : 8;
+    p.group = p.m_tiles < group ? p.m_tiles : group;
+    int* ready = plan->status_dev + kCtlReadyBase;
+    p.ready = ready + plan->ready_parity * kCtlReadyCount;
+    p.ready_clear = ready + (plan->ready_parity ^ 1) * kCtlReadyCount;
+    p.ready_clear_count = kCtlReadyCount;
+    p.ready_target = 8 * p.jl_blocks * n;   // the eight epilogue warps of every gate|up tile of a token tile
+    p.ready_all = p.ready + kCtlReadyCount - 1;   // last counter of the set: all token tiles together
+    p.ready_all_target = p.ready_target * p.m_tiles;
+    plan->ready_parity ^= 1;
+    fill_common(plan, p, p.gate_tiles + p.m_tiles * p.n_blocks);
+    return launch_pair_kernel(plan, tsp::pair_dyn_kernel<Policy>, p, sizeof(tsp::DynCtl), cs);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -780,8 +848,10 @@ struct StaticDeviceState {
     unsigned char* scratch;  // device address of g_static_scratch on this device
     int sm_count;
     int max_smem;
+    unsigned long long timeout_ns;  // limit of the device-side waits (TSP_MLP_TIMEOUT_MS, read at set-up; default 2 s)
     EncodeTiledFn encode;
 };
+int g_static_last_cuda_error = 0;   // cudaError_t of the last failed CUDA call inside tsp_mlp_forward_static
 constexpr int kMaxStaticDevices = 64;
 StaticDeviceState g_static_state[kMaxStaticDevices];
 std::mutex g_static_mutex;
@@ -806,6 +876,11 @@ tsp_status_t static_device_setup(int dev, StaticDeviceState** out) {
         if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || !ptr)
             return TSP_ERR_CUDA;
         st.scratch = ptr;
+        st.timeout_ns = 2000ull * 1000 * 1000;
+        if (const char* t = std::getenv("TSP_MLP_TIMEOUT_MS")) {
+            const long ms = std::atol(t);
+            if (ms > 0) st.timeout_ns = static_cast<unsigned long long>(ms) * 1000 * 1000;
+        }
         st.sm_count = sms;
         st.max_smem = smem;
         st.encode = reinterpret_cast<EncodeTiledFn>(fn);
@@ -824,18 +899,39 @@ extern "C" {
 
 // Device-side part of a plan, common to the MLP and the attention-projection entry points: device properties, the
 // tensor-map encoder, the status word, tunables.  The caller has validated the shape arguments it passes.
-static tsp_status_t make_plan(int H, int F, int D, tsp_mlp_plan_t** out);
+static tsp_status_t make_plan(int H, int F, int D, const tsp_mlp_options_t* opt, tsp_mlp_plan_t** out);
 
-tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
+void tsp_mlp_options_default(tsp_mlp_options_t* o) {
+    if (!o) return;
+    o->struct_bytes = static_cast<uint32_t>(sizeof(tsp_mlp_options_t));
+    o->use_pairs = o->gate_band = o->gate_order = o->down_group = o->dx_group = o->dw_group = TSP_OPT_AUTO;
+    o->wide_mask = o->pair_stages = o->chunk_bands = o->chunk_tiles = o->dw_chunk_rounds = TSP_OPT_AUTO;
+    o->phase_mask = o->timeout_ms = o->dynamic_tiles = o->fuse_ring_steps = TSP_OPT_AUTO;
+}
+
+static bool options_valid(const tsp_mlp_options_t* o) {
+    if (o->struct_bytes != sizeof(tsp_mlp_options_t)) return false;
+    auto in = [](int v, int lo, int hi) { return v == TSP_OPT_AUTO || (v >= lo && v <= hi); };
+    return in(o->use_pairs, 0, 1) && in(o->gate_band, 1, 1 << 16) && in(o->gate_order, 0, 1) &&
+           in(o->down_group, 1, 1 << 16) && in(o->dx_group, 1, 1 << 16) && in(o->dw_group, 1, 1 << 16) &&
+           in(o->wide_mask, 0, 7) && in(o->pair_stages, 2, tsp::kMaxStages) && in(o->chunk_bands, 0, 1 << 16) &&
+           in(o->chunk_tiles, 0, 1 << 20) && in(o->dw_chunk_rounds, 0, 1 << 20) && in(o->phase_mask, 0, 3) &&
+           in(o->timeout_ms, 1, 60000) && in(o->dynamic_tiles, 0, 15) && in(o->fuse_ring_steps, 0, 1);
+}
+
+tsp_status_t tsp_mlp_plan_ex(int H, int F, int D, const tsp_mlp_options_t* options, tsp_mlp_plan_t** out) {
     if (!out) return TSP_ERR_INVALID_ARG;
     *out = nullptr;
     if (H <= 0 || F <= 0 || D <= 0 || D > 64) return TSP_ERR_INVALID_ARG;
+    if (options && !options_valid(options)) return TSP_ERR_INVALID_ARG;
     if (F % D != 0 || (F / D) % 128 != 0 || H % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
     if (H > (1 << 20) || F > (1 << 24)) return TSP_ERR_UNSUPPORTED_SHAPE;
-    return make_plan(H, F, D, out);
+    return make_plan(H, F, D, options, out);
 }
 
-static tsp_status_t make_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
+tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out) { return tsp_mlp_plan_ex(H, F, D, nullptr, out); }
+
+static tsp_status_t make_plan(int H, int F, int D, const tsp_mlp_options_t* opt, tsp_mlp_plan_t** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return TSP_ERR_CUDA;
@@ -855,32 +951,40 @@ static tsp_status_t make_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
     plan->workspace_bytes = 0;
     plan->last_cuda_error = 0;
     plan->profile_next = 0;
-    plan->timeout_ns = 2000ull * 1000 * 1000;
-    if (const char* t = std::getenv("TSP_MLP_TIMEOUT_MS")) {
-        const long ms = std::atol(t);
-        if (ms > 0) plan->timeout_ns = static_cast<unsigned long long>(ms) * 1000 * 1000;
-    }
-    auto env_int = [](const char* name, int dflt) {
-        const char* v = std::getenv(name);
+    tsp_mlp_options_t o;
+    if (opt) o = *opt; else tsp_mlp_options_default(&o);
+    // an explicit option wins; a field left at "auto" takes the environment variable, if set, else the default
+    auto pick = [](int option, const char* env, int dflt) {
+        if (option != TSP_OPT_AUTO) return option;
+        const char* v = std::getenv(env);
         return v ? std::atoi(v) : dflt;
     };
-    plan->use_pairs = env_int("TSP_MLP_PAIR", 1);
-    plan->band = env_int("TSP_MLP_BAND", 0);
-    plan->shared_order = env_int("TSP_MLP_GATE_ORDER", 1);
-    plan->group = env_int("TSP_MLP_GROUP", 0);
-    plan->pair_stages = env_int("TSP_MLP_PAIR_STAGES", 0);
+    const int timeout_ms = pick(o.timeout_ms, "TSP_MLP_TIMEOUT_MS", 2000);
+    plan->timeout_ns = static_cast<unsigned long long>(timeout_ms > 0 ? timeout_ms : 2000) * 1000 * 1000;
+    plan->use_pairs = pick(o.use_pairs, "TSP_MLP_PAIR", 1);
+    plan->band = pick(o.gate_band, "TSP_MLP_BAND", 0);
+    plan->shared_order = pick(o.gate_order, "TSP_MLP_GATE_ORDER", 1);
+    plan->group = pick(o.down_group, "TSP_MLP_GROUP", 0);
+    plan->pair_stages = pick(o.pair_stages, "TSP_MLP_PAIR_STAGES", 0);
     plan->last_backward_kernels = 3;
     plan->last_forward_kernels = 2;
     plan->launch_count = 0;
     plan->host_ready = false;
-    plan->phase_mask = env_int("TSP_MLP_PHASES", 3);
+    plan->phase_mask = pick(o.phase_mask, "TSP_MLP_PHASES", 3);
     plan->act = TSP_ACT_SILU;
-    plan->wide_mask = env_int("TSP_MLP_WIDE", -1);   // -1: decide per launch from the tile counts
-    plan->dw_group = env_int("TSP_MLP_DW_GROUP", 0);
-    plan->chunk_bands = env_int("TSP_MLP_CHUNK_BANDS", 3);
-    plan->chunk_tiles = env_int("TSP_MLP_CHUNK_TILES", 96);
-    plan->dw_chunk_rounds = env_int("TSP_MLP_DW_CHUNK_ROUNDS", 0);
-    plan->dx_group = env_int("TSP_MLP_DX_GROUP", 0);
+    plan->wide_mask = pick(o.wide_mask, "TSP_MLP_WIDE", -1);   // -1: decide per launch from the tile counts
+    plan->dw_group = pick(o.dw_group, "TSP_MLP_DW_GROUP", 0);
+    plan->chunk_bands = pick(o.chunk_bands, "TSP_MLP_CHUNK_BANDS", 3);
+    plan->chunk_tiles = pick(o.chunk_tiles, "TSP_MLP_CHUNK_TILES", 96);
+    // option: 0 = one launch, n > 0 = n rounds; plan / environment: negative = one launch, 0 = about 3 ms per launch
+    plan->dw_chunk_rounds = o.dw_chunk_rounds == TSP_OPT_AUTO ? pick(TSP_OPT_AUTO, "TSP_MLP_DW_CHUNK_ROUNDS", 0)
+                                                              : (o.dw_chunk_rounds == 0 ? -1 : o.dw_chunk_rounds);
+    plan->dx_group = pick(o.dx_group, "TSP_MLP_DX_GROUP", 0);
+    plan->dynamic_tiles = pick(o.dynamic_tiles, "TSP_MLP_DYNAMIC", 0);
+    // measured: one fused launch is on a par with two launches at best (it saves a kernel boundary, but its phase
+    // change costs as much), so two launches stay the default
+    plan->fuse_steps = pick(o.fuse_ring_steps, "TSP_MLP_FUSE_STEPS", 0);
+    plan->ready_parity = 0;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
@@ -889,8 +993,8 @@ static tsp_status_t make_plan(int H, int F, int D, tsp_mlp_plan_t** out) {
         return TSP_ERR_CUDA;
     }
     plan->encode = reinterpret_cast<EncodeTiledFn>(fn);
-    e = cudaMalloc(reinterpret_cast<void**>(&plan->status_dev), sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(plan->status_dev, 0, sizeof(int));
+    e = cudaMalloc(reinterpret_cast<void**>(&plan->status_dev), kCtlBytes);
+    if (e == cudaSuccess) e = cudaMemset(plan->status_dev, 0, kCtlBytes);
     if (e != cudaSuccess) {
         if (plan->status_dev) cudaFree(plan->status_dev);
         delete plan;
@@ -1209,6 +1313,21 @@ tsp_status_t tsp_mlp_ring_step_down(tsp_mlp_plan_t* plan, const void* Wd_k, void
 tsp_status_t tsp_mlp_ring_step(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_k, const void* Wu_k,
                                const void* Wd_k, void* Y_p, int64_t S_loc, int t, int D, void* cuda_stream) {
     if (!Wd_k || !Y_p || !aligned16(Wd_k) || !aligned32(Y_p)) return TSP_ERR_INVALID_ARG;   // before anything is launched
+    if (plan && fused_steps_possible(plan, S_loc)) {
+        void* A_step = nullptr;
+        float* Yacc = nullptr;
+        tsp_status_t fs = ring_step_setup(plan, S_loc, t, D, &A_step, &Yacc);
+        if (fs != TSP_OK) return fs;
+        if (!X_p || !Wg_k || !Wu_k || !aligned16(X_p) || !aligned16(Wg_k) || !aligned16(Wu_k)) return TSP_ERR_INVALID_ARG;
+        cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+        plan->launch_count = 0;
+        Profiler prof(plan, cs);
+        fs = launch_steps_fused(plan, X_p, Wg_k, Wu_k, Wd_k, static_cast<size_t>(plan->H) * (plan->F / plan->D) * 2, 1,
+                                A_step, Yacc, Y_p, S_loc, D == 1 ? 3 : (t == 0 ? 0 : (t == D - 1 ? 2 : 1)), cs);
+        prof.mark();
+        plan->last_forward_kernels = plan->launch_count;
+        return fs;
+    }
     tsp_status_t st = tsp_mlp_ring_step_gate(plan, X_p, Wg_k, Wu_k, S_loc, t, D, cuda_stream);
     if (st != TSP_OK) return st;
     return tsp_mlp_ring_step_down(plan, Wd_k, Y_p, S_loc, t, D, cuda_stream);
@@ -1241,8 +1360,11 @@ tsp_status_t tsp_mlp_ring_steps(tsp_mlp_plan_t* plan, const void* X_p, const voi
     const size_t stride_bytes = n_shards > 1 ? static_cast<size_t>(shard_stride) * 2 : static_cast<size_t>(shard_elems) * 2;
     plan->launch_count = 0;
     Profiler prof(plan, cs);
-    tsp_status_t st = launch_steps_group(plan, X_p, Wg_first, Wu_first, Wd_first, stride_bytes, n_shards, base, Yacc, Y_p,
-                                         S_loc, mode, cs);
+    tsp_status_t st = fused_steps_possible(plan, S_loc)
+                          ? launch_steps_fused(plan, X_p, Wg_first, Wu_first, Wd_first, stride_bytes, n_shards, base, Yacc,
+                                               Y_p, S_loc, mode, cs)
+                          : launch_steps_group(plan, X_p, Wg_first, Wu_first, Wd_first, stride_bytes, n_shards, base, Yacc,
+                                               Y_p, S_loc, mode, cs);
     prof.mark();
     plan->last_forward_kernels = plan->launch_count;
     return st;
@@ -1436,20 +1558,32 @@ tsp_status_t tsp_mlp_forward_static(int H, int F, int D, const void* X, const vo
     tmp.workspace = sd->scratch + kStaticHeaderBytes;
     tmp.workspace_bytes = kStaticScratchBytes;
     tmp.last_cuda_error = 0;
-    tmp.timeout_ns = 2000ull * 1000 * 1000;
+    tmp.timeout_ns = sd->timeout_ns;
     tmp.encode = sd->encode;
     tmp.profile_next = 0;
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     // The array keeps what the previous call left: the status word has to start at zero.
-    if (cudaMemsetAsync(sd->scratch, 0, kStaticHeaderBytes, stream) != cudaSuccess) return TSP_ERR_CUDA;
+    {
+        cudaError_t e = cudaMemsetAsync(sd->scratch, 0, kStaticHeaderBytes, stream);
+        if (e != cudaSuccess) {
+            g_static_last_cuda_error = static_cast<int>(e);
+            return TSP_ERR_CUDA;
+        }
+    }
     st = launch_gate_up(&tmp, X, Wg, Wu, tmp.workspace, S, stream);
-    if (st != TSP_OK) return st;
-    st = launch_down(&tmp, tmp.workspace, Wd, Y, S, stream);
-    if (st != TSP_OK) return st;
-    if (timed_out_host &&
-        cudaMemcpyAsync(timed_out_host, sd->scratch, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-        return TSP_ERR_CUDA;
+    if (st == TSP_OK) st = launch_down(&tmp, tmp.workspace, Wd, Y, S, stream);
+    if (st != TSP_OK) {
+        g_static_last_cuda_error = tmp.last_cuda_error;   // the stack plan is gone after this call
+        return st;
+    }
+    if (timed_out_host) {
+        cudaError_t e = cudaMemcpyAsync(timed_out_host, sd->scratch, sizeof(int), cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) {
+            g_static_last_cuda_error = static_cast<int>(e);
+            return TSP_ERR_CUDA;
+        }
+    }
     return TSP_OK;
 }
 
@@ -1460,7 +1594,9 @@ tsp_status_t tsp_mlp_status(tsp_mlp_plan_t* plan) {
     if (e != cudaSuccess) return cuda_fail(plan, e);
     if (v != 0) {
         plan->last_cuda_error = v;
-        e = cudaMemset(plan->status_dev, 0, sizeof(int));
+        // kernels that gave up may have left scheduler words and ready counters half-way: start from zero again
+        e = cudaMemset(plan->status_dev, 0, kCtlBytes);
+        plan->ready_parity = 0;
         if (e != cudaSuccess) return cuda_fail(plan, e);
         return TSP_ERR_DEVICE_TIMEOUT;
     }
@@ -1489,7 +1625,7 @@ const char* tsp_mlp_error_string(tsp_status_t s) {
     return "unknown status";
 }
 
-int tsp_mlp_last_cuda_error(const tsp_mlp_plan_t* plan) { return plan ? plan->last_cuda_error : 0; }
+int tsp_mlp_last_cuda_error(const tsp_mlp_plan_t* plan) { return plan ? plan->last_cuda_error : g_static_last_cuda_error; }
 
 tsp_status_t tsp_mlp_ring_order(const tsp_mlp_plan_t* plan, int* table_host) {
     if (!plan || !table_host) return TSP_ERR_INVALID_ARG;

@@ -70,3 +70,24 @@ def test_no_gpu_means_loud_failure_not_fallback(lib):
         pytest.skip("a GPU is present")
     with pytest.raises(b.TspError):
         b.tsp_mlp_plan(256, 768, 2)
+
+
+def test_plan_options_defaults_and_validation(lib):
+    o = b.tsp_mlp_options_default()
+    assert o.struct_bytes == ctypes.sizeof(b.TspMlpOptions)
+    assert all(getattr(o, n) == -1 for n, _ in b.TspMlpOptions._fields_[1:])
+    out = ctypes.c_void_p()
+    # option checks come before any device call, so they can be exercised without a GPU
+    o.wide_mask = 8
+    assert lib.tsp_mlp_plan_ex(256, 768, 2, ctypes.byref(o), ctypes.byref(out)) == b.TSP_ERR_INVALID_ARG
+    o = b.tsp_mlp_options_default()
+    o.struct_bytes = 8
+    assert lib.tsp_mlp_plan_ex(256, 768, 2, ctypes.byref(o), ctypes.byref(out)) == b.TSP_ERR_INVALID_ARG
+    o = b.tsp_mlp_options_default()
+    o.timeout_ms = 0
+    assert lib.tsp_mlp_plan_ex(256, 768, 2, ctypes.byref(o), ctypes.byref(out)) == b.TSP_ERR_INVALID_ARG
+    o = b.tsp_mlp_options_default()
+    assert lib.tsp_mlp_plan_ex(128, 768, 2, ctypes.byref(o), ctypes.byref(out)) == b.TSP_ERR_UNSUPPORTED_SHAPE
+    assert not out.value
+    with pytest.raises(TypeError):
+        b.tsp_mlp_plan_ex(256, 768, 2, no_such_field=1)

@@ -307,3 +307,51 @@ def test_grouped_ring_steps_match_oracle_and_single_steps(S_loc, H, F, D, n):
     assert rel_fro(got, ref) <= TOL_ORACLE, rel_fro(got, ref)
     assert worst_row_error(got, ref) <= 0.08
     assert rel_fro(got, tensor_to_f64(Ys)) <= TOL_MODES
+
+
+@pytest.mark.parametrize("S_loc,H,F,D,n", [(1024, 1024, 7168, 4, 1), (1024, 512, 3584, 2, 2), (300, 512, 768, 6, 3),
+                                           (2304, 256, 1024, 4, 4), (40, 256, 512, 4, 1)])
+def test_fused_ring_steps_keep_the_bits_of_the_two_launch_path(S_loc, H, F, D, n):
+    # One launch per call (gate|up tiles, then down-projection tiles that wait for their token rows of A) against
+    # the two-launch path selected by a plan option: same tiles, same K order, same epilogues, so the same bits.
+    # Three passes with the fused plan: the ready counters alternate between two sets and must come back clean.
+    import torch
+
+    prob = DeviceProblem(S_loc, H, F, D, seed=38)
+    F_d = F // D
+    order = [ring.shard_at_step(0, t, D) for t in range(D)]
+    packed = torch.stack([ring.pack_shard(prob.Wg[k], prob.Wu[k], prob.Wd[k]) for k in order])
+    results = {}
+    for fused in (1, 0):
+        plan = b.tsp_mlp_plan_ex(H, F, D, fuse_ring_steps=fused)
+        try:
+            nbytes = max(b.tsp_mlp_workspace_bytes_ring_group(plan, S_loc, n),
+                         b.tsp_mlp_workspace_bytes_ring(plan, S_loc, b.TSP_WS_FORWARD))
+            ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+            b.tsp_mlp_set_workspace(plan, ws)
+            outs = []
+            for rep in range(3 if fused else 1):
+                Y = torch.full((S_loc, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+                ws.fill_(0xFF)                                   # stale scratch must not matter
+                if n == 1:
+                    for t, k in enumerate(order):
+                        b.tsp_mlp_ring_step(plan, prob.X, prob.Wg[k], prob.Wu[k], prob.Wd[k], Y, S_loc, t, D)
+                else:
+                    for t0 in range(0, D, n):
+                        Wg, Wu, Wd = ring.unpack_shard(packed[t0], H, F_d)
+                        b.tsp_mlp_ring_steps(plan, prob.X, Wg, Wu, Wd, packed.shape[1], min(n, D - t0), Y, S_loc, t0, D)
+                torch.cuda.synchronize()
+                assert b.tsp_mlp_status(plan) == b.TSP_OK
+                outs.append(Y)
+            calls = D if n == 1 else (D + n - 1) // n
+            assert b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD) == (1 if fused else 2), calls
+            results[fused] = outs
+        finally:
+            b.tsp_mlp_plan_destroy(plan)
+    for Y in results[1]:
+        assert torch.equal(Y.view(torch.int16), results[0][0].view(torch.int16))
+    X, Wg64, Wu64, Wd64 = prob.f64()
+    ref = orc.gated_mlp_forward(X, Wg64, Wu64, Wd64)
+    got = tensor_to_f64(results[1][0])
+    assert rel_fro(got, ref) <= TOL_ORACLE, rel_fro(got, ref)
+    assert worst_row_error(got, ref) <= 0.08

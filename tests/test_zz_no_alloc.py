@@ -76,3 +76,23 @@ def test_static_forward_refuses_what_does_not_fit():
     with pytest.raises(b.TspError) as err:
         b.tsp_mlp_forward_static(H, F, D, x, x, x, x, x, 101)
     assert err.value.code == b.TSP_ERR_UNSUPPORTED_SHAPE
+
+
+def test_static_forward_without_flag_and_on_a_side_stream():
+    import torch
+
+    # a caller on a latency-critical path passes no flag (nothing makes the host wait) or a flag in pinned memory,
+    # and usually launches on a stream of its own
+    prob = DeviceProblem(256, 256, 768, 2, seed=13)
+    want = prob.forward()
+    side = torch.cuda.Stream()
+    pinned = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+    for flag in (None, ctypes.cast(pinned.data_ptr(), ctypes.POINTER(ctypes.c_int)).contents):
+        Y = torch.full((prob.S, prob.H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            b.tsp_mlp_forward_static(prob.H, prob.F, prob.D, prob.X, prob.Wg, prob.Wu, prob.Wd, Y, prob.S, flag, side)
+        side.synchronize()
+        assert bool((Y.view(torch.int16) == want.view(torch.int16)).all())
+    assert int(pinned[0]) == 0
+    assert b.tsp_mlp_last_cuda_error(None) == 0
