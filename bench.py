@@ -690,7 +690,9 @@ def run_rank_steps(args, wl):
     Y_p = torch.empty_like(X_p)
     plan = b.tsp_mlp_plan(H, F, D)
     ws = torch.empty(max(b.tsp_mlp_workspace_bytes_ring(plan, S_loc, b.TSP_WS_BACKWARD),
-                         b.tsp_mlp_workspace_bytes_ring_group(plan, S_loc, g)), dtype=torch.uint8, device="cuda")
+                         b.tsp_mlp_workspace_bytes_ring_group(plan, S_loc, g),
+                         b.tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, g) if train else 0),
+                     dtype=torch.uint8, device="cuda")
     b.tsp_mlp_set_workspace(plan, ws)
     if train:
         dY_p, dX_p = dev(host.dY), torch.empty_like(X_p)
@@ -700,7 +702,15 @@ def run_rank_steps(args, wl):
         for t0 in range(0, D, g):
             a, u, d = ring.unpack_shard(packed[t0], H, F_d)
             b.tsp_mlp_ring_steps(plan, X_p, a, u, d, packed.shape[1], min(g, D - t0), Y_p, S_loc, t0, D)
-        if train:
+        if train and g > 1:      # grouped backward: three kernels per group, the weight gradients shard by shard
+            for t0 in range(0, D, g):
+                n = min(g, D - t0)
+                a, u, d = ring.unpack_shard(packed[t0], H, F_d)
+                b.tsp_mlp_ring_steps_backward_dx(plan, X_p, a, u, d, packed.shape[1], n, dY_p, dX_p, S_loc, t0, D)
+                for i in range(n):
+                    ga, gu, gd = ring.unpack_shard(dW[t0 + i], H, F_d)
+                    b.tsp_mlp_ring_steps_backward_dw(plan, X_p, dY_p, ga, gu, gd, S_loc, i, n, 0, D)
+        elif train:
             for t in range(D):
                 a, u, d = ring.unpack_shard(packed[t], H, F_d)
                 ga, gu, gd = ring.unpack_shard(dW[t], H, F_d)
@@ -738,14 +748,15 @@ def run_rank_steps(args, wl):
     assert b.tsp_mlp_status(plan) == b.TSP_OK, "device-side wait timed out"
     ms = e0.elapsed_time(e1) / args.steps
     flops = (6.0 + (12.0 if train else 0.0)) * S_loc * H * F
-    launches = b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD) * ((D + g - 1) // g) + (4 * D if train else 0)
+    launches = b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD) * ((D + g - 1) // g) + (
+        (3 * ((D + g - 1) // g) + D if g > 1 else 4 * D) if train else 0)
     line = {
         "metric": METRIC, "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "pass": "forward+backward (G, U recomputed)" if train else "forward",
                    "mode": "rank-steps (one rank's tokens, all shards local, per-rank step entry points)",
-                   "S_loc": S_loc, "H": H, "F": F, "D": D, "ring_steps_per_launch_forward": g,
+                   "S_loc": S_loc, "H": H, "F": F, "D": D, "ring_steps_per_launch": g,
                    "launches": "replayed from a CUDA graph" if args.graph else "issued by the host every step",
                    "kernels_per_forward_call": b.tsp_mlp_kernels_per_call(plan, b.TSP_WS_FORWARD),
                    "us_per_ring_step": 1e3 * ms / D},
@@ -766,7 +777,7 @@ def main():
     ap.add_argument("--stored-activations", action="store_true",
                     help="training step through tsp_mlp_forward_save / tsp_mlp_backward_saved (no recomputation)")
     ap.add_argument("--steps-per-launch", type=int, default=1,
-                    help="--mode rank-steps: ring steps applied per launch pair in the forward pass")
+                    help="--mode rank-steps: ring steps applied per group of launches (forward, and backward except dW)")
     ap.add_argument("--mode", default="direct", choices=["direct", "staged", "ring", "rank-steps"],
                     help="staged: Algorithm 2 step by step with the shard transfer emulated on a side stream; "
                          "ring: D = N ranks on N GPUs, the shards travel between the GPUs; "

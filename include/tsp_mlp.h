@@ -323,6 +323,35 @@ tsp_status_t tsp_mlp_ring_step_backward_dw(tsp_mlp_plan_t* plan, const void* X_p
                                            void* cuda_stream);
 
 /*
+ * Backward pass of n consecutive ring steps t_first .. t_first + n - 1 of ONE rank per call (the counterpart of
+ * tsp_mlp_ring_steps; Sections 4.3.4 and 4.7 as for the single-step calls).  With few tokens per rank the GEMMs of one
+ * step leave most of the GPU idle, so a rank that already holds the next n shards (same packed layout and
+ * shard_stride as for tsp_mlp_ring_steps, in the order it meets them) runs
+ *   tsp_mlp_ring_steps_backward_dx: dA = dY_p [Wd_0 .. Wd_n-1]^T (fp32), the gate|up GEMM over the n shards with the
+ *     backward epilogue (A, dG, dU for all n shards, bf16, left in the workspace), and ONE dX GEMM whose K loop walks
+ *     the n shards in the order given; the fp32 sum of dX_p is carried across calls as by the single-step call (first
+ *     call t_first = 0, the call ending at D stores bf16 dX_p).  Three kernels.  dX_p differs from the step-by-step
+ *     result only in the grouping of fp32 partial sums.
+ *   tsp_mlp_ring_steps_backward_dw: the weight gradients of ONE shard of the group (shard_in_group = 0 .. n-1), from
+ *     the A, dG, dU columns the _dx call left: exactly tsp_mlp_ring_step_backward_dw's arithmetic (accumulate = 1 adds
+ *     to a travelling accumulator in the kernel's epilogue), so the weight gradients keep every bit of the
+ *     step-by-step result and the order of the sum over ranks, r = (k + t) mod D.  It is a call of its own because a
+ *     shard's accumulator arrives from the left neighbour only after that rank has added its share: the caller issues
+ *     the n calls one by one as the accumulators arrive, while nothing else of the group has to wait.  One kernel.
+ * Workspace: tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, n) for the largest n used (dXacc, then A, dG,
+ * dU [S_loc, n F/D] bf16 and dA fp32); not to be mixed with the single-step backward calls within one pass.
+ * Needs (F/D) % 256 == 0.  Errors as for tsp_mlp_ring_steps / tsp_mlp_ring_step_backward_dw.
+ */
+size_t tsp_mlp_workspace_bytes_ring_group_backward(const tsp_mlp_plan_t* plan, int64_t S_loc, int n_shards);
+tsp_status_t tsp_mlp_ring_steps_backward_dx(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_first,
+                                            const void* Wu_first, const void* Wd_first, int64_t shard_stride,
+                                            int n_shards, const void* dY_p, void* dX_p, int64_t S_loc, int t_first, int D,
+                                            void* cuda_stream);
+tsp_status_t tsp_mlp_ring_steps_backward_dw(tsp_mlp_plan_t* plan, const void* X_p, const void* dY_p, float* dWg_k,
+                                            float* dWu_k, float* dWd_k, int64_t S_loc, int shard_in_group, int n_shards,
+                                            int accumulate, int D, void* cuda_stream);
+
+/*
  * tsp_mlp_forward_static - the forward pass for callers that cannot obtain device memory at call time.
  * (The paper has no counterpart of this entry point; it exists for integration reasons only.)
  *

@@ -56,6 +56,11 @@ SIGNATURES = {
     "tsp_mlp_workspace_bytes_ring_group": (ctypes.c_size_t, [_P, ctypes.c_int64, ctypes.c_int]),
     "tsp_mlp_ring_steps": (ctypes.c_int, [_P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P, ctypes.c_int64,
                                           ctypes.c_int, ctypes.c_int, _P]),
+    "tsp_mlp_workspace_bytes_ring_group_backward": (ctypes.c_size_t, [_P, ctypes.c_int64, ctypes.c_int]),
+    "tsp_mlp_ring_steps_backward_dx": (ctypes.c_int, [_P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, _P, _P,
+                                                      ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
+    "tsp_mlp_ring_steps_backward_dw": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                                      ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_ring_step": (ctypes.c_int, [_P, _P, _P, _P, _P, _P, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P]),
     "tsp_mlp_forward_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, _P,
                                               ctypes.c_int64, ctypes.POINTER(ctypes.c_int), _P]),
@@ -279,6 +284,26 @@ def tsp_mlp_ring_step_backward_dw(plan, X_p, dY_p, dWg_k, dWu_k, dWd_k, S_loc: i
     _check(load_library().tsp_mlp_ring_step_backward_dw(plan, _ptr(X_p), _ptr(dY_p), _ptr(dWg_k), _ptr(dWu_k),
                                                         _ptr(dWd_k), S_loc, accumulate, D, _stream_handle(stream)),
            "tsp_mlp_ring_step_backward_dw", plan)
+
+
+def tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc: int, n_shards: int) -> int:
+    return int(load_library().tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, n_shards))
+
+
+def tsp_mlp_ring_steps_backward_dx(plan, X_p, Wg_first, Wu_first, Wd_first, shard_stride: int, n_shards: int, dY_p, dX_p,
+                                   S_loc: int, t_first: int, D: int, stream=None) -> None:
+    """Backward of n consecutive ring steps of one rank, all but the weight gradients (dA, A/dG/dU, carried dX sum)."""
+    _check(load_library().tsp_mlp_ring_steps_backward_dx(plan, _ptr(X_p), _ptr(Wg_first), _ptr(Wu_first), _ptr(Wd_first),
+                                                         shard_stride, n_shards, _ptr(dY_p), _ptr(dX_p), S_loc, t_first, D,
+                                                         _stream_handle(stream)), "tsp_mlp_ring_steps_backward_dx", plan)
+
+
+def tsp_mlp_ring_steps_backward_dw(plan, X_p, dY_p, dWg_k, dWu_k, dWd_k, S_loc: int, shard_in_group: int, n_shards: int,
+                                   accumulate: int, D: int, stream=None) -> None:
+    """Weight gradients of one shard of the group the preceding tsp_mlp_ring_steps_backward_dx call processed."""
+    _check(load_library().tsp_mlp_ring_steps_backward_dw(plan, _ptr(X_p), _ptr(dY_p), _ptr(dWg_k), _ptr(dWu_k),
+                                                         _ptr(dWd_k), S_loc, shard_in_group, n_shards, accumulate, D,
+                                                         _stream_handle(stream)), "tsp_mlp_ring_steps_backward_dw", plan)
 
 
 def tsp_mlp_forward_static(H: int, F: int, D: int, X, Wg, Wu, Wd, Y, S: int, timed_out=None, stream=None) -> None:

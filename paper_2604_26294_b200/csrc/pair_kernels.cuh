@@ -595,6 +595,8 @@ struct PairDaPolicyT {
         __nv_bfloat16* dU;           // [S, F]
         int S, H, F, D, S_loc;
         int m_tiles, tiles_per_rank, j_tiles, band;
+        int j_tiles_per_shard;       // 0: Wd is one [F, H] matrix; n > 0: the map's third coordinate is the shard, each
+                                     // shard holding n tiles of 256 rows (packed shard buffers of a ring-step group)
         int mt_base;                 // first token tile of this launch
         int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
@@ -602,7 +604,7 @@ struct PairDaPolicyT {
         unsigned long long timeout_ns;
     };
     struct Tile {
-        int mt, jt, row0, valid;
+        int mt, jt, row0, valid, wz, wrow;   // wz, wrow: shard and first row inside it of the tile's 256 rows of Wd
     };
     __device__ static __forceinline__ int outer(const Params&) { return 1; }
     __device__ static __forceinline__ int inner(const Params& p) { return p.H / kBK; }
@@ -623,12 +625,14 @@ struct PairDaPolicyT {
         o.mt = p.mt_base + band_start + rem % band_sz;
         int r;
         token_tile(o.mt, p.tiles_per_rank, p.S_loc, 256, r, o.row0, o.valid);
+        o.wz = p.j_tiles_per_shard ? o.jt / p.j_tiles_per_shard : 0;
+        o.wrow = (o.jt - o.wz * p.j_tiles_per_shard) * 256;
         return o;
     }
     __device__ static __forceinline__ void load(const Params& p, const Tile& tl, int, int kb, uint32_t cta, uint32_t sa,
                                                 uint32_t sb, uint32_t bar) {
         pair_load_kmajor(sa, &p.map_dy, bar, kb * kBK, tl.row0 + cta * 128, 0);
-        pair_load_kmajor(sb, &p.map_wd, bar, kb * kBK, tl.jt * 256 + cta * 128, 0);
+        pair_load_kmajor(sb, &p.map_wd, bar, kb * kBK, tl.wrow + cta * 128, tl.wz);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         const bool live = static_cast<int>(cta) * 128 + row < tl.valid;
@@ -817,6 +821,7 @@ struct PairDxPolicy {
         __nv_bfloat16* dX;
         float* dXacc;  // [S, H] fp32 partial sums carried between launches (one ring step per launch), or null
         int carry;     // 0: the launch covers all shards, dX stored directly; 1 first, 2 middle, 3 last step of a carried sum
+        int linear_shards;  // 1: ONE rank, the D shards of the maps are the ones it meets, in that order (ring-step group)
         int S, H, F, D, F_d, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;
@@ -830,6 +835,7 @@ struct PairDxPolicy {
     __device__ static __forceinline__ int outer(const Params& p) { return p.D; }
     __device__ static __forceinline__ int inner(const Params& p) { return 2 * (p.F_d / kBK); }
     __device__ static __forceinline__ int select(const Params& p, const Tile& tl, int t) {
+        if (p.linear_shards) return t;
         const int k = tl.r - t;
         return k < 0 ? k + p.D : k;
     }
@@ -905,6 +911,8 @@ struct PairDwPolicy {
         int n_group;   // hidden blocks per group: their columns of X / dY stay in L2 while the [S,F] operand streams
         int k_linear;  // 0, or ceil(S / 64) when the token contraction runs in ascending order (ragged ranks)
         int accumulate;  // 0: dW overwritten; 1: the tile's sum is added to what dW holds (partial sums of other ranks)
+        long long out_shard_stride;  // elements between consecutive shards' matrices in each of dWd, dWg, dWu (H * F/D when
+                                     // the outputs are the contiguous [D][..][..] arrays)
         int wide_tiles;
         int tile_base;   // first entry of the tile list this launch covers (a long list is cut into several launches)
         int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
@@ -969,7 +977,7 @@ struct PairDwPolicy {
             tmem_ld_wait();
             const int h0 = h_base + c * 32;
             if (tl.which == 0) {
-                float* dst = p.dWd + static_cast<size_t>(j) * p.H + h0;
+                float* dst = p.dWd + static_cast<size_t>(tl.k) * p.out_shard_stride + static_cast<size_t>(j - tl.k * F_d) * p.H + h0;
                 if (p.accumulate) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
@@ -985,7 +993,7 @@ struct PairDwPolicy {
                     st_global_256(dst + q * 8, v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4], v[8 * q + 5],
                                   v[8 * q + 6], v[8 * q + 7]);
             } else {
-                float* base = (tl.which == 1 ? p.dWg : p.dWu) + static_cast<size_t>(tl.k) * p.H * F_d + (j - tl.k * F_d);
+                float* base = (tl.which == 1 ? p.dWg : p.dWu) + static_cast<size_t>(tl.k) * p.out_shard_stride + (j - tl.k * F_d);
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     float* dst = base + static_cast<size_t>(h0 + i) * F_d;

@@ -123,6 +123,19 @@ bool encode_sharded(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, ui
                       box0, box1);
 }
 
+// [n][rows][cols] bf16 with an arbitrary distance between consecutive matrices (packed shard buffers in a row).
+bool encode_strided(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, uint64_t n, uint64_t rows, uint64_t cols,
+                    uint64_t stride_bytes, uint32_t box0, uint32_t box1) {
+    return encode_map(plan, map, base, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, cols, rows, n, cols * 2, stride_bytes, box0, box1);
+}
+
+// [rows, cols] bf16 block of a wider row-major matrix (`pitch` elements per row), viewed as (cols, rows, 1).
+bool encode_block(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch,
+                  uint32_t box0, uint32_t box1) {
+    return encode_map(plan, map, base, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, cols, rows, 1, pitch * 2, rows * pitch * 2, box0,
+                      box1);
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }  // outputs: 256-bit stores
 
@@ -562,19 +575,21 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
 
 tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
                                 const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream,
-                                int accumulate = 0, bool linear = false) {
+                                int accumulate = 0, bool linear = false, int64_t pitch = 0) {
     const int H = plan->H, F = plan->F, D = plan->D;
+    if (pitch <= 0) pitch = F;   // A, dG, dU may be column blocks of wider matrices (the scratch of a ring-step group)
     tsp::PairDwPolicy::Params p;
     std::memset(&p, 0, sizeof(p));
-    if (!encode_matrix(plan, &p.map_a, A, S, F, 64, 64)) return TSP_ERR_CUDA;
-    if (!encode_matrix(plan, &p.map_dg, dG, S, F, 64, 64)) return TSP_ERR_CUDA;
-    if (!encode_matrix(plan, &p.map_du, dU, S, F, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_block(plan, &p.map_a, A, S, F, pitch, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_block(plan, &p.map_dg, dG, S, F, pitch, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_block(plan, &p.map_du, dU, S, F, pitch, 64, 64)) return TSP_ERR_CUDA;
     if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 64)) return TSP_ERR_CUDA;
     if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 64)) return TSP_ERR_CUDA;
     p.dWd = dWd; p.dWg = dWg; p.dWu = dWu;
     p.accumulate = accumulate;
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.F_d = F / D;
+    p.out_shard_stride = static_cast<long long>(H) * p.F_d;
     p.S_loc = static_cast<int>(S / D);
     p.k_linear = (linear || p.S_loc % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
     p.j_tiles = F / 256;
@@ -639,17 +654,19 @@ inline const void* row_offset(const void* base, int64_t row, int64_t cols) {
 // All weight gradients of the MLP for S tokens; `accumulate`: add to what dW* hold instead of overwriting.
 tsp_status_t launch_dw_all(tsp_mlp_plan_t* plan, const void* X, const void* dY, const void* A, const void* dG,
                            const void* dU, float* dWg, float* dWu, float* dWd, int64_t S, cudaStream_t stream,
-                           int accumulate) {
+                           int accumulate, int64_t pitch = 0) {
     const int H = plan->H, F = plan->F;
     const bool pairs = pairs_for_dw(plan);
+    if (pitch <= 0) pitch = F;
+    if (pitch != F && !pairs) return TSP_ERR_UNSUPPORTED_SHAPE;
     return for_token_chunks(S, [&](int64_t c0, int64_t len, bool chunked) {
         const int acc = (accumulate || c0 > 0) ? 1 : 0;
         const void* x = row_offset(X, c0, H);
         const void* dy = row_offset(dY, c0, H);
-        const void* a = row_offset(A, c0, F);
-        const void* dg = row_offset(dG, c0, F);
-        const void* du = row_offset(dU, c0, F);
-        return pairs ? launch_bwd_dw_pair(plan, x, dy, a, dg, du, dWg, dWu, dWd, len, stream, acc, chunked)
+        const void* a = row_offset(A, c0, pitch);
+        const void* dg = row_offset(dG, c0, pitch);
+        const void* du = row_offset(dU, c0, pitch);
+        return pairs ? launch_bwd_dw_pair(plan, x, dy, a, dg, du, dWg, dWu, dWd, len, stream, acc, chunked, pitch)
                      : launch_bwd_dw(plan, x, dy, a, dg, du, dWg, dWu, dWd, len, stream, acc, chunked);
     });
 }
@@ -733,12 +750,6 @@ tsp_status_t launch_forward_step(tsp_mlp_plan_t* plan, const void* X, const void
     return launch_step_down(plan, cur_d, A_step, Yacc, Y, S, n_ranks, mode, cs);
 }
 
-// [n][rows][cols] bf16 with an arbitrary distance between consecutive matrices (packed shard buffers in a row).
-bool encode_strided(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, uint64_t n, uint64_t rows, uint64_t cols,
-                    uint64_t stride_bytes, uint32_t box0, uint32_t box1) {
-    return encode_map(plan, map, base, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, cols, rows, n, cols * 2, stride_bytes, box0, box1);
-}
-
 // n consecutive ring steps of ONE rank in two launches: gate|up of the rank's tokens against the n shards (A becomes
 // [S, n * F/D]), then one down projection whose K loop runs over the n shards in the order given.
 tsp_status_t launch_steps_group(tsp_mlp_plan_t* plan, const void* X, const void* Wg0, const void* Wu0, const void* Wd0,
@@ -788,6 +799,101 @@ tsp_status_t launch_steps_group(tsp_mlp_plan_t* plan, const void* X, const void*
         fill_common(plan, p, p.m_tiles * p.n_blocks);
         return launch_pair<tsp::PairDownStagedPolicy>(plan, p, cs, kDynDown);
     }
+}
+
+// Backward of n consecutive ring steps of ONE rank, everything except the weight gradients: dA = dY_p [Wd_0 .. Wd_n-1]^T
+// (fp32, [S, n F/D]); the gate|up GEMM over the n shards with the backward epilogue (A, dG, dU, each [S, n F/D]); the
+// dX GEMM whose K loop walks the n shards in the order given and carries the fp32 sum from call to call.
+tsp_status_t launch_steps_group_backward(tsp_mlp_plan_t* plan, const void* X, const void* Wg0, const void* Wu0,
+                                         const void* Wd0, size_t stride_bytes, int n, const void* dY, void* A, void* dG,
+                                         void* dU, float* dA, float* dXacc, void* dX, int64_t S, int carry,
+                                         Profiler& prof, cudaStream_t cs) {
+    const int H = plan->H, F_d = plan->F / plan->D;
+    const int m_tiles = static_cast<int>((S + 255) / 256);
+    {
+        using Policy = tsp::PairDaPolicyT<false>;
+        Policy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(plan, &p.map_dy, dY, S, H, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_strided(plan, &p.map_wd, Wd0, n, F_d, H, stride_bytes, 64, 128)) return TSP_ERR_CUDA;
+        p.dA = dA;
+        p.S = static_cast<int>(S); p.H = H; p.F = n * F_d; p.D = 1;
+        p.S_loc = static_cast<int>(S);
+        p.tiles_per_rank = m_tiles;
+        p.m_tiles = m_tiles;
+        p.j_tiles = n * F_d / 256;
+        p.j_tiles_per_shard = F_d / 256;
+        p.band = gate_band(plan, m_tiles);
+        tsp_status_t st = for_tile_chunks(m_tiles, plan->chunk_bands * p.band, false, [&](int first, int count) {
+            p.mt_base = first;
+            p.m_tiles = count;
+            fill_common(plan, p, count * p.j_tiles);
+            return launch_pair<Policy>(plan, p, cs);
+        });
+        if (st != TSP_OK) return st;
+        prof.mark();
+    }
+    {
+        using Policy = tsp::PairGateUpPolicyT<1>;
+        Policy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_strided(plan, &p.map_wg, Wg0, n, H, F_d, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
+        if (!encode_strided(plan, &p.map_wu, Wu0, n, H, F_d, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
+        p.A = static_cast<__nv_bfloat16*>(A);
+        p.dA = dA;
+        p.dG = static_cast<__nv_bfloat16*>(dG);
+        p.dU = static_cast<__nv_bfloat16*>(dU);
+        p.S = static_cast<int>(S); p.H = H; p.F = n * F_d; p.D = n; p.F_d = F_d;
+        p.S_loc = static_cast<int>(S);
+        p.tiles_per_rank = m_tiles;
+        p.m_tiles = m_tiles;
+        p.jl_blocks = F_d / 128;
+        p.band = gate_band(plan, m_tiles);
+        p.shared_order = 1;
+        p.act = plan->act;
+        tsp_status_t st = for_tile_chunks(m_tiles, plan->chunk_bands * p.band, false, [&](int first, int count) {
+            p.mt_base = first;
+            p.m_tiles = count;
+            fill_common(plan, p, count * n * p.jl_blocks);
+            return launch_pair<Policy>(plan, p, cs);
+        });
+        if (st != TSP_OK) return st;
+        prof.mark();
+    }
+    {
+        tsp::PairDxPolicy::Params p;
+        std::memset(&p, 0, sizeof(p));
+        const uint64_t width = static_cast<uint64_t>(n) * F_d;
+        if (!encode_matrix(plan, &p.map_dg, dG, S, width, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_matrix(plan, &p.map_du, dU, S, width, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_strided(plan, &p.map_wg, Wg0, n, H, F_d, stride_bytes, 64, 128)) return TSP_ERR_CUDA;
+        if (!encode_strided(plan, &p.map_wu, Wu0, n, H, F_d, stride_bytes, 64, 128)) return TSP_ERR_CUDA;
+        p.dX = static_cast<__nv_bfloat16*>(dX);
+        p.dXacc = dXacc;
+        p.carry = carry;
+        p.linear_shards = 1;
+        p.S = static_cast<int>(S); p.H = H; p.F = n * F_d; p.D = n; p.F_d = F_d;
+        p.S_loc = static_cast<int>(S);
+        p.tiles_per_rank = m_tiles;
+        p.n_blocks = H / 256;
+        const int group = plan->dx_group > 0 ? plan->dx_group : 8;
+        tsp_status_t st = for_tile_chunks(m_tiles, plan->chunk_tiles, true, [&](int first, int count) {
+            p.mt_base = first;
+            p.m_tiles = count;
+            p.group = count < group ? count : group;
+            p.wide_tiles = mixed_wide_tiles(plan, 2, p.n_blocks, count * p.n_blocks, 2 * n * F_d / 64);
+            if (p.wide_tiles > 0) {
+                fill_common(plan, p, count * p.n_blocks - p.wide_tiles);
+                return launch_pair_wide<tsp::PairDxPolicy>(plan, p, cs, kDynDx);
+            }
+            fill_common(plan, p, count * p.n_blocks);
+            return launch_pair<tsp::PairDxPolicy>(plan, p, cs, kDynDx);
+        });
+        if (st != TSP_OK) return st;
+        prof.mark();
+    }
+    return TSP_OK;
 }
 
 // The same n ring steps of one rank as ONE launch (PairFusedStepPolicy): gate|up tiles, then down-projection tiles
@@ -1419,6 +1525,83 @@ tsp_status_t tsp_mlp_ring_step_backward_dw(tsp_mlp_plan_t* plan, const void* X_p
     OneShardView view(plan);
     tsp_status_t st = launch_dw_all(plan, X_p, dY_p, base, base + one, base + 2 * one, dWg_k, dWu_k, dWd_k, S_loc, cs,
                                     accumulate);
+    prof.mark();
+    return st;
+}
+
+size_t tsp_mlp_workspace_bytes_ring_group_backward(const tsp_mlp_plan_t* plan, int64_t S_loc, int n_shards) {
+    if (!plan || S_loc <= 0 || n_shards < 1 || n_shards > plan->D) return 0;
+    const size_t one = align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2 * n_shards, 256);
+    return align_up(static_cast<size_t>(S_loc) * plan->H * 4, 256) + 5 * one;   // dXacc | A | dG | dU | dA (fp32)
+}
+
+namespace {
+// layout of the grouped backward workspace; the accumulator comes first so that its place does not depend on n
+struct GroupBackwardWs {
+    float* dXacc;
+    uint8_t *A, *dG, *dU;
+    float* dA;
+};
+GroupBackwardWs group_backward_ws(const tsp_mlp_plan_t* plan, int64_t S_loc, int n) {
+    const size_t one = align_up(static_cast<size_t>(S_loc) * (plan->F / plan->D) * 2 * n, 256);
+    uint8_t* base = static_cast<uint8_t*>(plan->workspace);
+    GroupBackwardWs w;
+    w.dXacc = reinterpret_cast<float*>(base);
+    base += align_up(static_cast<size_t>(S_loc) * plan->H * 4, 256);
+    w.A = base;
+    w.dG = base + one;
+    w.dU = base + 2 * one;
+    w.dA = reinterpret_cast<float*>(base + 3 * one);
+    return w;
+}
+}  // namespace
+
+tsp_status_t tsp_mlp_ring_steps_backward_dx(tsp_mlp_plan_t* plan, const void* X_p, const void* Wg_first,
+                                            const void* Wu_first, const void* Wd_first, int64_t shard_stride,
+                                            int n_shards, const void* dY_p, void* dX_p, int64_t S_loc, int t_first, int D,
+                                            void* cuda_stream) {
+    if (!plan || D != plan->D || n_shards < 1 || t_first < 0 || t_first + n_shards > D) return TSP_ERR_INVALID_ARG;
+    if (S_loc < 1 || S_loc > (1ll << 24) || (plan->F / plan->D) % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X_p || !Wg_first || !Wu_first || !Wd_first || !dY_p || !dX_p) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X_p) || !aligned16(Wg_first) || !aligned16(Wu_first) || !aligned16(Wd_first) || !aligned16(dY_p) ||
+        !aligned32(dX_p))
+        return TSP_ERR_INVALID_ARG;
+    const int64_t shard_elems = static_cast<int64_t>(plan->H) * (plan->F / plan->D);
+    if (n_shards > 1 && (shard_stride < shard_elems || shard_stride % 8 != 0)) return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, n_shards))
+        return TSP_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    const GroupBackwardWs w = group_backward_ws(plan, S_loc, n_shards);
+    const bool first = t_first == 0, last = t_first + n_shards == D;
+    const int carry = first && last ? 0 : (first ? 1 : (last ? 3 : 2));
+    const size_t stride_bytes = n_shards > 1 ? static_cast<size_t>(shard_stride) * 2 : static_cast<size_t>(shard_elems) * 2;
+    plan->launch_count = 0;
+    Profiler prof(plan, cs);
+    tsp_status_t st = launch_steps_group_backward(plan, X_p, Wg_first, Wu_first, Wd_first, stride_bytes, n_shards, dY_p,
+                                                  w.A, w.dG, w.dU, w.dA, w.dXacc, dX_p, S_loc, carry, prof, cs);
+    plan->last_backward_kernels = plan->launch_count;
+    return st;
+}
+
+tsp_status_t tsp_mlp_ring_steps_backward_dw(tsp_mlp_plan_t* plan, const void* X_p, const void* dY_p, float* dWg_k,
+                                            float* dWu_k, float* dWd_k, int64_t S_loc, int shard_in_group, int n_shards,
+                                            int accumulate, int D, void* cuda_stream) {
+    if (!plan || D != plan->D || (accumulate != 0 && accumulate != 1)) return TSP_ERR_INVALID_ARG;
+    if (n_shards < 1 || n_shards > D || shard_in_group < 0 || shard_in_group >= n_shards) return TSP_ERR_INVALID_ARG;
+    if (S_loc < 1 || S_loc > (1ll << 24) || (plan->F / plan->D) % 256 != 0) return TSP_ERR_UNSUPPORTED_SHAPE;
+    if (!X_p || !dY_p || !dWg_k || !dWu_k || !dWd_k) return TSP_ERR_INVALID_ARG;
+    if (!aligned16(X_p) || !aligned16(dY_p) || !aligned32(dWg_k) || !aligned32(dWu_k) || !aligned32(dWd_k))
+        return TSP_ERR_INVALID_ARG;
+    if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, n_shards))
+        return TSP_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    const GroupBackwardWs w = group_backward_ws(plan, S_loc, n_shards);
+    const int F_d = plan->F / plan->D;
+    const size_t col = static_cast<size_t>(shard_in_group) * F_d * 2;   // this shard's column block of A, dG, dU
+    Profiler prof(plan, cs);
+    OneShardView view(plan);
+    tsp_status_t st = launch_dw_all(plan, X_p, dY_p, w.A + col, w.dG + col, w.dU + col, dWg_k, dWu_k, dWd_k, S_loc, cs,
+                                    accumulate, static_cast<int64_t>(n_shards) * F_d);
     prof.mark();
     return st;
 }

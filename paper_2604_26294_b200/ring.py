@@ -17,6 +17,7 @@ to the CUDA library.
 """
 from __future__ import annotations
 
+import contextlib
 from typing import Callable, Sequence
 
 import torch
@@ -33,12 +34,99 @@ def shard_at_step(rank: int, t: int, D: int) -> int:
     return (rank - t) % D
 
 
-def _exchange(send: torch.Tensor, recv: torch.Tensor, rank: int, D: int, group=None):
-    dst, src = ring_neighbours(rank, D)
-    if group is not None:
-        dst, src = dist.get_global_rank(group, dst), dist.get_global_rank(group, src)
-    ops = [dist.P2POp(dist.isend, send, dst, group), dist.P2POp(dist.irecv, recv, src, group)]
-    return dist.batch_isend_irecv(ops)
+class DistTransport:
+    """Ring transfers over torch.distributed (NCCL on GPUs, gloo on CPU): exchange() posts "send to p+1, receive from
+    p-1" and returns requests with a wait() method."""
+
+    def __init__(self, rank: int, D: int, group=None):
+        dst, src = ring_neighbours(rank, D)
+        if group is not None:
+            dst, src = dist.get_global_rank(group, dst), dist.get_global_rank(group, src)
+        self.dst, self.src, self.group = dst, src, group
+
+    def exchange(self, send: torch.Tensor, recv: torch.Tensor):
+        ops = [dist.P2POp(dist.isend, send, self.dst, self.group), dist.P2POp(dist.irecv, recv, self.src, self.group)]
+        return dist.batch_isend_irecv(ops)
+
+
+class HostOrder:
+    """Ordering between transfers and compute when request.wait() blocks the host (gloo, CPU tensors): program order
+    is enough, nothing to do."""
+
+    def begin(self) -> None:                      # start of a pass, after the own shard has been copied into its row
+        pass
+
+    def end(self) -> None:                        # end of a pass, after the last transfer has been waited for
+        pass
+
+    def transport(self):
+        return contextlib.nullcontext()
+
+    def shard_arrived(self, t: int) -> None:      # called in the transport context right after the wait for shard t
+        pass
+
+    def before_compute(self, steps) -> None:      # called before the compute call that reads the shards of `steps`
+        pass
+
+    def after_compute(self, steps) -> None:       # called after that compute call has been issued
+        pass
+
+    def before_overwrite(self, t: int) -> None:   # called in the transport context before the buffer of step t is reused
+        pass
+
+
+class StreamOrder(HostOrder):
+    """The same ordering on a GPU, where compute and transfers are asynchronous: every transfer is posted, and every
+    request waited for, with a dedicated transport stream current (request.wait() of NCCL makes the CURRENT stream wait,
+    so the compute stream is never held up by a transfer it does not need yet); the dependencies are explicit events:
+      shard t has arrived          -> recorded on the transport stream, the compute stream waits for it before the
+                                      compute call that reads shard t;
+      the steps of a call are done -> recorded on the compute stream, the transport stream waits for it before a
+                                      receive overwrites a buffer those steps read.
+    Nothing here relies on how the transport orders consecutive transfers among themselves.
+    """
+
+    def __init__(self, device=None):
+        self.compute = torch.cuda.current_stream(device)
+        self.stream = torch.cuda.Stream(device=device)
+        self.arrived: dict[int, torch.cuda.Event] = {}
+        self.computed: dict[int, torch.cuda.Event] = {}
+
+    def begin(self) -> None:
+        """Start of a pass: transfers may read buffers the compute stream has just written (the own shard)."""
+        self.compute = torch.cuda.current_stream()
+        self.arrived.clear()
+        self.computed.clear()
+        self.stream.wait_stream(self.compute)
+
+    def end(self) -> None:
+        """End of a pass: later work on the compute stream comes after the last transfers."""
+        self.compute.wait_stream(self.stream)
+
+    def transport(self):
+        return torch.cuda.stream(self.stream)
+
+    def shard_arrived(self, t: int) -> None:
+        ev = torch.cuda.Event()
+        ev.record(self.stream)
+        self.arrived[t] = ev
+
+    def before_compute(self, steps) -> None:
+        for t in steps:
+            ev = self.arrived.pop(t, None)
+            if ev is not None:
+                self.compute.wait_event(ev)
+
+    def after_compute(self, steps) -> None:
+        ev = torch.cuda.Event()
+        ev.record(self.compute)
+        for t in steps:
+            self.computed[t] = ev
+
+    def before_overwrite(self, t: int) -> None:
+        ev = self.computed.pop(t, None)
+        if ev is not None:
+            self.stream.wait_event(ev)
 
 
 def _wait(reqs) -> None:
@@ -48,7 +136,7 @@ def _wait(reqs) -> None:
 
 def ring_forward(compute: Callable[[int, int, torch.Tensor], None], own_shard: torch.Tensor,
                  recv_bufs: Sequence[torch.Tensor], rank: int, D: int, group=None,
-                 before_exchange: Callable[[int], None] | None = None) -> None:
+                 before_exchange: Callable[[int], None] | None = None, transport=None) -> None:
     """The loop of Algorithm 2 on one rank.
 
     compute(t, k, shard) runs ring step t with the packed shard k = (rank - t) mod D it is handed;
@@ -60,13 +148,14 @@ def ring_forward(compute: Callable[[int, int, torch.Tensor], None], own_shard: t
     """
     n = len(recv_bufs)
     cur = own_shard
+    transport = transport or DistTransport(rank, D, group)
     for t in range(D):
         reqs = []
         if t < D - 1:
             if before_exchange is not None:
                 before_exchange(t)
             nxt = recv_bufs[t % n]
-            reqs = _exchange(cur, nxt, rank, D, group)
+            reqs = transport.exchange(cur, nxt)
         compute(t, shard_at_step(rank, t, D), cur)
         _wait(reqs)                      # Wait(): the next shard has arrived, the current one has left
         if t < D - 1:
@@ -74,51 +163,81 @@ def ring_forward(compute: Callable[[int, int, torch.Tensor], None], own_shard: t
 
 
 def ring_forward_grouped(compute: Callable[[int, int, int], None], own_shard: torch.Tensor, slots: torch.Tensor,
-                         rank: int, D: int, g: int, group=None, ordered_transport: bool = False) -> None:
+                         rank: int, D: int, g: int, group=None, transport=None, order: HostOrder | None = None) -> None:
     """Algorithm 2 with g ring steps per compute call.
 
     With few tokens per rank one ring step does not fill a GPU, so a rank lets the transfers run ahead and applies
     g shards at a time.  slots [2g, n] is a ring of packed-shard buffers: the shard of step t lives in row t mod 2g,
     so the g shards of a group are consecutive rows (what `tsp_mlp_ring_steps` wants).  The rank's own shard is
     copied into row 0.  Every rank still forwards each shard it receives to p+1 exactly once: transfer t sends row
-    (t-1) mod 2g and receives row t mod 2g.  Before group j computes, the transfers for groups j and j+1 are posted,
-    so the next group's shards arrive while this one computes.
+    (t-1) mod 2g and receives row t mod 2g, and is posted only after the receive of row (t-1) mod 2g has been waited
+    for.  Before group j computes, the transfers for groups j and j+1 are posted, so the next group's shards arrive
+    while this one computes.
     compute(t_first, n_steps, first_row) applies steps t_first .. t_first + n_steps - 1, whose shards are rows
     first_row .. first_row + n_steps - 1.
-    ordered_transport: True when consecutive transfers are executed in posting order (NCCL: one stream), so that
-    a received shard can be forwarded without waiting for it on the host; False (gloo) waits before forwarding.
+    transport: object with exchange(send, recv) -> requests (default: torch.distributed send / receive to the ring
+    neighbours).  order: HostOrder (default; waits block the host) or StreamOrder (GPU: waits are stream-level, on a
+    dedicated transport stream, with explicit events towards the compute stream).
     """
-    n_slots = slots.shape[0]
-    assert n_slots >= 2 * g and g >= 1
-    slots[0].copy_(own_shard)
-    reqs: dict[int, list] = {}
-    posted = 0                                        # transfers 1 .. posted have been posted
-
-    def post_up_to(t_last: int) -> None:
-        nonlocal posted
-        while posted < min(t_last, D - 1):
-            t = posted + 1                            # delivers the shard of step t
-            if not ordered_transport and t - 1 in reqs:
-                _wait(reqs[t - 1])                    # the shard about to be forwarded has arrived
-                reqs[t - 1] = []                      # (a request is waited for once only: gloo blocks on a second wait)
-            reqs[t] = _exchange(slots[(t - 1) % n_slots], slots[t % n_slots], rank, D, group)
-            posted = t
-
+    pipe = _ShardPipeline(own_shard, slots, rank, D, g, transport or DistTransport(rank, D, group), order or HostOrder())
     for t0 in range(0, D, g):
         n = min(g, D - t0)
-        post_up_to(t0 + n - 1 + g)                    # this group's shards and the next group's
+        pipe.fetch_group(t0, n)
+        compute(t0, n, t0 % pipe.n_slots)
+        pipe.group_issued(t0, n)
+    pipe.finish()
+
+
+class _ShardPipeline:
+    """The weight shards of a rank running ahead of its compute through a ring of 2g packed buffers (see
+    ring_forward_grouped): transfer t sends row (t-1) mod 2g to p+1 and receives the shard of step t into row t mod 2g."""
+
+    def __init__(self, own_shard, slots, rank, D, g, transport, order):
+        self.slots, self.rank, self.D, self.g = slots, rank, D, g
+        self.transport, self.order = transport, order
+        self.n_slots = slots.shape[0]
+        assert self.n_slots >= 2 * g and g >= 1
+        slots[0].copy_(own_shard)
+        order.begin()
+        self.reqs: dict[int, list] = {}               # transfer t -> its requests, until they have been waited for
+        self.posted = 0                               # transfers 1 .. posted have been posted
+
+    def _arrive(self, t: int) -> None:
+        """Wait (once) for transfer t: shard t is in its row, and row (t-1) has been sent on."""
+        if t in self.reqs:
+            with self.order.transport():
+                _wait(self.reqs.pop(t))
+                self.order.shard_arrived(t)
+
+    def _post_up_to(self, t_last: int) -> None:
+        while self.posted < min(t_last, self.D - 1):
+            t = self.posted + 1                       # delivers the shard of step t
+            self._arrive(t - 1)                       # the shard about to be forwarded has arrived
+            with self.order.transport():
+                self.order.before_overwrite(t - self.n_slots)   # the steps that read row t mod 2g before are done
+                self.reqs[t] = self.transport.exchange(self.slots[(t - 1) % self.n_slots], self.slots[t % self.n_slots])
+            self.posted = t
+
+    def fetch_group(self, t0: int, n: int) -> None:
+        """Post the transfers of this group and the next, then wait for this group's shards."""
+        self._post_up_to(t0 + n - 1 + self.g)
         for t in range(t0, t0 + n):
-            if t in reqs:
-                _wait(reqs.pop(t))
-        compute(t0, n, t0 % n_slots)
-    for r in reqs.values():                           # sends of the last transfers
-        _wait(r)
+            self._arrive(t)
+        self.order.before_compute(range(t0, t0 + n))
+
+    def group_issued(self, t0: int, n: int) -> None:
+        self.order.after_compute(range(t0, t0 + n))
+
+    def finish(self) -> None:
+        for t in sorted(self.reqs):                   # sends of the last transfers
+            self._arrive(t)
+        self.order.end()
 
 
 def ring_backward(compute_dx: Callable[[int, int, torch.Tensor], None],
                   compute_dw: Callable[[int, int, torch.Tensor, bool], None], own_shard: torch.Tensor,
                   recv_bufs: Sequence[torch.Tensor], dw_bufs: Sequence[torch.Tensor], rank: int, D: int,
-                  group=None) -> torch.Tensor:
+                  group=None, transport=None) -> torch.Tensor:
     """Backward ring on one rank; returns the buffer holding the summed gradient of this rank's OWN shard.
 
     compute_dx(t, k, shard): everything of step t that does not touch the weight-gradient accumulator.
@@ -128,21 +247,58 @@ def ring_backward(compute_dx: Callable[[int, int, torch.Tensor], None],
     """
     cur = own_shard
     acc_reqs = []
+    transport = transport or DistTransport(rank, D, group)
     for t in range(D):
         reqs = []
         if t < D - 1:
             nxt = recv_bufs[t & 1]
-            reqs = _exchange(cur, nxt, rank, D, group)
+            reqs = transport.exchange(cur, nxt)
         k = shard_at_step(rank, t, D)
         compute_dx(t, k, cur)
         _wait(acc_reqs)                  # the accumulator of shard k has arrived from p-1 (nothing to wait for at t = 0)
         acc = dw_bufs[t & 1]
         compute_dw(t, k, acc, t > 0)
         if D > 1:                        # pass it on; the hop after the last step delivers it to the owner
-            acc_reqs = _exchange(acc, dw_bufs[(t + 1) & 1], rank, D, group)
+            acc_reqs = transport.exchange(acc, dw_bufs[(t + 1) & 1])
         _wait(reqs)
         if t < D - 1:
             cur = nxt
+    _wait(acc_reqs)
+    return dw_bufs[D & 1] if D > 1 else dw_bufs[0]
+
+
+def ring_backward_grouped(compute_group_dx: Callable[[int, int, int], None],
+                          compute_dw: Callable[[int, int, int, torch.Tensor, bool], None], own_shard: torch.Tensor,
+                          slots: torch.Tensor, dw_bufs: Sequence[torch.Tensor], rank: int, D: int, g: int, group=None,
+                          transport=None, order: HostOrder | None = None) -> torch.Tensor:
+    """Backward ring with g ring steps per compute call; returns the buffer holding the gradient of the rank's own shard.
+
+    The weights run ahead exactly as in ring_forward_grouped (slots [2g, n]).  Per group of steps t_first .. t_first + n - 1
+    compute_group_dx(t_first, n, first_row) does everything that does not touch a weight-gradient accumulator (dA, the
+    recomputed gate|up GEMM with its backward epilogue for all n shards, the carried dX sum).  The accumulators keep
+    travelling one shard at a time, because the accumulator of step t's shard leaves the left neighbour only after that
+    rank has added its share: for every step of the group, in order, the rank waits for the accumulator, lets
+    compute_dw(t, i, n, acc, accumulate) add the contribution of shard i of the group (at t = 0: write it), and passes
+    it on.  The sum over ranks therefore runs in the order the shard meets them, r = (k + t) mod D, as in ring_backward,
+    and only the kernels that do not depend on a neighbour's result are grouped.  The accumulator transfers are posted
+    and waited for with the compute stream current: each depends on the kernel that has just written the accumulator.
+    """
+    transport = transport or DistTransport(rank, D, group)
+    pipe = _ShardPipeline(own_shard, slots, rank, D, g, transport, order or HostOrder())
+    acc_reqs = []
+    for t0 in range(0, D, g):
+        n = min(g, D - t0)
+        pipe.fetch_group(t0, n)
+        compute_group_dx(t0, n, t0 % pipe.n_slots)
+        pipe.group_issued(t0, n)
+        for i in range(n):
+            t = t0 + i
+            _wait(acc_reqs)              # the accumulator of this step's shard has arrived from p-1 (nothing at t = 0)
+            acc = dw_bufs[t & 1]
+            compute_dw(t, i, n, acc, t > 0)
+            if D > 1:                    # pass it on; the hop after the last step delivers it to the owner
+                acc_reqs = transport.exchange(acc, dw_bufs[(t + 1) & 1])
+    pipe.finish()
     _wait(acc_reqs)
     return dw_bufs[D & 1] if D > 1 else dw_bufs[0]
 
@@ -182,7 +338,8 @@ class TspRingMlp:
             steps_per_launch = 4 if S_loc <= 2048 else 2
         self.g = max(1, min(steps_per_launch, D))
         nbytes = max(b.tsp_mlp_workspace_bytes_ring(self.plan, S_loc, b.TSP_WS_BACKWARD if training else b.TSP_WS_FORWARD),
-                     b.tsp_mlp_workspace_bytes_ring_group(self.plan, S_loc, self.g))
+                     b.tsp_mlp_workspace_bytes_ring_group(self.plan, S_loc, self.g),
+                     b.tsp_mlp_workspace_bytes_ring_group_backward(self.plan, S_loc, self.g) if training else 0)
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
         b.tsp_mlp_set_workspace(self.plan, self.workspace)
         n = 3 * H * self.F_d
@@ -192,6 +349,7 @@ class TspRingMlp:
         self.dw_bufs = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(2 if D > 1 else 1)] if training else []
         self.slots = torch.empty(2 * self.g, n, dtype=torch.bfloat16, device=dev) if (D > 1 and self.g > 1) else None
         self.down_stream = torch.cuda.Stream(device=dev)
+        self.order = StreamOrder(dev)                 # transfers of the grouped schedules: own stream, explicit events
         self._gate_done = [torch.cuda.Event() for _ in range(D)]
         self._down_done = [torch.cuda.Event() for _ in range(D)]
 
@@ -219,7 +377,7 @@ class TspRingMlp:
                 self.b.tsp_mlp_ring_steps(self.plan, X_p, Wg, Wu, Wd, n, n_steps, Y_p, self.S_loc, t_first, self.D, main)
 
             ring_forward_grouped(compute_group, shard, self.slots, self.rank, self.D, self.g, self.group,
-                                 ordered_transport=True)
+                                 order=self.order)
             return Y_p
         if self.S_loc > self.TWO_STREAM_MAX_TOKENS:   # a step fills the GPU by itself: one stream, no event traffic
             def compute_one_stream(t, k, buf):
@@ -254,6 +412,23 @@ class TspRingMlp:
             raise RuntimeError("TspRingMlp was created with training=False")
         if dX_p is None:
             dX_p = torch.empty_like(X_p)
+
+        if self.slots is not None:                    # g ring steps per launch group; accumulators still one by one
+            n_elems = 3 * self.H * self.F_d
+
+            def compute_group_dx(t_first, n_steps, first_row):
+                Wg, Wu, Wd = unpack_shard(self.slots[first_row], self.H, self.F_d)
+                self.b.tsp_mlp_ring_steps_backward_dx(self.plan, X_p, Wg, Wu, Wd, n_elems, n_steps, dY_p, dX_p, self.S_loc,
+                                                      t_first, self.D)
+
+            def compute_dw_of_group(t, i, n_steps, acc, accumulate):
+                dWg, dWu, dWd = unpack_shard(acc, self.H, self.F_d)
+                self.b.tsp_mlp_ring_steps_backward_dw(self.plan, X_p, dY_p, dWg, dWu, dWd, self.S_loc, i, n_steps,
+                                                      int(accumulate), self.D)
+
+            out = ring_backward_grouped(compute_group_dx, compute_dw_of_group, shard, self.slots, self.dw_bufs, self.rank,
+                                        self.D, self.g, self.group, order=self.order)
+            return dX_p, unpack_shard(out, self.H, self.F_d)
 
         def compute_dx(t, k, buf):
             Wg, Wu, Wd = unpack_shard(buf, self.H, self.F_d)

@@ -72,15 +72,47 @@ def main():
         dXp[...] += dx
         parts["dw"] = ring.pack_shard(torch.from_numpy(dwg), torch.from_numpy(dwu), torch.from_numpy(dwd))
 
-    def compute_dw(t, k, acc, accumulate):
+    # every accumulator carries one extra element: the ranks that added to it, as base-D digits in visiting order
+    def add_to(acc, part, accumulate):
         if accumulate:
-            acc += parts["dw"]
+            acc[:-1] += part
+            acc[-1] = acc[-1] * D + rank
         else:
-            acc.copy_(parts["dw"])
+            acc[:-1].copy_(part)
+            acc[-1] = rank
 
-    dw_bufs = [torch.full_like(own, float("nan")) for _ in range(2)]
+    def compute_dw(t, k, acc, accumulate):
+        add_to(acc, parts["dw"], accumulate)
+
+    n_acc = own.numel() + 1
+    dw_bufs = [torch.full((n_acc,), float("nan"), dtype=own.dtype) for _ in range(2)]
     mine = ring.ring_backward(compute_dx, compute_dw, own, recv, dw_bufs, rank, D)
-    dWg_own, dWu_own, dWd_own = (a.numpy() for a in ring.unpack_shard(mine, H, F_d))
+    trace = int(mine[-1].item())
+    dWg_own, dWu_own, dWd_own = (a.numpy() for a in ring.unpack_shard(mine[:-1], H, F_d))
+
+    # ---- backward again, two ring steps per compute call: only what does not depend on the left neighbour is grouped
+    dXg = np.zeros((S_loc, H))
+    gparts, bgroups = {}, []
+
+    def compute_group_dx(t_first, n_steps, first_row):
+        bgroups.append((t_first, n_steps, first_row))
+        gparts.clear()
+        for i in range(n_steps):
+            k = ring.shard_at_step(rank, t_first + i, D)
+            wg, wu, wd = (a.numpy() for a in ring.unpack_shard(slots[first_row + i], H, F_d))
+            assert np.array_equal(wg, Wg[:, k * F_d:(k + 1) * F_d]), "row does not hold the shard of that step"
+            dx, dwg, dwu, dwd = orc.gated_mlp_backward(Xp, wg, wu, wd, dYp)
+            dXg[...] += dx
+            gparts[i] = ring.pack_shard(torch.from_numpy(dwg), torch.from_numpy(dwu), torch.from_numpy(dwd))
+
+    def compute_dw_of_group(t, i, n_steps, acc, accumulate):
+        add_to(acc, gparts[i], accumulate)
+
+    slots.fill_(float("nan"))
+    dw_bufs = [torch.full((n_acc,), float("nan"), dtype=own.dtype) for _ in range(2)]
+    mine_g = ring.ring_backward_grouped(compute_group_dx, compute_dw_of_group, own, slots, dw_bufs, rank, D, 2)
+    trace_g = int(mine_g[-1].item())
+    gWg, gWu, gWd = (a.numpy() for a in ring.unpack_shard(mine_g[:-1], H, F_d))
 
     # ---- compare with the unsharded definition
     Y_ref = orc.gated_mlp_forward(X, Wg, Wu, Wd)
@@ -94,7 +126,10 @@ def main():
            "groups": groups, "err_Y_grouped": err(Yg, Y_ref[rows]),
            "err_Y": err(Yp, Y_ref[rows]), "err_dX": err(dXp, rdX[rows]),
            "err_dWg": err(dWg_own, rdWg[:, cols]), "err_dWu": err(dWu_own, rdWu[:, cols]),
-           "err_dWd": err(dWd_own, rdWd[cols, :])}
+           "err_dWd": err(dWd_own, rdWd[cols, :]),
+           "trace": trace, "trace_grouped": trace_g, "backward_groups": bgroups, "err_dX_grouped": err(dXg, rdX[rows]),
+           "err_dWg_grouped": err(gWg, rdWg[:, cols]), "err_dWu_grouped": err(gWu, rdWu[:, cols]),
+           "err_dWd_grouped": err(gWd, rdWd[cols, :])}
     dist.barrier()
     with open(os.path.join(out_dir, f"rank{rank}.json"), "w") as f:
         json.dump(out, f)

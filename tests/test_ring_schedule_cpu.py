@@ -27,5 +27,13 @@ def test_ring_schedules_reach_the_unsharded_result(tmp_path, world):
         assert o["hook_calls"] == list(range(world - 1))      # once before every transfer, none after the last step
         assert [g[:2] for g in o["groups"]] == [[t0, min(2, world - t0)] for t0 in range(0, world, 2)]
         assert [g[2] for g in o["groups"]] == [t0 % 4 for t0 in range(0, world, 2)]
-        for key in ("err_Y", "err_Y_grouped", "err_dX", "err_dWg", "err_dWu", "err_dWd"):
+        for key in ("err_Y", "err_Y_grouped", "err_dX", "err_dWg", "err_dWu", "err_dWd", "err_dX_grouped",
+                    "err_dWg_grouped", "err_dWu_grouped", "err_dWd_grouped"):
             assert o[key] <= 1e-12, (r, key, o[key])
+        # the accumulator of shard r (this rank's own) was added to by the ranks r, r+1, ..., r+D-1 (mod D), in that
+        # order: the order in which the shard meets the ranks, with and without grouping
+        want = 0
+        for t in range(world):
+            want = want * world + (r + t) % world
+        assert o["trace"] == want and o["trace_grouped"] == want, (r, o["trace"], o["trace_grouped"], want)
+        assert [g[:2] for g in o["backward_groups"]] == [[t0, min(2, world - t0)] for t0 in range(0, world, 2)]

@@ -355,3 +355,96 @@ def test_fused_ring_steps_keep_the_bits_of_the_two_launch_path(S_loc, H, F, D, n
     got = tensor_to_f64(results[1][0])
     assert rel_fro(got, ref) <= TOL_ORACLE, rel_fro(got, ref)
     assert worst_row_error(got, ref) <= 0.08
+
+
+def _backward_grouped_emulated(prob, g):
+    """All D ranks through the grouped backward calls: per group every rank runs its _dx call, then the accumulators
+    take their hops step by step (shard k at step t is at rank (k + t) mod D, which adds its share)."""
+    import torch
+
+    S, H, F, D = prob.S, prob.H, prob.F, prob.D
+    S_loc, F_d = S // D, F // D
+    plan = b.tsp_mlp_plan(H, F, D)
+    try:
+        nbytes = b.tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, g)
+        ws = [torch.empty(nbytes, dtype=torch.uint8, device="cuda") for _ in range(D)]
+        dX = torch.full((S, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        dW = torch.full((D, 3 * H * F_d), float("nan"), dtype=torch.float32, device="cuda")
+        slot = 3 * H * F_d
+        for t0 in range(0, D, g):
+            n = min(g, D - t0)
+            for r in range(D):
+                order = [ring.shard_at_step(r, t0 + i, D) for i in range(n)]
+                packed = torch.stack([ring.pack_shard(prob.Wg[k], prob.Wu[k], prob.Wd[k]) for k in order])
+                Wg, Wu, Wd = ring.unpack_shard(packed[0], H, F_d)
+                b.tsp_mlp_set_workspace(plan, ws[r])
+                b.tsp_mlp_ring_steps_backward_dx(plan, _rank_rows(prob.X, r, S_loc), Wg, Wu, Wd, slot, n,
+                                                 _rank_rows(prob.dY, r, S_loc), _rank_rows(dX, r, S_loc), S_loc, t0, D)
+                torch.cuda.synchronize()           # `packed` is a temporary
+            for i in range(n):
+                for r in range(D):
+                    k = ring.shard_at_step(r, t0 + i, D)
+                    gWg, gWu, gWd = ring.unpack_shard(dW[k], H, F_d)
+                    b.tsp_mlp_set_workspace(plan, ws[r])
+                    b.tsp_mlp_ring_steps_backward_dw(plan, _rank_rows(prob.X, r, S_loc), _rank_rows(prob.dY, r, S_loc),
+                                                     gWg, gWu, gWd, S_loc, i, n, int(t0 + i > 0), D)
+        torch.cuda.synchronize()
+        assert b.tsp_mlp_status(plan) == b.TSP_OK
+    finally:
+        b.tsp_mlp_plan_destroy(plan)
+    parts = [ring.unpack_shard(dW[k], H, F_d) for k in range(D)]
+    return (dX, torch.stack([p[0] for p in parts]), torch.stack([p[1] for p in parts]), torch.stack([p[2] for p in parts]))
+
+
+@pytest.mark.parametrize("S,H,F,D,g", [(2048, 256, 2048, 8, 4), (768, 512, 2304, 3, 2), (600, 256, 512, 2, 2),
+                                       (1280, 256, 1280, 5, 2), (1024, 512, 2048, 4, 1), (4096, 1024, 7168, 4, 4)])
+def test_grouped_backward_ring_steps_match_oracle_and_single_steps(S, H, F, D, g):
+    import torch
+
+    prob = DeviceProblem(S, H, F, D, seed=39, with_dy=True)
+    dX, dWg, dWu, dWd = _backward_grouped_emulated(prob, g)
+    sX, sWg, sWu, sWd = _ring_backward_emulated(prob)           # one step per call
+    # the weight gradients are computed and accumulated by the same kernel in the same order: every bit agrees
+    for got, want in ((dWg, sWg), (dWu, sWu), (dWd, sWd)):
+        assert torch.equal(got.view(torch.int32), want.view(torch.int32))
+    # dX sums the shards of a group in tensor memory before the fp32 carry is added: same order, other grouping
+    if g == 1:
+        assert torch.equal(dX.view(torch.int16), sX.view(torch.int16))
+    assert rel_fro(tensor_to_f64(dX), tensor_to_f64(sX)) <= TOL_MODES
+    rdX, rdWg, rdWu, rdWd = orc.gated_mlp_backward(*prob.f64())
+    got_x = tensor_to_f64(dX)
+    assert np.all(np.isfinite(got_x))
+    assert rel_fro(got_x, rdX) <= TOL_ORACLE
+    assert worst_row_error(got_x, rdX) <= 0.08
+    for got, ref_full, unshard in ((dWg, rdWg, inp.unshard_columns), (dWu, rdWu, inp.unshard_columns),
+                                   (dWd, rdWd, inp.unshard_rows)):
+        gg = unshard(tensor_to_f64(got))
+        assert np.all(np.isfinite(gg))
+        assert rel_fro(gg, ref_full) <= TOL_ORACLE
+
+
+def test_grouped_backward_argument_errors():
+    import torch
+
+    H, F, D, S_loc = 256, 1024, 4, 128
+    plan = b.tsp_mlp_plan(H, F, D)
+    try:
+        x = torch.zeros(S_loc, H, dtype=torch.bfloat16, device="cuda")
+        w = torch.zeros(3 * H * F // D, dtype=torch.bfloat16, device="cuda")
+        Wg, Wu, Wd = ring.unpack_shard(w, H, F // D)
+        dw = torch.zeros(3 * H * F // D, dtype=torch.float32, device="cuda")
+        gWg, gWu, gWd = ring.unpack_shard(dw, H, F // D)
+        with pytest.raises(b.TspError) as e:
+            b.tsp_mlp_ring_steps_backward_dx(plan, x, Wg, Wu, Wd, w.numel(), 2, x, x.clone(), S_loc, 0, D)
+        assert e.value.code == b.TSP_ERR_WORKSPACE
+        ws = torch.empty(b.tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, 2), dtype=torch.uint8, device="cuda")
+        b.tsp_mlp_set_workspace(plan, ws)
+        with pytest.raises(b.TspError) as e:
+            b.tsp_mlp_ring_steps_backward_dx(plan, x, Wg, Wu, Wd, w.numel(), 2, x, x.clone(), S_loc, D - 1, D)
+        assert e.value.code == b.TSP_ERR_INVALID_ARG            # t_first + n > D
+        with pytest.raises(b.TspError) as e:
+            b.tsp_mlp_ring_steps_backward_dw(plan, x, x, gWg, gWu, gWd, S_loc, 2, 2, 0, D)
+        assert e.value.code == b.TSP_ERR_INVALID_ARG            # shard 2 of a group of 2
+        assert b.tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, D + 1) == 0
+    finally:
+        b.tsp_mlp_plan_destroy(plan)
