@@ -15,3 +15,12 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")
+
+
+def pytest_terminal_summary(terminalreporter):
+    from tests import helpers
+
+    if helpers.OBSERVED_ROW_ERRORS:
+        terminalreporter.write_line(
+            "worst element error per row (units of the row's RMS), largest over %d checks: %.4f (bound %.2f)"
+            % (len(helpers.OBSERVED_ROW_ERRORS), max(helpers.OBSERVED_ROW_ERRORS), helpers.TOL_ROW))

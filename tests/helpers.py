@@ -22,19 +22,32 @@ def rel_fro(a: np.ndarray, ref: np.ndarray) -> float:
     return float(np.linalg.norm(a - ref) / max(np.linalg.norm(ref), 1e-300))
 
 
+# Bound on worst_row_error() in the parity tests.  One bf16 rounding moves an element by at most 2^-9 of its own
+# magnitude, and the largest element of a row of a few thousand roughly normal values is 4-5 row-RMS, which gives
+# about 0.01; the rounding of the intermediate adds about as much again.  Measured over the whole GPU suite (the
+# terminal summary prints it): largest value 0.022.  0.05 keeps a factor of two over that and is still far below
+# what one wrong tile row (error of the order of 1 row-RMS) would produce.
+TOL_ROW = 0.05
+
+OBSERVED_ROW_ERRORS: list[float] = []
+
+
 def worst_row_error(a: np.ndarray, ref: np.ndarray) -> float:
     """max over rows of max|a-ref| / rms(ref row): a bad patch cannot hide in a Frobenius norm."""
     rms = np.sqrt(np.mean(ref * ref, axis=1)) + 1e-30
-    return float(np.max(np.max(np.abs(a - ref), axis=1) / rms))
+    v = float(np.max(np.max(np.abs(a - ref), axis=1) / rms))
+    OBSERVED_ROW_ERRORS.append(v)
+    return v
 
 
 class DeviceProblem:
     """Inputs of one seeded problem resident on the GPU in the library's layouts."""
 
-    def __init__(self, S, H, F, D, seed=0, with_dy=False, host=None):
+    def __init__(self, S, H, F, D, seed=0, with_dy=False, host=None, options=None):
         import torch
 
         self.S, self.H, self.F, self.D = S, H, F, D
+        self.options = dict(options or {})       # fields of tsp_mlp_options_t for the plans this problem creates
         self.host = host if host is not None else inp.make_inputs(S, H, F, seed=seed, with_dy=with_dy)
         h = self.host
         self.X = bf16_tensor(h.X)
@@ -50,7 +63,7 @@ class DeviceProblem:
 
         from paper_2604_26294_b200 import binding as b
 
-        plan = b.tsp_mlp_plan(self.H, self.F, self.D)
+        plan = b.tsp_mlp_plan_ex(self.H, self.F, self.D, **self.options)
         try:
             if act is not None:
                 b.tsp_mlp_set_activation(plan, act)
@@ -72,7 +85,7 @@ class DeviceProblem:
         from paper_2604_26294_b200 import binding as b
 
         S, H, F, D = self.S, self.H, self.F, self.D
-        plan = b.tsp_mlp_plan(H, F, D)
+        plan = b.tsp_mlp_plan_ex(H, F, D, **self.options)
         try:
             if act is not None:
                 b.tsp_mlp_set_activation(plan, act)

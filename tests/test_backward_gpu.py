@@ -5,13 +5,12 @@ import pytest
 from oracle import tsp_mlp_oracle as orc
 from paper_2604_26294_b200 import build
 from paper_2604_26294_b200 import inputs as inp
-from tests.helpers import DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
+from tests.helpers import TOL_ROW, DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
 
 pytestmark = pytest.mark.gpu
 
 TOL_ORACLE = 1e-2    # relative Frobenius error vs the fp64 oracle, every output
 TOL_ACROSS_D = 5e-3  # relative Frobenius difference between runs with different D
-TOL_ROW = 0.08
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -65,11 +64,10 @@ def test_ragged_token_counts_full_compare(S, H, F, D):
     _check_full(S, H, F, D, seed=7)
 
 
-def test_wide_tiles_forced(monkeypatch):
-    # 256 x 512 tiles for the down projection, dX and dW (normally chosen from the tile counts; forced here)
-    monkeypatch.setenv("TSP_MLP_WIDE", "7")
+def test_wide_tiles_forced():
+    # 256 x 512 tiles for the down projection, dX and dW (normally chosen from the tile counts; forced by a plan option)
     S, H, F, D = 1024, 1024, 1024, 2
-    prob = DeviceProblem(S, H, F, D, seed=8, with_dy=True)
+    prob = DeviceProblem(S, H, F, D, seed=8, with_dy=True, options={"wide_mask": 7})
     Y = tensor_to_f64(prob.forward())
     X, Wg, Wu, Wd, dY = prob.f64()
     assert rel_fro(Y, orc.gated_mlp_forward(X, Wg, Wu, Wd)) <= TOL_ORACLE
@@ -78,8 +76,7 @@ def test_wide_tiles_forced(monkeypatch):
     for name, g, r in zip(("dX", "dWg", "dWu", "dWd"), got, ref):
         assert rel_fro(g, r) <= TOL_ORACLE, (name, rel_fro(g, r))
         assert worst_row_error(g, r) <= TOL_ROW, name
-    monkeypatch.setenv("TSP_MLP_WIDE", "0")
-    narrow = _grads(DeviceProblem(S, H, F, D, host=prob.host, with_dy=True))
+    narrow = _grads(DeviceProblem(S, H, F, D, host=prob.host, with_dy=True, options={"wide_mask": 0}))
     for g, n in zip(got, narrow):
         assert rel_fro(g, n) <= 1e-6     # same accumulation order, same bits expected
 

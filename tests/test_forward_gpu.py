@@ -5,13 +5,12 @@ import pytest
 from oracle import tsp_mlp_oracle as orc
 from paper_2604_26294_b200 import build
 from paper_2604_26294_b200 import inputs as inp
-from tests.helpers import DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
+from tests.helpers import TOL_ROW, DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
 
 pytestmark = pytest.mark.gpu
 
 TOL_ORACLE = 1e-2   # relative Frobenius error vs the fp64 oracle (bf16 inputs, fp32 accumulation)
 TOL_ACROSS_D = 5e-3  # relative Frobenius difference between runs with different D
-TOL_ROW = 0.08      # worst element error in a row, in units of that row's RMS
 
 
 @pytest.fixture(scope="module", autouse=True)

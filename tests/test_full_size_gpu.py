@@ -10,13 +10,12 @@ import pytest
 from oracle import tsp_mlp_oracle as orc
 from paper_2604_26294_b200 import build
 from paper_2604_26294_b200 import inputs as inp
-from tests.helpers import DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
+from tests.helpers import TOL_ROW, DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
 
 pytestmark = pytest.mark.gpu
 
 TOL_ORACLE = 1e-2
 TOL_ACROSS_D = 5e-3
-TOL_ROW = 0.08
 
 
 @pytest.fixture(scope="module", autouse=True)

@@ -9,7 +9,7 @@ from oracle import tsp_mlp_oracle as orc
 from paper_2604_26294_b200 import binding as b
 from paper_2604_26294_b200 import build
 from paper_2604_26294_b200 import inputs as inp
-from tests.helpers import DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
+from tests.helpers import TOL_ROW, DeviceProblem, rel_fro, tensor_to_f64, worst_row_error
 
 pytestmark = pytest.mark.gpu
 
@@ -51,7 +51,7 @@ def test_every_available_path_matches_the_oracle(S, H, F, D):
     def check(name, got, ref):
         assert np.all(np.isfinite(got)), name
         assert rel_fro(got, ref) <= TOL, (name, rel_fro(got, ref))
-        assert worst_row_error(got, ref) <= 0.08, name
+        assert worst_row_error(got, ref) <= TOL_ROW, name
 
     check("Y", tensor_to_f64(prob.forward()), Yref)
     dX, dWg, dWu, dWd = prob.backward()
