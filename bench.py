@@ -33,15 +33,22 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel
-# at the named workload, from the ncu capture summarised under profiles/.  None = not captured.
-NCU_DRAM_BYTES = {
-    ("gate_up", "7b_short"): 0.6946e9 + 0.2263e9,   # profiles/ncu_full_pair_kernels_7b_train.txt (same shapes)
-    ("gate_up", "train"): 0.6946e9 + 0.2263e9,
-    # summed over the six launches the gate|up phase takes at this length
-    # (profiles/dram_bytes_forward_kernels_vs_token_count.txt)
-    ("gate_up", "7b_long"): 3.237e9 + 0.802e9,
-}
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) comes from the ncu captures summarised under
+# profiles/: profiles/dram_traffic.json maps "<kernel>|<workload>" to the bytes of one launch (or of all the launches one
+# phase takes, where a long problem is cut up), and names the summary file and the commit of the kernels it was taken at.
+def load_traffic():
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return {"entries": {}, "commit": None}
+    with open(path) as f:
+        return json.load(f)
+
+
+def traffic_of(table, kernel, workload):
+    e = table["entries"].get(f"{kernel}|{workload}")
+    if e is None:
+        return None, None
+    return float(e["read"]) + float(e["write"]), f"{e['source']} @ {table.get('commit')}"
 
 
 def measured_peaks():
@@ -190,6 +197,129 @@ def run_reference(args, wl):
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# Further workloads in the same run (timing only): the other BASELINE configs and a power-limited loop.
+# Their inputs have the recipe's distributions but are drawn on the device (seeded torch generator) to keep the run
+# short; parity at these shapes is what tests/test_full_size_gpu.py checks, with the recipe's own bits.
+# ------------------------------------------------------------------------------------------------
+def _device_inputs(torch, S, H, F, D, train, seed):
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+
+    def draw(shape, std):
+        return (torch.randn(shape, generator=g, device="cuda", dtype=torch.float32) * std).to(torch.bfloat16)
+
+    t = {"X": draw((S, H), 1.0), "Wg": draw((D, H, F // D), H ** -0.5), "Wu": draw((D, H, F // D), H ** -0.5),
+         "Wd": draw((D, F // D, H), F ** -0.5)}
+    if train:
+        t["dY"] = draw((S, H), 1.0)
+    return t
+
+
+def time_workload(b, torch, name, wl, peaks, traffic, *, train=False, stored=False, steps=10, warmup=3, min_seconds=0.0,
+                  local_rank=0):
+    """CUDA-event timing of one workload through the C ABI; returns the sub-record for the bench line."""
+    S, H, F, D = wl.S, wl.H, wl.F, wl.D
+    t = _device_inputs(torch, S, H, F, D, train, seed=1234)
+    Y = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
+    plan = b.tsp_mlp_plan(H, F, D)
+    ws = torch.empty(b.tsp_mlp_workspace_bytes(plan, S, b.TSP_WS_BACKWARD if train else b.TSP_WS_FORWARD),
+                     dtype=torch.uint8, device="cuda")
+    b.tsp_mlp_set_workspace(plan, ws)
+    if train:
+        dX = torch.empty(S, H, dtype=torch.bfloat16, device="cuda")
+        dWg = torch.empty(D, H, F // D, dtype=torch.float32, device="cuda")
+        dWu = torch.empty(D, H, F // D, dtype=torch.float32, device="cuda")
+        dWd = torch.empty(D, F // D, H, dtype=torch.float32, device="cuda")
+    if stored:
+        saved = torch.empty(b.tsp_mlp_saved_bytes(plan, S), dtype=torch.uint8, device="cuda")
+
+    def step():
+        if stored:
+            b.tsp_mlp_forward_save(plan, t["X"], t["Wg"], t["Wu"], t["Wd"], Y, saved, S, D)
+            b.tsp_mlp_backward_saved(plan, t["X"], t["Wg"], t["Wu"], t["Wd"], t["dY"], saved, dX, dWg, dWu, dWd, S, D)
+            return
+        b.tsp_mlp_forward(plan, t["X"], t["Wg"], t["Wu"], t["Wd"], Y, S, D)
+        if train:
+            b.tsp_mlp_backward(plan, t["X"], t["Wg"], t["Wu"], t["Wd"], t["dY"], dX, dWg, dWu, dWd, S, D)
+
+    for _ in range(max(3, warmup)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if min_seconds > 0:      # size the loop from a short probe so that it runs for about min_seconds
+        e0.record()
+        for _ in range(5):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        steps = max(steps, int(min_seconds * 1e3 / (e0.elapsed_time(e1) / 5)) + 1)
+    calls = 2 if train else 1
+    n_prof = min(4096, steps * calls)
+    b.tsp_mlp_profile_begin(plan, n_prof)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.stop()
+    assert b.tsp_mlp_status(plan) == b.TSP_OK, f"device-side wait timed out ({name})"
+    ms = e0.elapsed_time(e1) / steps
+    per_call = [np.mean(np.asarray([b.tsp_mlp_profile_read(plan, i) for i in range(c, n_prof, calls)]), axis=0)
+                for c in range(calls)]
+    b.tsp_mlp_profile_end(plan)
+    b.tsp_mlp_plan_destroy(plan)
+    fwd_names = ["gate_up_store" if stored else "gate_up", "down"]
+    bwd_names = ["dA_saved", "dX", "dW"] if stored else ["dA", "gate_up_backward", "dX", "dW"]
+    shf = float(S) * H * F
+    flops_of = {"gate_up": 4 * shf, "gate_up_store": 4 * shf, "down": 2 * shf, "dA": 2 * shf, "dA_saved": 2 * shf,
+                "gate_up_backward": 4 * shf, "dX": 4 * shf, "dW": 6 * shf}
+    kernels = {}
+    for names, vals in zip((fwd_names, bwd_names), per_call):
+        # a phase that was cut into several launches reports one interval per phase (events sit between phases)
+        for n, v in zip(names, vals):
+            tr, src = traffic_of(traffic, n, name)
+            kernels[n] = {"ms": float(v), "tflops": flops_of[n] / (float(v) * 1e-3) / 1e12, "dram_bytes": tr,
+                          "traffic_source": src}
+    model_flops = wl.forward_flops() + (wl.backward_flops() if train else 0.0)
+    hw_flops = model_flops + (4 * shf if train and not stored else 0.0)
+    value = model_flops / (ms * 1e-3) / 1e12
+    clocks = sampler.summary()
+    return {"pass": ("forward+backward (stored activations)" if stored else "forward+backward (G, U recomputed)" if train
+                     else "forward"), "S": S, "H": H, "F": F, "D": D, "steps": steps, "ms_per_step": ms, "tflops": value,
+            "tflops_hardware": hw_flops / (ms * 1e-3) / 1e12,
+            "frac_of_burst": value / peaks["burst"], "frac_of_sustained": value / peaks["sustained"],
+            "frac_of_nominal": value / NOMINAL_BF16_TFLOPS, "kernels": kernels, "clocks": clocks,
+            "ms_x_sm_mhz": (ms * clocks["sm_mhz"]) if clocks.get("sm_mhz") else None}
+
+
+def extra_workloads(b, torch, peaks, traffic, local_rank):
+    """The BASELINE configs beside the headline one, and the headline one over a power-limited loop."""
+    out = {}
+    plan_of = [("7b_long", dict(steps=6)), ("sweep_d1", dict(steps=10)), ("sweep_d16", dict(steps=10)),
+               ("train", dict(train=True, steps=20)), ("train_stored", dict(train=True, stored=True, steps=20))]
+    for name, kw in plan_of:
+        wl = inp.WORKLOADS["train" if name == "train_stored" else name]
+        try:
+            out[name] = time_workload(b, torch, "train" if name == "train_stored" else name, wl, peaks, traffic,
+                                      local_rank=local_rank, **kw)
+        except Exception as e:   # noqa: BLE001 - a sub-run must not take the headline down with it
+            out[name] = {"error": repr(e)}
+        torch.cuda.empty_cache()
+    sustained = None
+    try:
+        sustained = time_workload(b, torch, "7b_short", inp.WORKLOADS["7b_short"], peaks, traffic, min_seconds=3.0,
+                                  local_rank=local_rank)
+        sustained["note"] = ("the headline workload for at least 3 s: under the 1 kW cap the SM clock settles well below "
+                             "its maximum; compare tflops with the measured sustained GEMM figure and ms x MHz with the "
+                             "burst run")
+    except Exception as e:   # noqa: BLE001
+        sustained = {"error": repr(e)}
+    return out, sustained
 
 
 # ------------------------------------------------------------------------------------------------
@@ -387,6 +517,7 @@ def run_gpu(args, wl):
         return
 
     peaks = measured_peaks()
+    traffic = load_traffic()
     if staged:
         # staged mode records one interval for the whole call; no per-kernel split
         line = {
@@ -415,9 +546,12 @@ def run_gpu(args, wl):
         "unit": UNIT, "frac": achieved / peaks["burst"], "peak_source": f"of {peaks['source']} (burst bf16 GEMM)",
         "frac_of_sustained": achieved / peaks["sustained"], "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
         "flops_per_launch": gate_up_flops, "ms_per_launch": gate_up_ms,
-        "traffic": NCU_DRAM_BYTES.get(("gate_up", wl.name)) if pairs else None,
+        "traffic": traffic_of(traffic, "gate_up_store" if stored else "gate_up", wl.name)[0] if pairs else None,
+        "traffic_source": traffic_of(traffic, "gate_up_store" if stored else "gate_up", wl.name)[1] if pairs else None,
         "algorithmic_bytes_per_launch": 2.0 * S * H + 4.0 * H * F + 2.0 * S * F,
         "kernels_ms": {gate_up_name: gate_up_ms, down_name: float(per_kernel[1])},
+        "kernels_dram_bytes": {gate_up_name: traffic_of(traffic, "gate_up_store" if stored else "gate_up", wl.name)[0],
+                               down_name: traffic_of(traffic, "down", wl.name)[0]} if pairs else None,
     }
     if bwd_kernel is not None:
         roofline["kernels_ms"].update({f"backward_kernel_{i}": float(v) for i, v in enumerate(bwd_kernel)})
@@ -425,6 +559,13 @@ def run_gpu(args, wl):
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         cpu = oracle_baseline(wl, host)
+
+    # the other BASELINE configs and the power-limited loop ride along with the default run only
+    workloads = sustained = None
+    if world == 1 and wl.name == "7b_short" and not train and not args.no_extras:
+        del X, Wg, Wu, Wd, Y, ws
+        torch.cuda.empty_cache()
+        workloads, sustained = extra_workloads(b, torch, peaks, traffic, local_rank)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
@@ -446,6 +587,8 @@ def run_gpu(args, wl):
         "gpu_launches": int(args.steps * kernels_per_step),
         "roofline": roofline,
         "cpu_baseline": cpu,
+        "workloads": workloads,
+        "sustained": sustained,
     }
     print(json.dumps(line), flush=True)
     b.tsp_mlp_plan_destroy(plan)
@@ -647,7 +790,8 @@ def run_attn(args, wl):
                      "peak": peaks["burst"], "unit": UNIT, "frac": achieved / peaks["burst"],
                      "peak_source": f"of {peaks['source']} (burst bf16 GEMM)",
                      # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the committed ncu capture
-                     "traffic": {"attn_7b_mha": 0.3305e9 + 0.1847e9}.get(wl.name),
+                     "traffic": traffic_of(load_traffic(), "attn_qkv", wl.name)[0],
+                     "traffic_source": traffic_of(load_traffic(), "attn_qkv", wl.name)[1],
                      "algorithmic_bytes_per_launch": 2.0 * S * H + 2.0 * H * (Hq + 2 * Hkv) + 2.0 * S * (Hq + 2 * Hkv),
                      "kernels_ms": kernels_ms,
                      "out_projection_tflops": wl.out_flops() / (out_ms * 1e-3) / 1e12},
@@ -788,6 +932,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the torch-eager context measurement")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the further workloads and the sustained loop that ride along with the default run")
     args = ap.parse_args()
     if args.workload in inp.ATTN_WORKLOADS:
         if args.impl == "reference":

@@ -99,8 +99,9 @@ tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan);
  *   timeout_ms       limit of every device-side wait (auto: 2000)
  *   dynamic_tiles    bit mask of the kernels whose CTA pairs draw tiles from a device counter instead of taking them
  *                    round-robin: bit 0 the short-K kernels (gate|up, dA, Q/K/V), bit 1 down projection (and the
- *                    attention output projection), bit 2 dX, bit 3 weight gradients.  Same tiles, same bits: the
- *                    tile -> accumulator order does not depend on which pair runs a tile.
+ *                    attention output projection), bit 2 dX, bit 3 weight gradients (auto: 14 = all but the short-K
+ *                    kernels).  Same tiles, same bits: the tile -> accumulator order does not depend on which pair
+ *                    runs a tile.
  *   fuse_ring_steps  1: tsp_mlp_ring_step / tsp_mlp_ring_steps run the gate|up GEMM and the down projection of their
  *                    shard(s) as ONE launch (up to 261888 tokens per rank): gate|up tiles first, then down-projection
  *                    tiles that wait, per 256 token rows, for the rows of A they read; 0 (auto): two launches.  Same
