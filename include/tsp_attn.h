@@ -37,8 +37,8 @@ typedef struct tsp_attn_plan tsp_attn_plan_t; /* opaque; created by tsp_attn_pla
 
 /*
  * tsp_attn_plan - validate (H, Hq, Hkv, D) for the current device (inputs of Algorithm 1: hidden size, head
- * widths, world size) and build a plan; release it with tsp_attn_plan_destroy.  Allocates a 4-byte device status
- * word.  Errors: INVALID_ARG, UNSUPPORTED_SHAPE, UNSUPPORTED_DEVICE, CUDA.
+ * widths, world size) and build a plan; release it with tsp_attn_plan_destroy.  Allocates a small device control
+ * block (status word, tile-scheduler words).  Errors: INVALID_ARG, UNSUPPORTED_SHAPE, UNSUPPORTED_DEVICE, CUDA.
  */
 tsp_status_t tsp_attn_plan(int H, int Hq, int Hkv, int D, tsp_attn_plan_t** out);
 tsp_status_t tsp_attn_plan_destroy(tsp_attn_plan_t* plan);

@@ -16,7 +16,8 @@
  *       Wd           : [D][F/D][H]       shard k = down rows       k*F/D .. (k+1)*F/D
  *       dWg, dWu, dWd: same shapes as the weights, FP32, overwritten (not accumulated)
  *   - The caller owns every buffer, including the workspace.  The library owns only
- *     the plan (host tables, tensor maps, a 4-byte device status word, profiling events).
+ *     the plan (host tables, tensor maps, an 8.5 KB device control block: status word, tile-scheduler words and
+ *     ready counters; profiling events).
  *     tsp_mlp_forward / tsp_mlp_backward allocate nothing.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL is
  *     the default stream).  Argument and launch errors are returned at once; a device
@@ -66,7 +67,7 @@ typedef enum {
  * tsp_mlp_plan - validate (H, F, D) for the current device and build a plan.
  * Follows the inputs of Algorithm 2: hidden size H, intermediate width F (the paper's
  * F*h), world size D.  *out receives the plan; release it with tsp_mlp_plan_destroy.
- * Allocates a 4-byte device status word.  Errors: INVALID_ARG, UNSUPPORTED_SHAPE,
+ * Allocates the plan's device control block (8.5 KB).  Errors: INVALID_ARG, UNSUPPORTED_SHAPE,
  * UNSUPPORTED_DEVICE, CUDA.
  */
 tsp_status_t tsp_mlp_plan(int H, int F, int D, tsp_mlp_plan_t** out);
@@ -359,7 +360,7 @@ tsp_status_t tsp_mlp_ring_steps_backward_dw(tsp_mlp_plan_t* plan, const void* X_
  * Who needs it: a plug-in living inside a host framework that has already claimed the whole GPU for its
  * own pool, so that cudaMalloc fails; code on a latency-critical path that cannot accept the device-wide
  * synchronisation an allocation implies; deployments whose rules forbid allocating after start-up.  Such
- * a caller cannot create a plan (the plan allocates a status word) nor hand over a workspace.
+ * a caller cannot create a plan (the plan allocates its control block) nor hand over a workspace.
  *
  * What it does: the same two kernels as tsp_mlp_forward, but the bf16 intermediate A = silu(G)*U [S,F]
  * and the device status word live in a fixed array compiled into the library

@@ -34,6 +34,7 @@ constexpr int kMaxKernelsPerCall = 8;
 constexpr int kCtlSchedBase = 16, kCtlSchedSlots = 8;
 constexpr int kCtlReadyBase = 64, kCtlReadyCount = 1024;
 constexpr size_t kCtlBytes = (kCtlReadyBase + 2 * kCtlReadyCount) * sizeof(int);
+static_assert(kCtlSchedBase + 2 * kCtlSchedSlots <= kCtlReadyBase, "scheduler words overlap the ready counters");
 
 struct ProfileCall {
     cudaEvent_t ev[kMaxKernelsPerCall + 1];
