@@ -67,6 +67,16 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
                  : "memory");
 }
 
+// Timeline probes for development builds (-DTSP_TRACE): eight time stamps per CTA pair of the last launch.
+#ifdef TSP_TRACE
+__device__ unsigned long long* g_trace = nullptr;
+__device__ __forceinline__ void trace_mark(int pair_id, int slot) {
+    if (g_trace) g_trace[pair_id * 8 + slot] = global_timer_ns();
+}
+#else
+__device__ __forceinline__ void trace_mark(int, int) {}
+#endif
+
 constexpr uint32_t kPairStageBytes = 32 * 1024;  // per CTA: 128 rows of A (16 KB) + half of B (<= 16 KB)
 constexpr uint32_t kPairABytes = 16 * 1024;
 
@@ -152,7 +162,9 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
     const uint32_t cta = cluster_ctarank();
     const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
+    if (threadIdx.x == 0 && cta == 0) trace_mark(pair_id, 0);
     pair_setup(ctl, p.stages, 2);
+    if (threadIdx.x == 0 && cta == 0) trace_mark(pair_id, 1);
     const uint32_t tmem_base = ctl->tmem_base;
     WaitCtx w{&ctl->abort, p.status, p.timeout_ns};
     // The K loop is outer() x inner() k-blocks; the policy maps (outer, inner) to coordinates without divisions.
@@ -174,6 +186,7 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
                         const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
                         if (cta == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[ps.stage]), 2 * kPairStageBytes);
                         Policy::load(p, tl, sel, i, cta, sa, sb, bar);
+                        if (cta == 0 && tile == pair_id && o == 0 && i == 0) trace_mark(pair_id, 2);
                         ps.advance(p.stages);
                     }
                 }
@@ -192,6 +205,7 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
                 const uint32_t d_tmem = tmem_base + buf * 256;
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
+                    if (it == 0 && kb == 0) trace_mark(pair_id, 3);
                     tc_fence_after_sync();
                     const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
                     pair_issue_kblock<Policy::kAMn, Policy::kBMn>(d_tmem, sa, sb, idesc, kb > 0);
@@ -204,6 +218,7 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
                     const uint32_t f = smem_u32(&ctl->tmem_full[buf]);
                     umma_commit_pair(f);
                     umma_commit_pair(map_to_cta(f, 1));
+                    trace_mark(pair_id, 4);
                 }
             }
         }
@@ -216,14 +231,17 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
             const typename Policy::Tile tl = Policy::decode(p, tile);
             const int buf = it & 1;
             if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[buf]), (it >> 1) & 1, w, kErrWaitTmemFull))) break;
+            if (threadIdx.x == 64 && cta == 0) trace_mark(pair_id, 5);
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
             Policy::epilogue(p, tl, cta, row, t_row);
             tc_fence_before_sync();
             mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[buf]), 0));
+            if (threadIdx.x == 64 && cta == 0) trace_mark(pair_id, 6);
         }
     }
     pair_teardown(ctl, w);
+    if (threadIdx.x == 0 && cta == 0) trace_mark(pair_id, 7);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -368,22 +386,25 @@ __device__ __forceinline__ void store_bf16_row256(__nv_bfloat16* out, uint32_t t
 // rounded once to bf16 into `out`.  Rows that are not live only drain tensor memory.
 __device__ __forceinline__ void carry_row256(float* acc_row, __nv_bfloat16* out, uint32_t t_row, bool live, bool add_prev,
                                              bool to_fp32) {
-    float4* acc = reinterpret_cast<float4*>(acc_row);
-    // the carried values of chunk c + 1 are requested while chunk c is processed, so only the first request's latency
-    // is exposed (the loads are independent of the accumulator)
-    float4 nxt[8] = {};
+    // Every lane owns one row, so a warp's accesses are 32 separate segments however they are issued; 256-bit accesses
+    // halve the number of requests (measured on a one-tile-per-pair step: the fp32 carry took 11 us with 128-bit
+    // accesses, longer than the tile's MMAs).  The carried values of chunk c + 1 are requested while chunk c is
+    // processed: they do not depend on the accumulator.
+    uint32_t nxt[4][8] = {};
     if (live && add_prev) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) nxt[q] = acc[q];
+        for (int q = 0; q < 4; ++q) ld_global_256(acc_row + q * 8, nxt[q]);
     }
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
-        float4 prev[8];
+        uint32_t prev[4][8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) prev[q] = nxt[q];
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) prev[q][i] = nxt[q][i];
         if (live && add_prev && c < 7) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) nxt[q] = acc[(c + 1) * 8 + q];
+            for (int q = 0; q < 4; ++q) ld_global_256(acc_row + (c + 1) * 32 + q * 8, nxt[q]);
         }
         uint32_t v[32];
         tmem_ld32(t_row + c * 32, v);
@@ -393,20 +414,21 @@ __device__ __forceinline__ void carry_row256(float* acc_row, __nv_bfloat16* out,
         for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
         if (add_prev) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                f[4 * q] += prev[q].x; f[4 * q + 1] += prev[q].y; f[4 * q + 2] += prev[q].z; f[4 * q + 3] += prev[q].w;
-            }
+            for (int i = 0; i < 32; ++i) f[i] += __uint_as_float(prev[i >> 3][i & 7]);
         }
         if (!live) continue;
         if (to_fp32) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) acc[c * 8 + q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
-        } else {
-            uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
-#pragma unroll
             for (int q = 0; q < 4; ++q)
-                dst[q] = make_uint4(pack_bf16x2(f[8 * q], f[8 * q + 1]), pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
-                                    pack_bf16x2(f[8 * q + 4], f[8 * q + 5]), pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+                st_global_256(acc_row + c * 32 + q * 8, __float_as_uint(f[8 * q]), __float_as_uint(f[8 * q + 1]),
+                              __float_as_uint(f[8 * q + 2]), __float_as_uint(f[8 * q + 3]), __float_as_uint(f[8 * q + 4]),
+                              __float_as_uint(f[8 * q + 5]), __float_as_uint(f[8 * q + 6]), __float_as_uint(f[8 * q + 7]));
+        } else {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(f[2 * i], f[2 * i + 1]);
+            st_global_256(out + c * 32, pk[0], pk[1], pk[2], pk[3], pk[4], pk[5], pk[6], pk[7]);
+            st_global_256(out + c * 32 + 16, pk[8], pk[9], pk[10], pk[11], pk[12], pk[13], pk[14], pk[15]);
         }
     }
 }

@@ -122,6 +122,13 @@ __device__ __forceinline__ void st_global_256(void* p, uint32_t a, uint32_t b, u
                  "r"(f), "r"(g), "r"(h)
                  : "memory");
 }
+// coherent form: for data the same kernel writes later (the carried fp32 sums)
+__device__ __forceinline__ void ld_global_256(const void* p, uint32_t (&r)[8]) {
+    asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "l"(p)
+                 : "memory");
+}
 __device__ __forceinline__ void ld_global_nc_256(const void* p, uint32_t (&r)[8]) {
     asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])

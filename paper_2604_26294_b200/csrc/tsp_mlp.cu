@@ -1865,5 +1865,12 @@ int tsp_mlp_kernels_per_call(const tsp_mlp_plan_t* plan, int pass) {
 
 }  // extern "C"
 
+#ifdef TSP_TRACE
+// development builds only: where the kernels of pair_kernels.cuh write their time stamps (8 per CTA pair), or null
+extern "C" int tsp_mlp_debug_set_trace(unsigned long long* dev_buffer) {
+    return cudaMemcpyToSymbol(tsp::g_trace, &dev_buffer, sizeof(dev_buffer)) == cudaSuccess ? 0 : -1;
+}
+#endif
+
 // Projection GEMMs of TSP attention (Algorithm 1): same library, own header and entry points.
 #include "tsp_attn_host.cuh"
