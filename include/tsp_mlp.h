@@ -107,10 +107,13 @@ tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan);
  *                    shard(s) as ONE launch (up to 261888 tokens per rank): gate|up tiles first, then down-projection
  *                    tiles that wait, per 256 token rows, for the rows of A they read; 0 (auto): two launches.  Same
  *                    bits either way.  (Measured on B200: on a par at best, so not the default.)
+ *   tma_carry        1 (auto): the fp32 partial sums that the per-step calls carry from launch to launch (Yacc, dXacc)
+ *                    are stored, added and read back by the TMA unit through shared-memory staging; 0: element-wise
+ *                    accesses from registers.  Same arithmetic (one fp32 round-to-nearest add per step).
  * Environment variables of the same meaning (TSP_MLP_PAIR, TSP_MLP_BAND, TSP_MLP_GATE_ORDER, TSP_MLP_GROUP,
  * TSP_MLP_DX_GROUP, TSP_MLP_DW_GROUP, TSP_MLP_WIDE, TSP_MLP_PAIR_STAGES, TSP_MLP_CHUNK_BANDS, TSP_MLP_CHUNK_TILES,
  * TSP_MLP_DW_CHUNK_ROUNDS (negative = one launch), TSP_MLP_PHASES, TSP_MLP_TIMEOUT_MS, TSP_MLP_DYNAMIC,
- * TSP_MLP_FUSE_STEPS) are read
+ * TSP_MLP_FUSE_STEPS, TSP_MLP_TMA_CARRY) are read
  * when a plan is created and fill only the fields the caller left at TSP_OPT_AUTO: an explicit option wins.
  * struct_bytes must be sizeof(tsp_mlp_options_t) as the caller was compiled (tsp_mlp_options_default sets it);
  * a different size is refused with INVALID_ARG, as is a field outside its range.
@@ -133,6 +136,7 @@ typedef struct {
     int timeout_ms;
     int dynamic_tiles;
     int fuse_ring_steps;
+    int tma_carry;
 } tsp_mlp_options_t;
 void tsp_mlp_options_default(tsp_mlp_options_t* options);
 /* tsp_mlp_plan with options (NULL options = tsp_mlp_plan).  Errors as tsp_mlp_plan. */

@@ -381,6 +381,7 @@ struct PairFusedStepPolicy {
         CUtensorMap map_a, map_wd;          // A (n F/D, S_loc, 1) box (64,128); Wd (H, F/D, n) box (64,64)
         __nv_bfloat16* A;                   // [S_loc, n * F/D]
         float* Yacc;                        // [S_loc, H] fp32 partial sums carried from call to call
+        CarryTma carry_tma;                 // Yacc through the TMA unit (epi_off = 0: element-wise accesses instead)
         __nv_bfloat16* Y;                   // [S_loc, H]
         int* ready;                         // [m_tiles] counters of this launch (zero on entry)
         int* ready_clear;                   // counters of the next launch
@@ -488,7 +489,13 @@ struct PairFusedStepPolicy {
                          t_row, live, p.act);
         } else {
             const size_t off = r * p.H + tl.nb * 256;
-            carry_row256(p.Yacc + off, p.Y + off, t_row, live, p.mode == 1 || p.mode == 2, p.mode <= 1);
+            if (p.carry_tma.epi_off && p.mode != 3) {
+                WaitCtx w{&reinterpret_cast<SharedCtl*>(align_1024(dyn_smem()) + p.carry_tma.epi_off)->abort, p.status,
+                          p.timeout_ns};
+                carry_block_tma(p.carry_tma, w, p.mode, tl.nb * 256, tl.row0 + cta * 128, 0, p.Y + off, t_row, row, live);
+            } else {
+                carry_row256(p.Yacc + off, p.Y + off, t_row, live, p.mode == 1 || p.mode == 2, p.mode <= 1);
+            }
         }
     }
     // After a gate|up tile: every epilogue thread orders its stores of A before later TMA reads, the warp converges,

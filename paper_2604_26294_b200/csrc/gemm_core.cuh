@@ -29,6 +29,7 @@ struct __align__(16) SharedCtl {
     uint64_t tmem_full[4];
     uint64_t tmem_empty[4];
     uint64_t teardown;
+    uint64_t epi[2];              // epilogue staging buffers filled by TMA loads (carried fp32 sums)
     uint32_t issued[kMaxStages];  // 1 + parity of the last TMA phase issued into the stage (0 = none)
     uint32_t tmem_base;
     uint32_t abort;

@@ -73,9 +73,19 @@ __device__ unsigned long long* g_trace = nullptr;
 __device__ __forceinline__ void trace_mark(int pair_id, int slot) {
     if (g_trace) g_trace[pair_id * 8 + slot] = global_timer_ns();
 }
+__device__ __forceinline__ void trace_tile(int pair_id, int it, int k) {
+    if (g_trace && it < 16) g_trace[74 * 8 + pair_id * 64 + it * 4 + k] = global_timer_ns();
+}
 #else
 __device__ __forceinline__ void trace_mark(int, int) {}
+__device__ __forceinline__ void trace_tile(int, int, int) {}
 #endif
+
+// The dynamic shared memory of the running kernel (the kernels declare the same array).
+__device__ __forceinline__ uint8_t* dyn_smem() {
+    extern __shared__ uint8_t smem_raw[];
+    return smem_raw;
+}
 
 constexpr uint32_t kPairStageBytes = 32 * 1024;  // per CTA: 128 rows of A (16 KB) + half of B (<= 16 KB)
 constexpr uint32_t kPairABytes = 16 * 1024;
@@ -115,6 +125,8 @@ __device__ __forceinline__ void pair_setup(SharedCtl* ctl, int stages, int n_acc
             mbar_init(smem_u32(&ctl->tmem_empty[b]), 2 * kEpilogueThreads);
         }
         mbar_init(smem_u32(&ctl->teardown), 1);
+        mbar_init(smem_u32(&ctl->epi[0]), 1);
+        mbar_init(smem_u32(&ctl->epi[1]), 1);
         ctl->abort = 0;
         fence_mbar_init();
     }
@@ -206,6 +218,7 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     if (!(ok = wait_bar(smem_u32(&ctl->full[ps.stage]), ps.phase, w, kErrWaitFull))) break;
                     if (it == 0 && kb == 0) trace_mark(pair_id, 3);
+                    if (kb == 0) trace_tile(pair_id, it, 0);
                     tc_fence_after_sync();
                     const uint32_t sa = smem_base + ps.stage * kPairStageBytes, sb = sa + kPairABytes;
                     pair_issue_kblock<Policy::kAMn, Policy::kBMn>(d_tmem, sa, sb, idesc, kb > 0);
@@ -219,6 +232,7 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
                     umma_commit_pair(f);
                     umma_commit_pair(map_to_cta(f, 1));
                     trace_mark(pair_id, 4);
+                    trace_tile(pair_id, it, 1);
                 }
             }
         }
@@ -231,13 +245,13 @@ pair_gemm_kernel(const __grid_constant__ typename Policy::Params p) {
             const typename Policy::Tile tl = Policy::decode(p, tile);
             const int buf = it & 1;
             if (!(ok = wait_bar(smem_u32(&ctl->tmem_full[buf]), (it >> 1) & 1, w, kErrWaitTmemFull))) break;
-            if (threadIdx.x == 64 && cta == 0) trace_mark(pair_id, 5);
+            if (threadIdx.x == 64 && cta == 0) { trace_mark(pair_id, 5); trace_tile(pair_id, it, 2); }
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
             Policy::epilogue(p, tl, cta, row, t_row);
             tc_fence_before_sync();
             mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->tmem_empty[buf]), 0));
-            if (threadIdx.x == 64 && cta == 0) trace_mark(pair_id, 6);
+            if (threadIdx.x == 64 && cta == 0) { trace_mark(pair_id, 6); trace_tile(pair_id, it, 3); }
         }
     }
     pair_teardown(ctl, w);
@@ -431,6 +445,126 @@ __device__ __forceinline__ void carry_row256(float* acc_row, __nv_bfloat16* out,
             st_global_256(out + c * 32 + 16, pk[8], pk[9], pk[10], pk[11], pk[12], pk[13], pk[14], pk[15]);
         }
     }
+}
+
+// The same carried sum with the fp32 traffic done by the TMA unit (one 128-row x 256-column block per CTA).
+// A lane owns one accumulator row, so element-wise accesses from registers are 32 scattered segments per warp
+// instruction; the carried sums are 1 KB per row in, 1 KB out, and on a step with one tile per CTA pair that epilogue
+// took longer than the tile's MMAs.  Here the rows go through two 16 KB staging buffers (128 rows x 32 columns,
+// 128-byte swizzle, conflict-free for row-per-lane accesses) after the pipeline stages:
+//   kind 0  store:     staging -> global (TMA store)
+//   kind 1  add:       staging -> global with an fp32 add performed by the memory system (TMA reduce-add)
+//   kind 2  add+round: global -> staging (TMA loads running ahead of their use), accumulator + carried value
+//                      rounded once to bf16 and stored from registers
+// The tensor map is (H, tokens of one rank, ranks): rows past a rank's end are clipped by the TMA unit on the way out
+// and zero-filled on the way in.  `epi_off` is the byte offset of the control block after the pipeline stages; the
+// staging buffers follow it at +1024.  Called by the 128 epilogue threads of a CTA together (hardware barrier 1).
+struct CarryTma {
+    CUtensorMap map;      // fp32 (H, S_loc, ranks), box (32, 128)
+    uint32_t epi_off;     // 0: not used (element-wise path)
+};
+
+__device__ __forceinline__ void carry_block_tma(const CarryTma& ct, const WaitCtx& w, int kind, int x0, int y0, int z,
+                                                __nv_bfloat16* out_row, uint32_t t_row, int row, bool live) {
+    uint8_t* base = align_1024(dyn_smem()) + ct.epi_off;
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(base);
+    const uint32_t stage = smem_u32(base + 1024);
+    const bool elected = threadIdx.x == 64;
+    const uint32_t my_row = static_cast<uint32_t>(row) * 128u, sw = static_cast<uint32_t>(row) & 7u;
+    if (kind == 2 && elected) {
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            mbar_arrive_expect_tx(smem_u32(&ctl->epi[b]), 16384u);
+            tma_load_3d(stage + b * 16384u, &ct.map, smem_u32(&ctl->epi[b]), x0 + b * 32, y0, z);
+        }
+    }
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+        const uint32_t sbuf = stage + static_cast<uint32_t>(c & 1) * 16384u + my_row;
+        uint32_t v[32];
+        if (kind == 2) {
+            // a failed wait has set the status word; control flow stays uniform so that nobody is left at a barrier
+            (void)wait_bar(smem_u32(&ctl->epi[c & 1]), static_cast<uint32_t>(c >> 1) & 1u, w, kErrWaitFull);
+            uint32_t prev[32];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                ld_shared_v4(sbuf + ((static_cast<uint32_t>(j) ^ sw) << 4), prev[4 * j], prev[4 * j + 1], prev[4 * j + 2],
+                             prev[4 * j + 3]);
+            named_bar_sync(1, kEpilogueThreads);      // everybody has read this buffer
+            if (elected && c + 2 < 8) {
+                mbar_arrive_expect_tx(smem_u32(&ctl->epi[c & 1]), 16384u);
+                tma_load_3d(stage + static_cast<uint32_t>(c & 1) * 16384u, &ct.map, smem_u32(&ctl->epi[c & 1]),
+                            x0 + (c + 2) * 32, y0, z);
+            }
+            tmem_ld32(t_row + c * 32, v);
+            tmem_ld_wait();
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) + __uint_as_float(prev[2 * i]),
+                                    __uint_as_float(v[2 * i + 1]) + __uint_as_float(prev[2 * i + 1]));
+            if (live) {
+                st_global_256(out_row + c * 32, pk[0], pk[1], pk[2], pk[3], pk[4], pk[5], pk[6], pk[7]);
+                st_global_256(out_row + c * 32 + 16, pk[8], pk[9], pk[10], pk[11], pk[12], pk[13], pk[14], pk[15]);
+            }
+        } else {
+            if (c >= 2) {   // the transfer that read this buffer two chunks ago has finished reading it
+                if (elected) bulk_wait_group_read<1>();
+                named_bar_sync(1, kEpilogueThreads);
+            }
+            tmem_ld32(t_row + c * 32, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                st_shared_v4(sbuf + ((static_cast<uint32_t>(j) ^ sw) << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            fence_proxy_async_smem();
+            named_bar_sync(1, kEpilogueThreads);      // the buffer is complete
+            if (elected) {
+                const uint32_t src = stage + static_cast<uint32_t>(c & 1) * 16384u;
+                if (kind == 0) tma_store_3d(&ct.map, src, x0 + c * 32, y0, z);
+                else tma_reduce_add_3d(&ct.map, src, x0 + c * 32, y0, z);
+                bulk_commit_group();
+            }
+        }
+    }
+    if (kind != 2) {   // both buffers free again before the next block (or the end of the kernel)
+        if (elected) bulk_wait_group_read<0>();
+        named_bar_sync(1, kEpilogueThreads);
+    }
+}
+
+// A 128-row x 256-column block of the accumulator written TRANSPOSED (global element [column][row]) by the TMA unit:
+// two staging buffers of 32 columns x 128 rows (512-byte lines, no swizzle: for a fixed column the 32 lanes of a warp
+// write consecutive words).  kind 0 stores, kind 1 adds.  The tensor map is (rows, columns, shards) with boxes (128, 32).
+__device__ __forceinline__ void store_block_tma_transposed(const CUtensorMap* map, uint32_t epi_off, int kind, int x0, int y0,
+                                                           int z, uint32_t t_row, int row) {
+    const uint32_t stage = smem_u32(align_1024(dyn_smem()) + epi_off + 1024);
+    const bool elected = threadIdx.x == 64;
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+        const uint32_t sbuf = stage + static_cast<uint32_t>(c & 1) * 16384u;
+        if (c >= 2) {
+            if (elected) bulk_wait_group_read<1>();
+            named_bar_sync(1, kEpilogueThreads);
+        }
+        uint32_t v[32];
+        tmem_ld32(t_row + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(sbuf + static_cast<uint32_t>(i) * 512u + static_cast<uint32_t>(row) * 4u),
+                         "r"(v[i])
+                         : "memory");
+        fence_proxy_async_smem();
+        named_bar_sync(1, kEpilogueThreads);
+        if (elected) {
+            if (kind == 0) tma_store_3d(map, sbuf, x0, y0 + c * 32, z);
+            else tma_reduce_add_3d(map, sbuf, x0, y0 + c * 32, z);
+            bulk_commit_group();
+        }
+    }
+    if (elected) bulk_wait_group_read<0>();
+    named_bar_sync(1, kEpilogueThreads);
 }
 
 // One accumulator row of a gate|up tile: tensor-memory columns 0..127 hold G, 128..255 hold U; writes
@@ -789,6 +923,7 @@ struct PairDownStagedPolicy {
         CUtensorMap map_a, map_wd;  // A_step (F/D, S, 1) box (64,128); Wd buffers (H, F/D, D) box (64,64)
         float* Yacc;                // [S, H] fp32
         __nv_bfloat16* Y;           // [S, H]
+        CarryTma carry_tma;         // Yacc through the TMA unit (epi_off = 0: element-wise accesses instead)
         int S, H, F_d, D, mode, S_loc;
         int n_shards;               // 0: one ring step of every rank (buffer slot = rank).  n > 0: ONE rank, n consecutive
                                     // ring steps in one launch: A is [S, n * F/D], the weight map holds the n shards in
@@ -831,7 +966,13 @@ struct PairDownStagedPolicy {
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         const bool live = static_cast<int>(cta) * 128 + row < tl.valid;
         const size_t off = static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + tl.nb * 256;
-        carry_row256(p.Yacc + off, p.Y + off, t_row, live, p.mode == 1 || p.mode == 2, p.mode <= 1);
+        if (p.carry_tma.epi_off && p.mode != 3) {
+            WaitCtx w{&reinterpret_cast<SharedCtl*>(align_1024(dyn_smem()) + p.carry_tma.epi_off)->abort, p.status, p.timeout_ns};
+            carry_block_tma(p.carry_tma, w, p.mode, tl.nb * 256, tl.row0 - tl.r * p.S_loc + cta * 128, tl.r, p.Y + off, t_row,
+                            row, live);
+        } else {
+            carry_row256(p.Yacc + off, p.Y + off, t_row, live, p.mode == 1 || p.mode == 2, p.mode <= 1);
+        }
     }
 };
 
@@ -842,6 +983,7 @@ struct PairDxPolicy {
         CUtensorMap map_dg, map_du, map_wg, map_wu;  // boxes (64,128) all
         __nv_bfloat16* dX;
         float* dXacc;  // [S, H] fp32 partial sums carried between launches (one ring step per launch), or null
+        CarryTma carry_tma;  // dXacc through the TMA unit (epi_off = 0: element-wise accesses instead)
         int carry;     // 0: the launch covers all shards, dX stored directly; 1 first, 2 middle, 3 last step of a carried sum
         int linear_shards;  // 1: ONE rank, the D shards of the maps are the ones it meets, in that order (ring-step group)
         int S, H, F, D, F_d, S_loc;
@@ -892,8 +1034,15 @@ struct PairDxPolicy {
                                                        uint32_t t_row, int nb) {
         const size_t off = static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + nb * 256;
         const bool live = static_cast<int>(cta) * 128 + row < tl.valid;
-        if (p.carry == 0) store_bf16_row256(p.dX + off, t_row, live);
-        else carry_row256(p.dXacc + off, p.dX + off, t_row, live, p.carry >= 2, p.carry <= 2);
+        if (p.carry == 0) {
+            store_bf16_row256(p.dX + off, t_row, live);
+        } else if (p.carry_tma.epi_off) {
+            WaitCtx w{&reinterpret_cast<SharedCtl*>(align_1024(dyn_smem()) + p.carry_tma.epi_off)->abort, p.status, p.timeout_ns};
+            carry_block_tma(p.carry_tma, w, p.carry - 1, nb * 256, tl.row0 - tl.r * p.S_loc + cta * 128, tl.r, p.dX + off, t_row,
+                            row, live);
+        } else {
+            carry_row256(p.dXacc + off, p.dX + off, t_row, live, p.carry >= 2, p.carry <= 2);
+        }
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_block(p, tl, cta, row, t_row, tl.nb);
@@ -935,6 +1084,8 @@ struct PairDwPolicy {
         int accumulate;  // 0: dW overwritten; 1: the tile's sum is added to what dW holds (partial sums of other ranks)
         long long out_shard_stride;  // elements between consecutive shards' matrices in each of dWd, dWg, dWu (H * F/D when
                                      // the outputs are the contiguous [D][..][..] arrays)
+        CarryTma carry_tma;          // dWd (H, F/D, D) through the TMA unit (epi_off = 0: element-wise accesses instead)
+        CUtensorMap map_owg, map_owu;  // dWg, dWu (F/D, H, D), boxes (128, 32), written transposed through the TMA unit
         int wide_tiles;
         int tile_base;   // first entry of the tile list this launch covers (a long list is cut into several launches)
         int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
@@ -992,6 +1143,18 @@ struct PairDwPolicy {
                                                       uint32_t t_row, int h_base) {
         const int j = tl.jt * 256 + cta * 128 + row;  // global intermediate index of this lane
         const int F_d = p.F_d;
+        if (p.carry_tma.epi_off) {
+            const int jl0 = tl.jt * 256 + static_cast<int>(cta) * 128 - tl.k * F_d;   // first row of this CTA inside shard k
+            if (tl.which == 0) {
+                WaitCtx w{&reinterpret_cast<SharedCtl*>(align_1024(dyn_smem()) + p.carry_tma.epi_off)->abort, p.status,
+                          p.timeout_ns};
+                carry_block_tma(p.carry_tma, w, p.accumulate ? 1 : 0, h_base, jl0, tl.k, nullptr, t_row, row, true);
+            } else {
+                store_block_tma_transposed(tl.which == 1 ? &p.map_owg : &p.map_owu, p.carry_tma.epi_off, p.accumulate ? 1 : 0,
+                                           jl0, h_base, tl.k, t_row, row);
+            }
+            return;
+        }
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
             uint32_t v[32];

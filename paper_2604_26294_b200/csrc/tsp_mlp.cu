@@ -77,6 +77,8 @@ struct tsp_mlp_plan {
     int dynamic_tiles;          // CTA pairs draw their tiles from a device counter instead of a fixed round-robin
     int fuse_steps;             // per-rank ring steps: gate|up and down projection in one launch
     int ready_parity;           // which of the two ready-counter sets the next fused launch uses
+    int tma_carry;              // carried fp32 sums (Yacc, dXacc) move through the TMA unit
+    int64_t tma_dw_max_tokens;  // weight gradients also go out through the TMA unit up to this many tokens per launch
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
     cudaStream_t host_copy_stream;           // tsp_mlp_forward_host: uploads Wd while the gate|up kernel runs
     cudaEvent_t host_events[8];
@@ -95,14 +97,14 @@ tsp_status_t cuda_fail(tsp_mlp_plan_t* plan, int err) {
 // 3-D bf16 tensor map with 128-byte swizzle: dims (d0 innermost, d1, d2), byte strides of d1 and d2.
 bool encode_map(tsp_mlp_plan_t* plan, CUtensorMap* map, const void* base, CUtensorMapDataType dtype, size_t elem,
                 uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1, uint64_t stride2, uint32_t box0,
-                uint32_t box1) {
+                uint32_t box1, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     cuuint64_t dims[3] = {d0, d1, d2};
     cuuint64_t strides[2] = {stride1, stride2};
     cuuint32_t box[3] = {box0, box1, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     (void)elem;
     CUresult r = plan->encode(map, dtype, 3, const_cast<void*>(base), dims, strides, box, estr,
-                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         plan->last_cuda_error = static_cast<int>(r);
@@ -148,8 +150,13 @@ tsp_status_t check_call(const tsp_mlp_plan_t* plan, int64_t S, int D) {
     return TSP_OK;
 }
 
-int pick_stages(const tsp_mlp_plan_t* plan, size_t stage_bytes, int want) {
-    const size_t fixed = sizeof(tsp::SharedCtl) + 1024;
+// Shared-memory layout of the pair kernels: [stages][1 KB control area: SharedCtl, DynCtl][optional 32 KB of epilogue
+// staging (carried fp32 sums through the TMA unit)], plus 1 KB of slack for the 1024-byte alignment of the base.
+constexpr size_t kCtlAreaBytes = 1024, kEpiStagingBytes = 32 * 1024;
+static_assert(sizeof(tsp::SharedCtl) + sizeof(tsp::DynCtl) <= kCtlAreaBytes, "control area too small");
+
+int pick_stages(const tsp_mlp_plan_t* plan, size_t stage_bytes, int want, size_t extra_fixed = 0) {
+    const size_t fixed = kCtlAreaBytes + 1024 + extra_fixed;
     int s = want;
     while (s > 2 && s * stage_bytes + fixed > static_cast<size_t>(plan->max_smem)) --s;
     return s;
@@ -402,14 +409,39 @@ void fill_common(tsp_mlp_plan_t* plan, Params& p, int num_tiles, int sched_slot 
     p.timeout_ns = plan->timeout_ns;
 }
 
+// Params with a `carry_tma` member may route their carried fp32 sums through the TMA unit: the launch then reserves the
+// staging buffers and tells the kernel where the control block sits (which depends on the stage count chosen here).
+template <class P>
+auto carry_wanted(const P& p, int) -> decltype(p.carry_tma.epi_off, bool()) { return p.carry_tma.epi_off != 0; }
+template <class P>
+bool carry_wanted(const P&, long) { return false; }
+template <class P>
+auto carry_place(P& p, uint32_t off, int) -> decltype(p.carry_tma.epi_off, void()) { p.carry_tma.epi_off = off; }
+template <class P>
+void carry_place(P&, uint32_t, long) {}
+
+// fp32 [ranks][rows][H] accumulator viewed as (H, rows, ranks) with boxes of 32 columns x 128 rows, 128-byte swizzle
+bool encode_carry(tsp_mlp_plan_t* plan, tsp::CarryTma* ct, const float* acc, uint64_t rows_per_rank, uint64_t ranks) {
+    const uint64_t H = plan->H;
+    ct->epi_off = 0;
+    if (!plan->tma_carry || !acc) return true;
+    if (!encode_map(plan, &ct->map, acc, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, H, rows_per_rank, ranks, H * 4,
+                    rows_per_rank * H * 4, 32, 128))
+        return false;
+    ct->epi_off = 1;   // "wanted"; the launch replaces it by the real offset
+    return true;
+}
+
 // Which kernels draw their tiles dynamically (bits of the plan's dynamic_tiles mask).
 constexpr int kDynGate = 1, kDynDown = 2, kDynDx = 4, kDynDw = 8;
 
 template <class Policy>
 tsp_status_t launch_pair_wide(tsp_mlp_plan_t* plan, typename Policy::Params& p, cudaStream_t stream, int kind) {
-    p.stages = pick_stages(plan, tsp::kWideStageBytes, 4);
+    const bool staging = carry_wanted(p, 0);
+    p.stages = pick_stages(plan, tsp::kWideStageBytes, 4, staging ? kEpiStagingBytes : 0);
     const bool dynamic = (plan->dynamic_tiles & kind) != 0;
-    const size_t smem = p.stages * tsp::kWideStageBytes + sizeof(tsp::SharedCtl) + (dynamic ? sizeof(tsp::DynCtl) : 0) + 1024;
+    if (staging) carry_place(p, static_cast<uint32_t>(p.stages * tsp::kWideStageBytes), 0);
+    const size_t smem = p.stages * tsp::kWideStageBytes + kCtlAreaBytes + (staging ? kEpiStagingBytes : 0) + 1024;
     auto kernel = dynamic ? tsp::pair_wide_dyn_kernel<Policy> : tsp::pair_wide_kernel<Policy>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return cuda_fail(plan, e);
@@ -422,8 +454,13 @@ tsp_status_t launch_pair_wide(tsp_mlp_plan_t* plan, typename Policy::Params& p, 
 }
 
 template <class Kernel, class Params>
-tsp_status_t launch_pair_kernel(tsp_mlp_plan_t* plan, Kernel kernel, const Params& p, size_t extra_smem, cudaStream_t stream) {
-    const size_t smem = p.stages * tsp::kPairStageBytes + sizeof(tsp::SharedCtl) + extra_smem + 1024;
+tsp_status_t launch_pair_kernel(tsp_mlp_plan_t* plan, Kernel kernel, Params p, cudaStream_t stream) {
+    const bool staging = carry_wanted(p, 0);
+    if (staging) {
+        p.stages = pick_stages(plan, tsp::kPairStageBytes, p.stages, kEpiStagingBytes);
+        carry_place(p, static_cast<uint32_t>(p.stages * tsp::kPairStageBytes), 0);
+    }
+    const size_t smem = p.stages * tsp::kPairStageBytes + kCtlAreaBytes + (staging ? kEpiStagingBytes : 0) + 1024;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int pairs_avail = plan->sm_count / 2;
@@ -438,8 +475,8 @@ tsp_status_t launch_pair_kernel(tsp_mlp_plan_t* plan, Kernel kernel, const Param
 template <class Policy>
 tsp_status_t launch_pair(tsp_mlp_plan_t* plan, const typename Policy::Params& p, cudaStream_t stream, int kind = kDynGate) {
     if (plan->dynamic_tiles & kind)
-        return launch_pair_kernel(plan, tsp::pair_dyn_kernel<tsp::DynOf<Policy>>, p, sizeof(tsp::DynCtl), stream);
-    return launch_pair_kernel(plan, tsp::pair_gemm_kernel<Policy>, p, 0, stream);
+        return launch_pair_kernel(plan, tsp::pair_dyn_kernel<tsp::DynOf<Policy>>, p, stream);
+    return launch_pair_kernel(plan, tsp::pair_gemm_kernel<Policy>, p, stream);
 }
 
 template <int kMode>
@@ -554,6 +591,7 @@ tsp_status_t launch_bwd_dx_pair(tsp_mlp_plan_t* plan, const void* dG, const void
     p.dX = static_cast<__nv_bfloat16*>(dX);
     p.dXacc = dXacc;
     p.carry = carry;
+    if (carry != 0 && !encode_carry(plan, &p.carry_tma, dXacc, static_cast<uint64_t>(S / D), D)) return TSP_ERR_CUDA;
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D; p.F_d = F_d;
     p.S_loc = static_cast<int>(S / D);
     p.tiles_per_rank = (p.S_loc + 255) / 256;
@@ -591,6 +629,21 @@ tsp_status_t launch_bwd_dw_pair(tsp_mlp_plan_t* plan, const void* X, const void*
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D;
     p.F_d = F / D;
     p.out_shard_stride = static_cast<long long>(H) * p.F_d;
+    // With few tokens the K loop of a tile is shorter than its epilogue (256 KB of fp32 per tile, read and written when
+    // accumulating): the outputs then go through the TMA unit (stores, or adds performed by the memory system).
+    if (plan->tma_carry && S <= plan->tma_dw_max_tokens) {
+        const uint64_t st = static_cast<uint64_t>(p.out_shard_stride) * 4;
+        if (!encode_map(plan, &p.carry_tma.map, dWd, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, H, p.F_d, D, static_cast<uint64_t>(H) * 4,
+                        st, 32, 128))
+            return TSP_ERR_CUDA;
+        if (!encode_map(plan, &p.map_owg, dWg, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.F_d, H, D,
+                        static_cast<uint64_t>(p.F_d) * 4, st, 128, 32, CU_TENSOR_MAP_SWIZZLE_NONE))
+            return TSP_ERR_CUDA;
+        if (!encode_map(plan, &p.map_owu, dWu, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, p.F_d, H, D,
+                        static_cast<uint64_t>(p.F_d) * 4, st, 128, 32, CU_TENSOR_MAP_SWIZZLE_NONE))
+            return TSP_ERR_CUDA;
+        p.carry_tma.epi_off = 1;
+    }
     p.S_loc = static_cast<int>(S / D);
     p.k_linear = (linear || p.S_loc % 64 != 0) ? static_cast<int>((S + 63) / 64) : 0;
     p.j_tiles = F / 256;
@@ -728,6 +781,7 @@ tsp_status_t launch_step_down(tsp_mlp_plan_t* plan, const void* cur_d, const voi
         if (!encode_sharded(plan, &p.map_wd, cur_d, D, F_d, H, 64, 64)) return TSP_ERR_CUDA;
         p.Yacc = Yacc;
         p.Y = static_cast<__nv_bfloat16*>(Y);
+        if (!encode_carry(plan, &p.carry_tma, Yacc, static_cast<uint64_t>(S / D), D)) return TSP_ERR_CUDA;
         p.S = static_cast<int>(S); p.H = H; p.F_d = F_d; p.D = D;
         p.mode = mode;
         p.S_loc = static_cast<int>(S / D);
@@ -788,6 +842,7 @@ tsp_status_t launch_steps_group(tsp_mlp_plan_t* plan, const void* X, const void*
         if (!encode_strided(plan, &p.map_wd, Wd0, n, F_d, H, stride_bytes, 64, 64)) return TSP_ERR_CUDA;
         p.Yacc = Yacc;
         p.Y = static_cast<__nv_bfloat16*>(Y);
+        if (!encode_carry(plan, &p.carry_tma, Yacc, static_cast<uint64_t>(S), 1)) return TSP_ERR_CUDA;
         p.S = static_cast<int>(S); p.H = H; p.F_d = F_d; p.D = 1;
         p.mode = mode;
         p.n_shards = n;
@@ -873,6 +928,7 @@ tsp_status_t launch_steps_group_backward(tsp_mlp_plan_t* plan, const void* X, co
         p.dX = static_cast<__nv_bfloat16*>(dX);
         p.dXacc = dXacc;
         p.carry = carry;
+        if (carry != 0 && !encode_carry(plan, &p.carry_tma, dXacc, static_cast<uint64_t>(S), 1)) return TSP_ERR_CUDA;
         p.linear_shards = 1;
         p.S = static_cast<int>(S); p.H = H; p.F = n * F_d; p.D = n; p.F_d = F_d;
         p.S_loc = static_cast<int>(S);
@@ -885,6 +941,7 @@ tsp_status_t launch_steps_group_backward(tsp_mlp_plan_t* plan, const void* X, co
             p.group = count < group ? count : group;
             p.wide_tiles = mixed_wide_tiles(plan, 2, p.n_blocks, count * p.n_blocks, 2 * n * F_d / 64);
             if (p.wide_tiles > 0) {
+                p.carry_tma.epi_off = 0;   // long K loop: the epilogue is a small part, element-wise accesses do (measured)
                 fill_common(plan, p, count * p.n_blocks - p.wide_tiles);
                 return launch_pair_wide<tsp::PairDxPolicy>(plan, p, cs, kDynDx);
             }
@@ -918,6 +975,7 @@ tsp_status_t launch_steps_fused(tsp_mlp_plan_t* plan, const void* X, const void*
     p.A = static_cast<__nv_bfloat16*>(A);
     p.Yacc = Yacc;
     p.Y = static_cast<__nv_bfloat16*>(Y);
+    if (!encode_carry(plan, &p.carry_tma, Yacc, static_cast<uint64_t>(S), 1)) return TSP_ERR_CUDA;
     p.S_loc = static_cast<int>(S); p.H = H; p.F_d = F_d; p.n_shards = n;
     p.mode = mode;
     p.act = plan->act;
@@ -937,7 +995,7 @@ tsp_status_t launch_steps_fused(tsp_mlp_plan_t* plan, const void* X, const void*
     p.ready_all_target = p.ready_target * p.m_tiles;
     plan->ready_parity ^= 1;
     fill_common(plan, p, p.gate_tiles + p.m_tiles * p.n_blocks);
-    return launch_pair_kernel(plan, tsp::pair_dyn_kernel<Policy>, p, sizeof(tsp::DynCtl), cs);
+    return launch_pair_kernel(plan, tsp::pair_dyn_kernel<Policy>, p, cs);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1013,7 +1071,7 @@ void tsp_mlp_options_default(tsp_mlp_options_t* o) {
     o->struct_bytes = static_cast<uint32_t>(sizeof(tsp_mlp_options_t));
     o->use_pairs = o->gate_band = o->gate_order = o->down_group = o->dx_group = o->dw_group = TSP_OPT_AUTO;
     o->wide_mask = o->pair_stages = o->chunk_bands = o->chunk_tiles = o->dw_chunk_rounds = TSP_OPT_AUTO;
-    o->phase_mask = o->timeout_ms = o->dynamic_tiles = o->fuse_ring_steps = TSP_OPT_AUTO;
+    o->phase_mask = o->timeout_ms = o->dynamic_tiles = o->fuse_ring_steps = o->tma_carry = TSP_OPT_AUTO;
 }
 
 static bool options_valid(const tsp_mlp_options_t* o) {
@@ -1023,7 +1081,8 @@ static bool options_valid(const tsp_mlp_options_t* o) {
            in(o->down_group, 1, 1 << 16) && in(o->dx_group, 1, 1 << 16) && in(o->dw_group, 1, 1 << 16) &&
            in(o->wide_mask, 0, 7) && in(o->pair_stages, 2, tsp::kMaxStages) && in(o->chunk_bands, 0, 1 << 16) &&
            in(o->chunk_tiles, 0, 1 << 20) && in(o->dw_chunk_rounds, 0, 1 << 20) && in(o->phase_mask, 0, 3) &&
-           in(o->timeout_ms, 1, 60000) && in(o->dynamic_tiles, 0, 15) && in(o->fuse_ring_steps, 0, 1);
+           in(o->timeout_ms, 1, 60000) && in(o->dynamic_tiles, 0, 15) && in(o->fuse_ring_steps, 0, 1) &&
+           in(o->tma_carry, 0, 1);
 }
 
 tsp_status_t tsp_mlp_plan_ex(int H, int F, int D, const tsp_mlp_options_t* options, tsp_mlp_plan_t** out) {
@@ -1095,6 +1154,8 @@ static tsp_status_t make_plan(int H, int F, int D, const tsp_mlp_options_t* opt,
     // change costs as much), so two launches stay the default
     plan->fuse_steps = pick(o.fuse_ring_steps, "TSP_MLP_FUSE_STEPS", 0);
     plan->ready_parity = 0;
+    plan->tma_carry = pick(o.tma_carry, "TSP_MLP_TMA_CARRY", 1);
+    plan->tma_dw_max_tokens = pick(TSP_OPT_AUTO, "TSP_MLP_TMA_DW_TOKENS", 4096);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);

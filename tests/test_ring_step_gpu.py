@@ -448,3 +448,46 @@ def test_grouped_backward_argument_errors():
         assert b.tsp_mlp_workspace_bytes_ring_group_backward(plan, S_loc, D + 1) == 0
     finally:
         b.tsp_mlp_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("S_loc,H,F,D", [(1024, 512, 2048, 4), (300, 256, 768, 3), (40, 256, 1024, 4), (2304, 256, 512, 2)])
+def test_carried_sums_through_the_tma_unit_keep_the_bits(S_loc, H, F, D):
+    # The per-step calls carry fp32 partial sums (Yacc, dXacc) from launch to launch.  By default they are stored, added
+    # (by the memory system) and read back through the TMA unit; the plan option selects element-wise accesses from
+    # registers instead.  Either way every step adds once in fp32 round-to-nearest, so the results agree bit for bit,
+    # ragged token counts (rows clipped by the TMA unit) included.
+    import torch
+
+    prob = DeviceProblem(S_loc, H, F, D, seed=40, with_dy=True)
+    outs = {}
+    for tma in (1, 0):
+        plan = b.tsp_mlp_plan_ex(H, F, D, tma_carry=tma)
+        try:
+            nbytes = max(b.tsp_mlp_workspace_bytes_ring(plan, S_loc, b.TSP_WS_BACKWARD),
+                         b.tsp_mlp_workspace_bytes_ring(plan, S_loc, b.TSP_WS_FORWARD))
+            ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+            b.tsp_mlp_set_workspace(plan, ws)
+            Y = torch.full((S_loc, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+            dX = torch.full((S_loc, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+            dW = torch.empty(3 * H * (F // D), dtype=torch.float32, device="cuda")
+            gWg, gWu, gWd = ring.unpack_shard(dW, H, F // D)
+            for rep in range(2):                       # twice: staging buffers and barriers are reused across calls
+                for t in range(D):
+                    b.tsp_mlp_ring_step(plan, prob.X, prob.Wg[t], prob.Wu[t], prob.Wd[t], Y, S_loc, t, D)
+                if (F // D) % 256 == 0:
+                    for t in range(D):          # one accumulator for all shards: written at t = 0, added to afterwards
+                        b.tsp_mlp_ring_step_backward_dx(plan, prob.X, prob.Wg[t], prob.Wu[t], prob.Wd[t], prob.dY, dX, S_loc, t, D)
+                        b.tsp_mlp_ring_step_backward_dw(plan, prob.X, prob.dY, gWg, gWu, gWd, S_loc, int(t > 0), D)
+            torch.cuda.synchronize()
+            assert b.tsp_mlp_status(plan) == b.TSP_OK
+            outs[tma] = (Y, dX, dW)
+        finally:
+            b.tsp_mlp_plan_destroy(plan)
+    assert torch.equal(outs[1][0].view(torch.int16), outs[0][0].view(torch.int16))
+    if (F // D) % 256 == 0:
+        assert torch.equal(outs[1][1].view(torch.int16), outs[0][1].view(torch.int16))
+        assert bool(torch.isfinite(outs[1][2]).all())
+        assert torch.equal(outs[1][2].view(torch.int32), outs[0][2].view(torch.int32))    # weight gradients (sum over shards)
+    # shards were applied in index order 0 .. D-1 here: any order gives the same Y up to rounding
+    ref = orc.gated_mlp_forward(*prob.f64()[:4])
+    assert rel_fro(tensor_to_f64(outs[1][0]), ref) <= TOL_ORACLE
