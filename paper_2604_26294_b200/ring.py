@@ -331,9 +331,9 @@ class TspRingMlp:
         self.plan = b.tsp_mlp_plan(H, F, D)
         if activation is not None:
             b.tsp_mlp_set_activation(self.plan, activation)
-        # ring steps applied per launch in the forward pass (measured on one rank's step sequence at H = 4096,
-        # F/D = 1792: 1024 tokens per rank 746 -> 1030 / 1223 TFLOP/s with 2 / 4 steps per launch; 8192 tokens 1240 -> 1373 /
-        # 1427); more steps per launch also mean more shards in flight (2 g receive buffers)
+        # ring steps applied per group of launches, forward and backward (measured on one rank's step sequence at
+        # H = 4096, F/D = 1792, forward: 1024 tokens per rank 1027 -> 1215 / 1305 TFLOP/s with 2 / 4 steps per launch; 8192
+        # tokens 1277 -> 1452 / 1505); more steps per launch also mean more shards in flight (2 g receive buffers)
         if steps_per_launch is None:
             steps_per_launch = 4 if S_loc <= 2048 else 2
         self.g = max(1, min(steps_per_launch, D))
