@@ -215,11 +215,14 @@ tsp_status_t tsp_mlp_backward_saved(tsp_mlp_plan_t* plan, const void* X, const v
 
 /*
  * tsp_mlp_forward_host - the same forward for callers whose tensors live in HOST
- * memory (pinned memory gives asynchronous copies).  Copies X, Wg, Wu to device
- * staging inside the workspace, runs the gate|up kernel while Wd is still being
- * copied on a plan-owned side stream (created on first use), runs the down projection in four
- * launches over token ranges and copies each range of Y back on the side stream while the next range is
- * computed; ordered with respect to `cuda_stream` (synchronizing it is enough to read Y_host).  Needs a workspace of tsp_mlp_workspace_bytes_host(plan, S) bytes.
+ * memory (pinned memory gives asynchronous copies).  Everything is uploaded on one plan-owned side stream in the
+ * order it is needed - X, then shard by shard Wg_k and Wu_k, then Wd in four blocks of hidden columns - into staging
+ * inside the workspace; the gate|up tiles of shard k are launched on `cuda_stream` as soon as shard k has arrived, the
+ * down projection of a column block as soon as its part of Wd has, and every column block of Y goes back to Y_host on
+ * a second side stream while later uploads are still running.  Same tiles, same K order: Y has the bits of
+ * tsp_mlp_forward.  Ordered with respect to `cuda_stream` (synchronizing it is enough to read Y_host).  Small shapes
+ * (single-CTA path, or H / 256 not a multiple of 8) upload everything first and run the two kernels unsplit.  The side
+ * streams and events are created on first use.  Needs a workspace of tsp_mlp_workspace_bytes_host(plan, S) bytes.
  */
 size_t tsp_mlp_workspace_bytes_host(const tsp_mlp_plan_t* plan, int64_t S);
 tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, const void* Wg_host,

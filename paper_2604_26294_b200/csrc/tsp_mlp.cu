@@ -80,8 +80,10 @@ struct tsp_mlp_plan {
     int tma_carry;              // carried fp32 sums (Yacc, dXacc) move through the TMA unit
     int64_t tma_dw_max_tokens;  // weight gradients also go out through the TMA unit up to this many tokens per launch
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
-    cudaStream_t host_copy_stream;           // tsp_mlp_forward_host: uploads Wd while the gate|up kernel runs
+    cudaStream_t host_copy_stream;           // tsp_mlp_forward_host: uploads (X, then the shards, then Wd by column blocks)
+    cudaStream_t host_down_stream;           // tsp_mlp_forward_host: downloads of Y
     cudaEvent_t host_events[8];
+    std::vector<cudaEvent_t> host_shard_events;   // "shard k has arrived"
     bool host_ready;
 };
 
@@ -515,6 +517,35 @@ tsp_status_t launch_gate_up_pair(tsp_mlp_plan_t* plan, const void* X, const void
     return launch_gate_pair<0>(plan, X, Wg, Wu, A, nullptr, nullptr, nullptr, S, stream);
 }
 
+// The gate|up tiles of ONE shard k for all tokens (the host-buffer forward launches shard by shard, each as soon as its
+// weights have arrived): the same tiles as in the full launch, writing columns k F/D .. of A.
+tsp_status_t launch_gate_up_shard(tsp_mlp_plan_t* plan, const void* X, const void* Wg, const void* Wu, void* A, int k,
+                                  int64_t S, cudaStream_t stream) {
+    using Policy = tsp::PairGateUpPolicyT<0>;
+    const int H = plan->H, F = plan->F, D = plan->D, F_d = F / D;
+    const size_t shard = static_cast<size_t>(H) * F_d * 2;
+    Policy::Params p;
+    std::memset(&p, 0, sizeof(p));
+    if (!encode_matrix(plan, &p.map_x, X, S, H, 64, 128)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wg, static_cast<const uint8_t*>(Wg) + k * shard, 1, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    if (!encode_sharded(plan, &p.map_wu, static_cast<const uint8_t*>(Wu) + k * shard, 1, H, F_d, 64, 64)) return TSP_ERR_CUDA;
+    p.A = static_cast<__nv_bfloat16*>(A) + static_cast<size_t>(k) * F_d;
+    p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = 1; p.F_d = F_d;
+    p.S_loc = static_cast<int>(S / D);
+    p.tiles_per_rank = (p.S_loc + 255) / 256;
+    p.m_tiles = D * p.tiles_per_rank;
+    p.jl_blocks = F_d / 128;
+    p.band = gate_band(plan, p.m_tiles);
+    p.shared_order = 1;
+    p.act = plan->act;
+    return for_tile_chunks(p.m_tiles, plan->chunk_bands * p.band, false, [&](int first, int count) {
+        p.mt_base = first;
+        p.m_tiles = count;
+        fill_common(plan, p, count * p.jl_blocks);
+        return launch_pair<Policy>(plan, p, stream);
+    });
+}
+
 // dA = dY Wd^T (needs F % 256 == 0).  kSaved = false: fp32 dA out; kSaved = true: dG = dA*P, dU = dA*Q out.
 template <bool kSaved>
 tsp_status_t launch_da_pair_t(tsp_mlp_plan_t* plan, const void* dY, const void* Wd, float* dA, const void* P, const void* Q,
@@ -549,19 +580,24 @@ tsp_status_t launch_da_pair(tsp_mlp_plan_t* plan, const void* dY, const void* Wd
 }
 
 // tile_first / tile_count: restrict the launch to a range of token tiles (default: all of them)
+// tile_first / tile_count restrict the launch to a range of token tiles, nb_first / nb_count to a range of 256-column
+// hidden blocks (default: everything); the tiles and their K loops are the same whichever way the work is cut
 tsp_status_t launch_down_pair(tsp_mlp_plan_t* plan, const void* A, const void* Wd, void* Y, int64_t S, cudaStream_t stream,
-                              int tile_first = 0, int tile_count = -1) {
+                              int tile_first = 0, int tile_count = -1, int nb_first = 0, int nb_count = -1) {
     const int H = plan->H, F = plan->F, D = plan->D;
+    if (nb_count < 0) nb_count = H / 256 - nb_first;
     tsp::PairDownPolicy::Params p;
     std::memset(&p, 0, sizeof(p));
     if (!encode_matrix(plan, &p.map_a, A, S, F, 64, 128)) return TSP_ERR_CUDA;
-    if (!encode_matrix(plan, &p.map_wd, Wd, F, H, 64, 64)) return TSP_ERR_CUDA;
-    p.Y = static_cast<__nv_bfloat16*>(Y);
+    if (!encode_block(plan, &p.map_wd, static_cast<const uint8_t*>(Wd) + static_cast<size_t>(nb_first) * 512, F,
+                      static_cast<uint64_t>(nb_count) * 256, H, 64, 64))
+        return TSP_ERR_CUDA;
+    p.Y = static_cast<__nv_bfloat16*>(Y) + static_cast<size_t>(nb_first) * 256;
     p.S = static_cast<int>(S); p.H = H; p.F = F; p.D = D; p.F_d = F / D;
     p.S_loc = static_cast<int>(S / D);
     p.tiles_per_rank = (p.S_loc + 255) / 256;
     p.m_tiles = D * p.tiles_per_rank;
-    p.n_blocks = H / 256;
+    p.n_blocks = nb_count;
     const int group = plan->group > 0 ? plan->group : 8;
     if (tile_count < 0) tile_count = p.m_tiles - tile_first;
     // chunks from the last token tiles to the first: the rows the gate|up kernel wrote last are still in L2
@@ -1181,7 +1217,9 @@ tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan) {
     for (auto& ev : plan->staged_events) cudaEventDestroy(ev);
     if (plan->host_ready) {
         for (auto& ev : plan->host_events) cudaEventDestroy(ev);
+        for (auto& ev : plan->host_shard_events) cudaEventDestroy(ev);
         cudaStreamDestroy(plan->host_copy_stream);
+        cudaStreamDestroy(plan->host_down_stream);
     }
     if (plan->status_dev) cudaFree(plan->status_dev);
     delete plan;
@@ -1265,9 +1303,10 @@ tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, cons
     if (!X_host || !Wg_host || !Wu_host || !Wd_host || !Y_host) return TSP_ERR_INVALID_ARG;
     if (!plan->workspace || plan->workspace_bytes < tsp_mlp_workspace_bytes_host(plan, S)) return TSP_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const size_t a = align_up(static_cast<size_t>(S) * plan->F * 2, 256);
-    const size_t xb = static_cast<size_t>(S) * plan->H * 2, x = align_up(xb, 256);
-    const size_t wb = static_cast<size_t>(plan->H) * plan->F * 2, w = align_up(wb, 256);
+    const int H = plan->H, F = plan->F, F_d = F / D;
+    const size_t a = align_up(static_cast<size_t>(S) * F * 2, 256);
+    const size_t xb = static_cast<size_t>(S) * H * 2, x = align_up(xb, 256);
+    const size_t wb = static_cast<size_t>(H) * F * 2, w = align_up(wb, 256);
     uint8_t* base = static_cast<uint8_t*>(plan->workspace);
     uint8_t* dX = base + a;
     uint8_t* dY = dX + x;
@@ -1275,62 +1314,91 @@ tsp_status_t tsp_mlp_forward_host(tsp_mlp_plan_t* plan, const void* X_host, cons
     uint8_t* dWu = dWg + w;
     uint8_t* dWd = dWu + w;
     cudaError_t e;
-    if (!plan->host_ready) {   // created on first use: a side stream and three events (no device memory)
+    if (!plan->host_ready) {   // created on first use: two side streams and a few events (no device memory)
         if ((e = cudaStreamCreateWithFlags(&plan->host_copy_stream, cudaStreamNonBlocking)) != cudaSuccess)
+            return cuda_fail(plan, e);
+        if ((e = cudaStreamCreateWithFlags(&plan->host_down_stream, cudaStreamNonBlocking)) != cudaSuccess)
             return cuda_fail(plan, e);
         for (auto& ev : plan->host_events)
             if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(plan, e);
         plan->host_ready = true;
     }
-    cudaStream_t side = plan->host_copy_stream;
-    // X, Wg, Wu first: the gate|up kernel needs them; Wd follows on the side stream and arrives while gate|up runs.
-    if ((e = cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
-    if ((e = cudaMemcpyAsync(dWg, Wg_host, wb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
-    if ((e = cudaMemcpyAsync(dWu, Wu_host, wb, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return cuda_fail(plan, e);
+    while (plan->host_shard_events.size() < static_cast<size_t>(D)) {
+        cudaEvent_t ev;
+        if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(plan, e);
+        plan->host_shard_events.push_back(ev);
+    }
+    cudaStream_t up = plan->host_copy_stream, down = plan->host_down_stream;
+    // the staging buffers may still be in use by whatever precedes this call on `stream`
     if ((e = cudaEventRecord(plan->host_events[0], stream)) != cudaSuccess) return cuda_fail(plan, e);
-    if ((e = cudaStreamWaitEvent(side, plan->host_events[0], 0)) != cudaSuccess) return cuda_fail(plan, e);
-    if ((e = cudaMemcpyAsync(dWd, Wd_host, wb, cudaMemcpyHostToDevice, side)) != cudaSuccess) return cuda_fail(plan, e);
-    if ((e = cudaEventRecord(plan->host_events[1], side)) != cudaSuccess) return cuda_fail(plan, e);
-    // The forward proper uses only the first `a` bytes of the workspace.
+    if ((e = cudaStreamWaitEvent(up, plan->host_events[0], 0)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaStreamWaitEvent(down, plan->host_events[0], 0)) != cudaSuccess) return cuda_fail(plan, e);
+
     const int tiles_per_rank = static_cast<int>((S / D + 255) / 256), m_tiles = D * tiles_per_rank;
+    const int n_blocks = H / 256;
     constexpr int kParts = 4;
-    if (!pairs_for_tokens(plan, S) || m_tiles < 2 * kParts || plan->phase_mask != 3) {
-        st = forward_impl(plan, dX, dWg, dWu, dWd, dY, S, D, cuda_stream, plan->host_events[1]);
+    const bool pipelined = pairs_for_tokens(plan, S) && plan->phase_mask == 3 && n_blocks % (2 * kParts) == 0 && m_tiles >= 4;
+    if (!pipelined) {
+        // small or unusual shapes: upload everything, run the two kernels, download Y
+        if ((e = cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(plan, e);
+        if ((e = cudaMemcpyAsync(dWg, Wg_host, wb, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(plan, e);
+        if ((e = cudaMemcpyAsync(dWu, Wu_host, wb, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(plan, e);
+        if ((e = cudaEventRecord(plan->host_events[1], up)) != cudaSuccess) return cuda_fail(plan, e);
+        if ((e = cudaMemcpyAsync(dWd, Wd_host, wb, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(plan, e);
+        if ((e = cudaEventRecord(plan->host_events[2], up)) != cudaSuccess) return cuda_fail(plan, e);
+        if ((e = cudaStreamWaitEvent(stream, plan->host_events[1], 0)) != cudaSuccess) return cuda_fail(plan, e);
+        st = forward_impl(plan, dX, dWg, dWu, dWd, dY, S, D, cuda_stream, plan->host_events[2]);
         if (st != TSP_OK) return st;
         if ((e = cudaMemcpyAsync(Y_host, dY, xb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(plan, e);
         return TSP_OK;
     }
-    // The down projection runs in kParts launches over token ranges, last range first; each range of Y goes back to the
-    // host on the side stream while the next range is computed.
-    auto row_of = [&](int mt) {
-        const int64_t r = mt / tiles_per_rank, j = mt % tiles_per_rank;
-        const int64_t row = r * (S / D) + j * 256;
-        return row < S ? row : S;
-    };
+    // Uploads in the order they are needed, all on one stream (the link is the bottleneck): X, then shard by shard
+    // Wg_k and Wu_k, then Wd in kParts blocks of hidden columns.  The gate|up tiles of shard k are launched as soon as
+    // shard k is on the device, the down projection of a column block as soon as its part of Wd is, and every block of
+    // Y goes back on a third stream while later uploads are still running (the link is full duplex).
+    const size_t shard_bytes = static_cast<size_t>(H) * F_d * 2;
+    if ((e = cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(plan, e);
+    for (int k = 0; k < D; ++k) {
+        if ((e = cudaMemcpyAsync(dWg + k * shard_bytes, static_cast<const uint8_t*>(Wg_host) + k * shard_bytes, shard_bytes,
+                                 cudaMemcpyHostToDevice, up)) != cudaSuccess)
+            return cuda_fail(plan, e);
+        if ((e = cudaMemcpyAsync(dWu + k * shard_bytes, static_cast<const uint8_t*>(Wu_host) + k * shard_bytes, shard_bytes,
+                                 cudaMemcpyHostToDevice, up)) != cudaSuccess)
+            return cuda_fail(plan, e);
+        if ((e = cudaEventRecord(plan->host_shard_events[k], up)) != cudaSuccess) return cuda_fail(plan, e);
+    }
+    const int nb_per = n_blocks / kParts;
+    const size_t col_bytes = static_cast<size_t>(nb_per) * 256 * 2, pitch = static_cast<size_t>(H) * 2;
+    for (int q = 0; q < kParts; ++q) {
+        if ((e = cudaMemcpy2DAsync(dWd + q * col_bytes, pitch, static_cast<const uint8_t*>(Wd_host) + q * col_bytes, pitch,
+                                   col_bytes, static_cast<size_t>(F), cudaMemcpyHostToDevice, up)) != cudaSuccess)
+            return cuda_fail(plan, e);
+        if ((e = cudaEventRecord(plan->host_events[1 + q], up)) != cudaSuccess) return cuda_fail(plan, e);
+    }
     plan->launch_count = 0;
     Profiler prof(plan, stream);
-    st = launch_gate_up_pair(plan, dX, dWg, dWu, plan->workspace, S, stream);
-    if (st != TSP_OK) return st;
-    prof.mark();
-    if ((e = cudaStreamWaitEvent(stream, plan->host_events[1], 0)) != cudaSuccess) return cuda_fail(plan, e);   // Wd has arrived
-    const int per = m_tiles / kParts;
-    for (int q = kParts - 1; q >= 0; --q) {
-        const int first = q * per, count = q == kParts - 1 ? m_tiles - first : per;
-        st = launch_down_pair(plan, plan->workspace, dWd, dY, S, stream, first, count);
+    for (int k = 0; k < D; ++k) {
+        if ((e = cudaStreamWaitEvent(stream, plan->host_shard_events[k], 0)) != cudaSuccess) return cuda_fail(plan, e);
+        st = launch_gate_up_shard(plan, dX, dWg, dWu, plan->workspace, k, S, stream);
         if (st != TSP_OK) return st;
-        const int64_t r0 = row_of(first), r1 = q == kParts - 1 ? S : row_of(first + count);
-        cudaEvent_t ev = plan->host_events[3 + q];
+    }
+    prof.mark();
+    for (int q = 0; q < kParts; ++q) {
+        if ((e = cudaStreamWaitEvent(stream, plan->host_events[1 + q], 0)) != cudaSuccess) return cuda_fail(plan, e);
+        st = launch_down_pair(plan, plan->workspace, dWd, dY, S, stream, 0, -1, q * nb_per, nb_per);
+        if (st != TSP_OK) return st;
+        cudaEvent_t ev = plan->host_events[5];          // reused: the download stream has waited for it before the next record
         if ((e = cudaEventRecord(ev, stream)) != cudaSuccess) return cuda_fail(plan, e);
-        if ((e = cudaStreamWaitEvent(side, ev, 0)) != cudaSuccess) return cuda_fail(plan, e);
-        const size_t off = static_cast<size_t>(r0) * plan->H * 2, len = static_cast<size_t>(r1 - r0) * plan->H * 2;
-        if ((e = cudaMemcpyAsync(static_cast<uint8_t*>(Y_host) + off, dY + off, len, cudaMemcpyDeviceToHost, side)) != cudaSuccess)
+        if ((e = cudaStreamWaitEvent(down, ev, 0)) != cudaSuccess) return cuda_fail(plan, e);
+        if ((e = cudaMemcpy2DAsync(static_cast<uint8_t*>(Y_host) + q * col_bytes, pitch, dY + q * col_bytes, pitch, col_bytes,
+                                   static_cast<size_t>(S), cudaMemcpyDeviceToHost, down)) != cudaSuccess)
             return cuda_fail(plan, e);
     }
     prof.mark();
     plan->last_forward_kernels = plan->launch_count;
-    // the caller synchronizes `stream`: make it wait for the copies on the side stream
-    if ((e = cudaEventRecord(plan->host_events[2], side)) != cudaSuccess) return cuda_fail(plan, e);
-    if ((e = cudaStreamWaitEvent(stream, plan->host_events[2], 0)) != cudaSuccess) return cuda_fail(plan, e);
+    // the caller synchronizes `stream`: make it wait for the downloads
+    if ((e = cudaEventRecord(plan->host_events[6], down)) != cudaSuccess) return cuda_fail(plan, e);
+    if ((e = cudaStreamWaitEvent(stream, plan->host_events[6], 0)) != cudaSuccess) return cuda_fail(plan, e);
     return TSP_OK;
 }
 
