@@ -110,10 +110,19 @@ tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan);
  *   tma_carry        1 (auto): the fp32 partial sums that the per-step calls carry from launch to launch (Yacc, dXacc)
  *                    are stored, added and read back by the TMA unit through shared-memory staging; 0: element-wise
  *                    accesses from registers.  Same arithmetic (one fp32 round-to-nearest add per step).
+ *   rank_pair_tiles  bit 0 down projection, bit 1 dX: when a rank owns at most 8 token tiles (S/D <= 2048), D is even
+ *                    and the whole problem is one launch, tiles hold the same 256 token rows of TWO neighbouring
+ *                    ranks.  Rank 2q meets the shards in the order of rank 2q+1 shifted by one ring step, so one
+ *                    loaded weight panel serves both ranks (each in its own step), which halves the weight traffic
+ *                    into shared memory.  Every rank still adds its D partial products in ring order: same bits.
+ *                    As many whole rounds of the CTA pairs as fit without adding a time unit run as two-rank tiles,
+ *                    the rest as one-rank tiles; bit 2 makes every position a two-rank tile (tests, sweeps).
+ *                    0: one-rank tiles only.  Needs the dynamic hand-out of the kernel (dynamic_tiles).
+ *                    Auto: 2 (dX only; measured slower for the down projection), 0 when wide_mask is given.
  * Environment variables of the same meaning (TSP_MLP_PAIR, TSP_MLP_BAND, TSP_MLP_GATE_ORDER, TSP_MLP_GROUP,
  * TSP_MLP_DX_GROUP, TSP_MLP_DW_GROUP, TSP_MLP_WIDE, TSP_MLP_PAIR_STAGES, TSP_MLP_CHUNK_BANDS, TSP_MLP_CHUNK_TILES,
  * TSP_MLP_DW_CHUNK_ROUNDS (negative = one launch), TSP_MLP_PHASES, TSP_MLP_TIMEOUT_MS, TSP_MLP_DYNAMIC,
- * TSP_MLP_FUSE_STEPS, TSP_MLP_TMA_CARRY) are read
+ * TSP_MLP_FUSE_STEPS, TSP_MLP_TMA_CARRY, TSP_MLP_RANK_PAIRS) are read
  * when a plan is created and fill only the fields the caller left at TSP_OPT_AUTO: an explicit option wins.
  * struct_bytes must be sizeof(tsp_mlp_options_t) as the caller was compiled (tsp_mlp_options_default sets it);
  * a different size is refused with INVALID_ARG, as is a field outside its range.
@@ -137,6 +146,7 @@ typedef struct {
     int dynamic_tiles;
     int fuse_ring_steps;
     int tma_carry;
+    int rank_pair_tiles;
 } tsp_mlp_options_t;
 void tsp_mlp_options_default(tsp_mlp_options_t* options);
 /* tsp_mlp_plan with options (NULL options = tsp_mlp_plan).  Errors as tsp_mlp_plan. */

@@ -7,7 +7,7 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 SOURCES = [os.path.join(HERE, "csrc", "tsp_mlp.cu")]
-HEADERS = [os.path.join(HERE, "csrc", n) for n in ("ptx.cuh", "gemm_core.cuh", "fwd_kernels.cuh", "bwd_kernels.cuh", "dyn_kernels.cuh",
+HEADERS = [os.path.join(HERE, "csrc", n) for n in ("ptx.cuh", "gemm_core.cuh", "fwd_kernels.cuh", "bwd_kernels.cuh", "dyn_kernels.cuh", "skew_kernels.cuh",
                                                    "pair_kernels.cuh", "attn_kernels.cuh", "tsp_attn_host.cuh")]
 HEADERS += [os.path.join(os.path.dirname(HERE), "include", n) for n in ("tsp_mlp.h", "tsp_attn.h")]
 LIB = os.path.join(HERE, "libtsp_mlp.so")

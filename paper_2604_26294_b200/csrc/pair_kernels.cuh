@@ -847,6 +847,7 @@ struct PairDownPolicy {
         int S, H, F, D, F_d, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;   // mixed-width kernel: number of 256 x 512 tiles at the head of the tile list
+        int skew_tiles;   // two-rank kernel: number of tall tiles (both ranks of a pair) at the head of the tile list
         int mt_base;  // first token tile of this launch (a long problem is cut into several launches)
         int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
@@ -886,6 +887,13 @@ struct PairDownPolicy {
         const int f0 = k * p.F_d + i * kBK;
         pair_load_kmajor(sa, &p.map_a, bar, f0, tl.row0 + cta * 128, 0);
         pair_load_mnmajor(sb, &p.map_wd, bar, tl.nb * 256 + cta * 128, f0, 0, 2);
+    }
+    // the two operands separately (two-rank kernel): `row` is this CTA's first token row
+    __device__ static __forceinline__ void load_a(const Params& p, int row, int k, int i, uint32_t, uint32_t sa, uint32_t bar) {
+        pair_load_kmajor(sa, &p.map_a, bar, k * p.F_d + i * kBK, row, 0);
+    }
+    __device__ static __forceinline__ void load_b(const Params& p, int nb, int k, int i, uint32_t cta, uint32_t sb, uint32_t bar) {
+        pair_load_mnmajor(sb, &p.map_wd, bar, nb * 256 + cta * 128, k * p.F_d + i * kBK, 0, 2);
     }
     __device__ static __forceinline__ void epilogue(const Params& p, const Tile& tl, uint32_t cta, int row, uint32_t t_row) {
         store_bf16_row256(p.Y + static_cast<size_t>(tl.row0 + cta * 128 + row) * p.H + tl.nb * 256, t_row,
@@ -989,6 +997,7 @@ struct PairDxPolicy {
         int S, H, F, D, F_d, S_loc;
         int m_tiles, n_blocks, tiles_per_rank, group;
         int wide_tiles;
+        int skew_tiles;   // two-rank kernel: number of tall tiles at the head of the tile list
         int mt_base;   // first token tile of this launch
         int* sched;   // dynamic tile hand-out: {next list index, leaders done} in global memory (unused by the static kernels)
         int num_tiles, stages;
@@ -1029,6 +1038,13 @@ struct PairDxPolicy {
         const bool up = i & 1;
         pair_load_kmajor(sa, up ? &p.map_du : &p.map_dg, bar, k * p.F_d + j0, tl.row0 + cta * 128, 0);
         pair_load_kmajor(sb, up ? &p.map_wu : &p.map_wg, bar, j0, tl.nb * 256 + cta * 128, k);
+    }
+    // the two operands separately (two-rank kernel): `row` is this CTA's first token row
+    __device__ static __forceinline__ void load_a(const Params& p, int row, int k, int i, uint32_t, uint32_t sa, uint32_t bar) {
+        pair_load_kmajor(sa, (i & 1) ? &p.map_du : &p.map_dg, bar, k * p.F_d + (i >> 1) * kBK, row, 0);
+    }
+    __device__ static __forceinline__ void load_b(const Params& p, int nb, int k, int i, uint32_t cta, uint32_t sb, uint32_t bar) {
+        pair_load_kmajor(sb, (i & 1) ? &p.map_wu : &p.map_wg, bar, (i >> 1) * kBK, nb * 256 + cta * 128, k);
     }
     __device__ static __forceinline__ void store_block(const Params& p, const Tile& tl, uint32_t cta, int row,
                                                        uint32_t t_row, int nb) {

@@ -87,6 +87,9 @@ def test_plan_options_defaults_and_validation(lib):
     o.timeout_ms = 0
     assert lib.tsp_mlp_plan_ex(256, 768, 2, ctypes.byref(o), ctypes.byref(out)) == b.TSP_ERR_INVALID_ARG
     o = b.tsp_mlp_options_default()
+    o.rank_pair_tiles = 8
+    assert lib.tsp_mlp_plan_ex(256, 768, 2, ctypes.byref(o), ctypes.byref(out)) == b.TSP_ERR_INVALID_ARG
+    o = b.tsp_mlp_options_default()
     assert lib.tsp_mlp_plan_ex(128, 768, 2, ctypes.byref(o), ctypes.byref(out)) == b.TSP_ERR_UNSUPPORTED_SHAPE
     assert not out.value
     with pytest.raises(TypeError):
