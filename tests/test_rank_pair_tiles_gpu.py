@@ -51,8 +51,9 @@ def _same_bits(a, c):
 
 
 # every position a two-rank tile (option bit 2); D = 2 is the shortest ring (three slots), the third shape has two
-# token tiles per rank, the last one an 8-rank ring
-@pytest.mark.parametrize("S,H,F,D", [(512, 512, 1024, 2), (1024, 256, 1536, 4), (2048, 256, 1536, 4), (2048, 512, 2048, 8)])
+# token tiles per rank, the fourth an 8-rank ring, the last a ragged last token tile per rank (1000 tokens = 3 tiles + 232 rows)
+@pytest.mark.parametrize("S,H,F,D", [(512, 512, 1024, 2), (1024, 256, 1536, 4), (2048, 256, 1536, 4), (2048, 512, 2048, 8),
+                                     (4000, 256, 1536, 4)])
 def test_two_rank_tiles_keep_every_bit_and_match_the_oracle(S, H, F, D):
     prob = DeviceProblem(S, H, F, D, seed=61, with_dy=True)
     one_rank = _run(prob, reps=1, rank_pair_tiles=0)[0]
