@@ -1250,8 +1250,8 @@ static tsp_status_t make_plan(int H, int F, int D, const tsp_mlp_options_t* opt,
     plan->tma_carry = pick(o.tma_carry, "TSP_MLP_TMA_CARRY", 1);
     plan->tma_dw_max_tokens = pick(TSP_OPT_AUTO, "TSP_MLP_TMA_DW_TOKENS", 4096);
     // measured (S = 8192, D = 8, 7B shapes): two-rank tiles cut the DRAM reads of dX from 2.7 to 2.0 GB and gain 0.7-0.9 %
-    // on a training step; for the down projection they lose 1.3 % against the mixed-width list (their first and last
-    // slot run at half rate with less data in flight), so only dX takes them.  A caller who forces a tile width gets it.
+    // on a training step; for the down projection they lose 1.3 % against the mixed-width list, so only dX takes them.
+    // A caller who forces a tile width gets it.
     plan->rank_pair_tiles = pick(o.rank_pair_tiles, "TSP_MLP_RANK_PAIRS", plan->wide_mask >= 0 ? 0 : 2);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
