@@ -119,10 +119,15 @@ tsp_status_t tsp_mlp_plan_destroy(tsp_mlp_plan_t* plan);
  *                    the rest as one-rank tiles; bit 2 makes every position a two-rank tile (tests, sweeps).
  *                    0: one-rank tiles only.  Needs the dynamic hand-out of the kernel (dynamic_tiles).
  *                    Auto: 2 (dX only; measured slower for the down projection), 0 when wide_mask is given.
+ *   overlap_launches 1 (auto): the CTA-pair kernels are launched with programmatic stream serialisation: a kernel's
+ *                    CTAs may start while the previous kernel of the stream is finishing, set up their barriers and
+ *                    tensor memory, and wait on the device for the previous grid to complete (and its writes to be
+ *                    visible) before their first access to global memory.  Hides the launch gap and the set-up at
+ *                    every kernel boundary; results are the same.  0: ordinary launches.
  * Environment variables of the same meaning (TSP_MLP_PAIR, TSP_MLP_BAND, TSP_MLP_GATE_ORDER, TSP_MLP_GROUP,
  * TSP_MLP_DX_GROUP, TSP_MLP_DW_GROUP, TSP_MLP_WIDE, TSP_MLP_PAIR_STAGES, TSP_MLP_CHUNK_BANDS, TSP_MLP_CHUNK_TILES,
  * TSP_MLP_DW_CHUNK_ROUNDS (negative = one launch), TSP_MLP_PHASES, TSP_MLP_TIMEOUT_MS, TSP_MLP_DYNAMIC,
- * TSP_MLP_FUSE_STEPS, TSP_MLP_TMA_CARRY, TSP_MLP_RANK_PAIRS) are read
+ * TSP_MLP_FUSE_STEPS, TSP_MLP_TMA_CARRY, TSP_MLP_RANK_PAIRS, TSP_MLP_OVERLAP_LAUNCHES) are read
  * when a plan is created and fill only the fields the caller left at TSP_OPT_AUTO: an explicit option wins.
  * struct_bytes must be sizeof(tsp_mlp_options_t) as the caller was compiled (tsp_mlp_options_default sets it);
  * a different size is refused with INVALID_ARG, as is a field outside its range.
@@ -147,6 +152,7 @@ typedef struct {
     int fuse_ring_steps;
     int tma_carry;
     int rank_pair_tiles;
+    int overlap_launches;
 } tsp_mlp_options_t;
 void tsp_mlp_options_default(tsp_mlp_options_t* options);
 /* tsp_mlp_plan with options (NULL options = tsp_mlp_plan).  Errors as tsp_mlp_plan. */

@@ -164,7 +164,7 @@ class TspMlpOptions(ctypes.Structure):
 
     _fields_ = [("struct_bytes", ctypes.c_uint32)] + [(n, ctypes.c_int) for n in (
         "use_pairs", "gate_band", "gate_order", "down_group", "dx_group", "dw_group", "wide_mask", "pair_stages",
-        "chunk_bands", "chunk_tiles", "dw_chunk_rounds", "phase_mask", "timeout_ms", "dynamic_tiles", "fuse_ring_steps", "tma_carry", "rank_pair_tiles")]
+        "chunk_bands", "chunk_tiles", "dw_chunk_rounds", "phase_mask", "timeout_ms", "dynamic_tiles", "fuse_ring_steps", "tma_carry", "rank_pair_tiles", "overlap_launches")]
 
 
 def tsp_mlp_options_default() -> TspMlpOptions:

@@ -67,13 +67,16 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
                  : "memory");
 }
 
-// Timeline probes for development builds (-DTSP_TRACE): eight time stamps per CTA pair of the last launch.
+// Timeline probes for development builds (-DTSP_TRACE=2): eight time stamps per CTA pair of the last launch;
+// -DTSP_TRACE=1 keeps only kernel entry, last epilogue end and exit (slots 0, 6, 7), which do not touch the MMA lane's loop.
 #ifdef TSP_TRACE
 __device__ unsigned long long* g_trace = nullptr;
 __device__ __forceinline__ void trace_mark(int pair_id, int slot) {
+    if (TSP_TRACE < 2 && slot != 0 && slot != 6 && slot != 7) return;
     if (g_trace) g_trace[pair_id * 8 + slot] = global_timer_ns();
 }
 __device__ __forceinline__ void trace_tile(int pair_id, int it, int k) {
+    if (TSP_TRACE < 2) return;
     if (g_trace && it < 16) g_trace[74 * 8 + pair_id * 64 + it * 4 + k] = global_timer_ns();
 }
 #else
@@ -137,6 +140,12 @@ __device__ __forceinline__ void pair_setup(SharedCtl* ctl, int stages, int n_acc
     tc_fence_before_sync();
     cluster_sync_all();
     tc_fence_after_sync();
+    // Everything above touched only this CTA's shared and tensor memory, so it may run while the previous kernel of the
+    // stream is still finishing (the host launches the pair kernels with programmatic serialisation).  From here on
+    // the kernel reads and writes global memory: wait for the previous grid, then let the next one start its own set-up
+    // under this kernel's tail.  The trigger comes after the wait, so at most two kernels overlap.
+    griddep_wait();
+    griddep_launch_dependents();
 }
 
 __device__ __forceinline__ void pair_teardown(SharedCtl* ctl, const WaitCtx& w) {

@@ -84,6 +84,11 @@ __device__ __forceinline__ void bulk_wait_group_read() {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 // Barrier among `count` threads of the CTA (a multiple of 32) on hardware barrier `id` (1..15; 0 is __syncthreads).
+// Programmatic dependent launch.  wait: blocks until every grid this one was allowed to start ahead of has completed
+// and its memory operations are visible (returns at once for an ordinary launch).  launch_dependents: lets the next
+// kernel of the stream, if it was launched with programmatic serialisation, start its CTAs as soon as SMs are free.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }

@@ -80,6 +80,7 @@ struct tsp_mlp_plan {
     int ready_parity;           // which of the two ready-counter sets the next fused launch uses
     int tma_carry;              // carried fp32 sums (Yacc, dXacc) move through the TMA unit
     int rank_pair_tiles;        // bit 0 down, bit 1 dX: tiles of two neighbouring ranks share their weight panels
+    int overlap_launches;       // pair kernels are launched with programmatic serialisation
     int64_t tma_dw_max_tokens;  // weight gradients also go out through the TMA unit up to this many tokens per launch
     std::vector<cudaEvent_t> staged_events;  // 2 per ring step: "shards received", "step computed"
     cudaStream_t host_copy_stream;           // tsp_mlp_forward_host: uploads (X, then the shards, then Wd by column blocks)
@@ -436,6 +437,26 @@ bool encode_carry(tsp_mlp_plan_t* plan, tsp::CarryTma* ct, const float* acc, uin
     return true;
 }
 
+// Launch of a CTA-pair kernel.  With `overlap_launches` the launch carries the programmatic-serialisation attribute:
+// its CTAs may become resident while the previous kernel of the stream is finishing, run their set-up (barriers,
+// tensor-memory allocation, cluster sync) and then wait, on the device, for the previous grid to complete before they
+// touch global memory (pair_setup).  After anything that is not such a kernel the launch is ordered as usual.
+template <class Kernel, class Params>
+cudaError_t launch_pairs(const tsp_mlp_plan_t* plan, Kernel kernel, int pairs, size_t smem, cudaStream_t stream,
+                         const Params& p) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(tsp::kNumThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = plan->overlap_launches ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 // Which kernels draw their tiles dynamically (bits of the plan's dynamic_tiles mask).
 constexpr int kDynGate = 1, kDynDown = 2, kDynDx = 4, kDynDw = 8;
 
@@ -451,9 +472,9 @@ tsp_status_t launch_pair_wide(tsp_mlp_plan_t* plan, typename Policy::Params& p, 
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int pairs_avail = plan->sm_count / 2;
     const int pairs = p.num_tiles < pairs_avail ? p.num_tiles : pairs_avail;
-    kernel<<<2 * pairs, tsp::kNumThreads, smem, stream>>>(p);
+    e = launch_pairs(plan, kernel, pairs, smem, stream, p);
     ++plan->launch_count;
-    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
 
@@ -489,9 +510,9 @@ tsp_status_t launch_pair_skew(tsp_mlp_plan_t* plan, typename Policy::Params& p, 
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int pairs_avail = plan->sm_count / 2;
     const int pairs = p.num_tiles < pairs_avail ? p.num_tiles : pairs_avail;
-    kernel<<<2 * pairs, tsp::kNumThreads, smem, stream>>>(p);
+    e = launch_pairs(plan, kernel, pairs, smem, stream, p);
     ++plan->launch_count;
-    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
 
@@ -507,9 +528,9 @@ tsp_status_t launch_pair_kernel(tsp_mlp_plan_t* plan, Kernel kernel, Params p, c
     if (e != cudaSuccess) return cuda_fail(plan, e);
     const int pairs_avail = plan->sm_count / 2;
     const int pairs = p.num_tiles < pairs_avail ? p.num_tiles : pairs_avail;
-    kernel<<<2 * pairs, tsp::kNumThreads, smem, stream>>>(p);
+    e = launch_pairs(plan, kernel, pairs, smem, stream, p);
     ++plan->launch_count;
-    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? TSP_OK : cuda_fail(plan, e);
 }
 
@@ -1164,7 +1185,7 @@ void tsp_mlp_options_default(tsp_mlp_options_t* o) {
     o->use_pairs = o->gate_band = o->gate_order = o->down_group = o->dx_group = o->dw_group = TSP_OPT_AUTO;
     o->wide_mask = o->pair_stages = o->chunk_bands = o->chunk_tiles = o->dw_chunk_rounds = TSP_OPT_AUTO;
     o->phase_mask = o->timeout_ms = o->dynamic_tiles = o->fuse_ring_steps = o->tma_carry = TSP_OPT_AUTO;
-    o->rank_pair_tiles = TSP_OPT_AUTO;
+    o->rank_pair_tiles = o->overlap_launches = TSP_OPT_AUTO;
 }
 
 static bool options_valid(const tsp_mlp_options_t* o) {
@@ -1175,7 +1196,7 @@ static bool options_valid(const tsp_mlp_options_t* o) {
            in(o->wide_mask, 0, 7) && in(o->pair_stages, 2, tsp::kMaxStages) && in(o->chunk_bands, 0, 1 << 16) &&
            in(o->chunk_tiles, 0, 1 << 20) && in(o->dw_chunk_rounds, 0, 1 << 20) && in(o->phase_mask, 0, 3) &&
            in(o->timeout_ms, 1, 60000) && in(o->dynamic_tiles, 0, 15) && in(o->fuse_ring_steps, 0, 1) &&
-           in(o->tma_carry, 0, 1) && in(o->rank_pair_tiles, 0, 7);
+           in(o->tma_carry, 0, 1) && in(o->rank_pair_tiles, 0, 7) && in(o->overlap_launches, 0, 1);
 }
 
 tsp_status_t tsp_mlp_plan_ex(int H, int F, int D, const tsp_mlp_options_t* options, tsp_mlp_plan_t** out) {
@@ -1252,6 +1273,7 @@ static tsp_status_t make_plan(int H, int F, int D, const tsp_mlp_options_t* opt,
     // measured (S = 8192, D = 8, 7B shapes): two-rank tiles cut the DRAM reads of dX from 2.7 to 2.0 GB and gain 0.7-0.9 %
     // on a training step; for the down projection they lose 1.3 % against the mixed-width list, so only dX takes them.
     // A caller who forces a tile width gets it.
+    plan->overlap_launches = pick(o.overlap_launches, "TSP_MLP_OVERLAP_LAUNCHES", 1);
     plan->rank_pair_tiles = pick(o.rank_pair_tiles, "TSP_MLP_RANK_PAIRS", plan->wide_mask >= 0 ? 0 : 2);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
